@@ -1,0 +1,203 @@
+/*
+ * thinfer.h - C ABI of the B200 (sm_100a) FP16 Llama-style decoder forward.
+ *
+ * The library runs the two phases of the paper's Prefill-Buffer-Decode pipeline
+ * (Section 3.4.2) for one decoder layer or a stack of them on ONE GPU:
+ *
+ *   prefill  dense projections on tcgen05 tensor cores + causal attention
+ *            (Eq. 6, the staged attention of Section 3.3.2)
+ *   decode   one token per request: weight-streaming GEMV / skinny GEMM
+ *            (the small-M path of Section 3.2.2) + attention over the FP16
+ *            KV cache, with the density-driven fusion units of Section 3.3.1:
+ *            RMSNorm -> QKV -> RoPE + cache append (Algorithm 1), attention,
+ *            O-projection + residual, RMSNorm -> gate/up -> SwiGLU,
+ *            down-projection + residual.
+ *
+ * Conventions
+ *   - Plain C.  No exception or abort crosses the boundary.  Every call
+ *     returns 0 (THINFER_OK) or a negative thinfer_err; thinfer_last_error()
+ *     gives a text for the most recent failure of a context.
+ *   - "device" pointers are CUDA device memory of the current device, owned by
+ *     the caller, 256-byte aligned unless stated otherwise.  "host" pointers
+ *     are ordinary host memory.  The library allocates no device memory except
+ *     one pinned, host-mapped status word per context.
+ *   - Arguments are validated on the host before anything is enqueued.
+ *     Compute is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream) and the call returns without
+ *     synchronising.  Calls on one context must be issued from one thread at
+ *     a time; work of one context must stay ordered on the device (use one
+ *     stream, or order the streams with events).
+ *   - Storage is IEEE FP16, accumulation and the norm / softmax reductions are
+ *     FP32 (Section 3.2.4).  Matrices are row-major [out, in] (the paper's
+ *     Y = X W, Section 3.2.1, with W stored transposed so that the contraction
+ *     index is contiguous for both operands).
+ *   - Device-side waits are bounded: a pipeline that does not make progress
+ *     writes THINFER_ETIMEOUT to the status word and the kernel returns.
+ */
+#ifndef THINFER_H
+#define THINFER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  THINFER_OK = 0,
+  THINFER_EINVAL = -1,       /* NULL pointer, bad size, bad slot, wrong mode      */
+  THINFER_EUNSUPPORTED = -2, /* shape outside what the kernels cover              */
+  THINFER_ECAPACITY = -3,    /* batch > max_batch, or the sequence would exceed max_seq, or a workspace is too small */
+  THINFER_EBUSY = -4,        /* prefill into a slot that has not been released (back-pressure, Section 3.4.2) */
+  THINFER_ECUDA = -5,        /* a CUDA runtime / driver call failed               */
+  THINFER_ETIMEOUT = -6      /* a bounded device-side wait expired                */
+} thinfer_err;
+
+typedef struct thinfer_ctx thinfer_ctx; /* opaque host object */
+
+/* Layer shapes (Section 4.1: Llama-2 family).  Supported: head_dim 64 or 128;
+ * n_q_heads a multiple of n_kv_heads; hidden, ffn and n_q_heads*head_dim
+ * multiples of 8; max_batch <= 64 (decode rows); max_seq >= 1. */
+typedef struct {
+  int32_t hidden, n_q_heads, n_kv_heads, head_dim, ffn, n_layers;
+  int32_t vocab;      /* 0: layer-only mode, hidden states in and out; > 0: token ids in, next ids / logits out */
+  float rms_eps;      /* inside the square root */
+  float rope_base;    /* angle of pair j at position p = p * rope_base^(-2j/head_dim) */
+  int32_t max_batch;  /* requests per slot */
+  int32_t max_seq;    /* KV positions per request */
+  int32_t buf_slots;  /* Buf_max: number of KV slots in the bounded buffer, >= 1 */
+} thinfer_config;
+
+/* Device pointers, FP16, caller-owned, read-only, must outlive the context.
+ * Norm gains are [hidden]; wq [n_q_heads*head_dim, hidden]; wk, wv
+ * [n_kv_heads*head_dim, hidden]; wo [hidden, n_q_heads*head_dim]; w_gate, w_up
+ * [ffn, hidden]; w_down [hidden, ffn]. */
+typedef struct {
+  const void *attn_norm, *wq, *wk, *wv, *wo;
+  const void *ffn_norm, *w_gate, *w_up, *w_down;
+} thinfer_layer_weights;
+
+typedef struct {
+  const thinfer_layer_weights* layers; /* host array [n_layers] (copied by thinfer_create) */
+  const void *embed;                   /* device FP16 [vocab, hidden]; NULL when vocab == 0 */
+  const void *final_norm;              /* device FP16 [hidden];        NULL when vocab == 0 */
+  const void *lm_head;                 /* device FP16 [vocab, hidden]; NULL when vocab == 0 */
+} thinfer_weights;
+
+/* Sizes of the two caller-allocated device regions.
+ * kv_bytes: buf_slots x n_layers x {K,V} x [max_batch][n_kv_heads][max_seq][head_dim] FP16
+ * (K is stored after RoPE, Algorithm 1).  scratch_bytes: activations, RoPE
+ * table, split-KV partials, staging for the *_host calls.  Host pointers out. */
+int thinfer_workspace_bytes(const thinfer_config* cfg, size_t* kv_bytes, size_t* scratch_bytes);
+
+/* Builds a context.  cfg, weights: host.  kv_workspace, scratch: device, at
+ * least the sizes above (else THINFER_ECAPACITY); the context uses them until
+ * thinfer_destroy.  Synchronises the device once (table set-up).  *out is set
+ * only on success. */
+int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights,
+                   void* kv_workspace, size_t kv_bytes, void* scratch, size_t scratch_bytes,
+                   thinfer_ctx** out);
+
+/* Prefill (Section 3.4.2: the Prefill pool produces the first token and the
+ * initial KV cache).  Processes `batch` prompts of uniform length `seq_len`
+ * (Section 4.1: prompts padded to one length; every position is a real token,
+ * position = index in the sequence) and fills KV slot `slot` for positions
+ * 0..seq_len-1.
+ *   vocab == 0: input  device FP16 [batch, seq_len, hidden];
+ *               out_primary device FP16 [batch, seq_len, hidden] (layer-stack output); out_logits must be NULL.
+ *   vocab  > 0: input  device int32 [batch, seq_len] token ids in [0, vocab);
+ *               out_primary device int32 [batch] greedy next ids of the last position (may be NULL);
+ *               out_logits  device FP32 [batch, vocab] logits of the last position (may be NULL).
+ * Errors: THINFER_EBUSY if the slot holds an unreleased sequence;
+ * THINFER_ECAPACITY if batch > max_batch or seq_len > max_seq. */
+int thinfer_prefill(thinfer_ctx* ctx, int32_t slot, const void* input, int32_t batch, int32_t seq_len,
+                    void* out_primary, void* out_logits, void* cuda_stream);
+
+/* One decode step for every request of `slot` (Section 3.4.1, selective
+ * batching: projections batched over requests, attention per request).  The
+ * new token sits at position cur_len (the number of positions the slot holds);
+ * its key and value are appended and cur_len grows by one.
+ *   vocab == 0: input device FP16 [batch, hidden]; out_primary device FP16 [batch, hidden].
+ *   vocab  > 0: input device int32 [batch];        out_primary int32 [batch] / out_logits FP32 [batch, vocab].
+ * Errors: THINFER_EINVAL if the slot is empty; THINFER_ECAPACITY if cur_len == max_seq. */
+int thinfer_decode_step(thinfer_ctx* ctx, int32_t slot, const void* input,
+                        void* out_primary, void* out_logits, void* cuda_stream);
+
+/* The same two calls with HOST buffers: the input is copied to a staging area
+ * in `scratch`, the step runs, and out_primary (and out_logits if not NULL) is
+ * copied back, all enqueued on cuda_stream; the host buffers may be read once
+ * the stream has been synchronised.  Pinned host memory makes the copies
+ * asynchronous. */
+int thinfer_prefill_host(thinfer_ctx* ctx, int32_t slot, const void* host_input, int32_t batch, int32_t seq_len,
+                         void* host_out_primary, void* host_out_logits, void* cuda_stream);
+int thinfer_decode_step_host(thinfer_ctx* ctx, int32_t slot, const void* host_input,
+                             void* host_out_primary, void* host_out_logits, void* cuda_stream);
+
+/* Bounded buffer of Section 3.4.2: marks `slot` free so that a later prefill
+ * may reuse it.  Host state only; work already enqueued on the slot's KV is
+ * ordered by the caller's stream. */
+int thinfer_release_slot(thinfer_ctx* ctx, int32_t slot, void* cuda_stream);
+
+/* Host queries (no device work).  *batch / *cur_len: what the slot holds (0, 0 when free). */
+int thinfer_slot_state(const thinfer_ctx* ctx, int32_t slot, int32_t* batch, int32_t* cur_len);
+
+/* Device address of K (which = 0) or V (which = 1) of `layer` in `slot`:
+ * FP16 [max_batch][n_kv_heads][max_seq][head_dim].  For inspection by tests. */
+int thinfer_kv_pointer(const thinfer_ctx* ctx, int32_t slot, int32_t layer, int32_t which, void** device_ptr);
+
+/* Reads the device status word (0, or a thinfer_err a kernel wrote) without
+ * synchronising; meaningful after the caller synchronised the stream. */
+int thinfer_status(thinfer_ctx* ctx, int32_t* device_status);
+
+/* Unified launch (Section 3.3.3: one submission for the whole operator graph
+ * instead of one per operator).  mode 0: plain launches; 1: launches chained
+ * with programmatic dependent launch; 2: each decode step is replayed from a
+ * CUDA graph captured on first use per (slot, batch) and updated in place. */
+int thinfer_set_launch_mode(thinfer_ctx* ctx, int32_t mode);
+
+/* Per-kernel timing for roofline reports.  When `kernel_id` >= 0 every launch
+ * of that kernel (thinfer_kernel_id) is bracketed by CUDA events on its own
+ * stream; thinfer_profile_read synchronises those events and returns the count
+ * and the summed duration since the last read.  -1 switches it off. */
+typedef enum {
+  THINFER_K_RMSNORM = 0, THINFER_K_QKV = 1, THINFER_K_ATTN = 2, THINFER_K_ATTN_COMBINE = 3,
+  THINFER_K_OPROJ = 4, THINFER_K_GATEUP = 5, THINFER_K_DOWN = 6, THINFER_K_HEAD = 7,
+  THINFER_K_EMBED = 8, THINFER_K_ARGMAX = 9, THINFER_K_COUNT = 10
+} thinfer_kernel_id;
+int thinfer_profile_select(thinfer_ctx* ctx, int32_t kernel_id);
+int thinfer_profile_read(thinfer_ctx* ctx, int32_t* launches, float* total_ms);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t thinfer_launch_count(const thinfer_ctx* ctx);
+
+const char* thinfer_last_error(const thinfer_ctx* ctx);
+void thinfer_destroy(thinfer_ctx* ctx);
+
+/* ------------------------------------------------------------------------ *
+ * Single operators (the paper's operator layer, Section 3.2), exposed for
+ * parity tests and micro-benchmarks at the shapes of Tables 8 and 9.  All
+ * pointers are device pointers; work is enqueued on cuda_stream.
+ * ------------------------------------------------------------------------ */
+
+/* y[rows, n_out] = x[rows, k] * w[n_out, k]^T  (Section 3.2.1).  FP16 in,
+ * FP16 out (out_fp32 == 0) or FP32 out.  path 0: tcgen05 tensor-core tiles
+ * (any rows); path 1: the weight-streaming GEMV (rows <= 16).  k % 8 == 0. */
+int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k,
+                      int32_t out_fp32, int32_t path, void* cuda_stream);
+
+/* Causal attention of Eq. 6 for a batch: q FP16 [batch, n_q_heads, seq, head_dim],
+ * k, v FP16 [batch, n_kv_heads, kv_stride, head_dim] (first seq positions used),
+ * out FP16 [batch, seq, n_q_heads*head_dim]. */
+int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, void* out,
+                                 int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t seq,
+                                 int32_t kv_stride, int32_t head_dim, void* cuda_stream);
+
+/* y = x * gain / sqrt(mean(x^2) + eps), rows of length n (Section 3.2.4). */
+int thinfer_op_rmsnorm(const void* x, const void* gain, void* y, int32_t rows, int32_t n, float eps,
+                       void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* THINFER_H */

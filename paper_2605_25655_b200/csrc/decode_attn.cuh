@@ -1,0 +1,194 @@
+// Decode attention over the FP16 KV cache: Eq. 6 for one query row per
+// (request, head), the M = 1 case of the staged attention of Section 3.3.2.
+// Per request (selective batching, Section 3.4.1) and bandwidth-bound: K and V
+// rows are streamed once with 128-bit loads; the query heads that share a KV
+// head are processed in the same pass.  The KV range is split across CTAs
+// (split-KV); every lane group keeps a running (max, sum, output) triple that
+// is merged by the online-softmax rule first inside the warp, then across the
+// CTA's warps, then across splits by a small combine kernel.
+#pragma once
+#include "common.cuh"
+
+namespace thinfer {
+
+constexpr int kAttnDecWarps = 4;
+constexpr int kAttnDecUnroll = 4;
+
+struct AttnDecArgs {
+  const __half* q;        // [batch][n_q_heads][D], already rotated
+  const __half* k_cache;  // [max_batch][n_kv_heads][t_max][D]
+  const __half* v_cache;
+  __half* out;            // [batch][n_q_heads * D]
+  float* part_o;          // [batch][n_q_heads][splits][D]   un-normalised partial outputs
+  float* part_ml;         // [batch][n_q_heads][splits][2]   (max in log2 units, sum)
+  int n_q_heads, n_kv_heads;
+  int t_len;              // keys to attend: positions 0 .. t_len-1
+  int t_max;
+  int splits, chunk;      // chunk = keys per split
+  float scale_log2;       // log2(e) / sqrt(D)
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const AttnDecArgs a) {
+  constexpr int LPK = D / 8;     // lanes that cover one key row
+  constexpr int KPL = 32 / LPK;  // keys per warp-wide load
+  constexpr int UN = kAttnDecUnroll;
+  __shared__ float sm_m[kAttnDecWarps][G], sm_l[kAttnDecWarps][G];
+  __shared__ float sm_o[kAttnDecWarps][G][D];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPK, dl = lane % LPK;
+  const int split = blockIdx.x, b = blockIdx.z;
+  const int h0 = blockIdx.y * G;                                   // first query head of this CTA
+  const int hk = h0 / (a.n_q_heads / a.n_kv_heads);
+  const int t0 = split * a.chunk;
+  const int t1 = min(a.t_len, t0 + a.chunk);
+
+  float q[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    unpack8(ldg_cached(a.q + (static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + dl * 8), q[g]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[g][i] *= a.scale_log2;
+  }
+  const __half* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+  const __half* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+
+  float m[G], l[G], o[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    m[g] = -INFINITY;
+    l[g] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
+  }
+
+  for (int tb = t0 + warp * (UN * KPL); tb < t1; tb += kAttnDecWarps * UN * KPL) {
+    uint4 kv[UN], vv[UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      const int t = tb + u * KPL + sub;
+      if (t < t1) {
+        kv[u] = ldg_stream(kb + static_cast<size_t>(t) * D);
+        vv[u] = ldg_stream(vb + static_cast<size_t>(t) * D);
+      } else {
+        kv[u] = make_uint4(0, 0, 0, 0);
+        vv[u] = make_uint4(0, 0, 0, 0);
+      }
+    }
+    float s[G][UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      float fk[8];
+      unpack8(kv[u], fk);
+      const bool valid = (tb + u * KPL + sub) < t1;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) d = fmaf(q[g][i], fk[i], d);
+#pragma unroll
+        for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        s[g][u] = valid ? d : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float mx = m[g];
+#pragma unroll
+      for (int u = 0; u < UN; ++u) mx = fmaxf(mx, s[g][u]);
+      const float ms = (mx == -INFINITY) ? 0.f : mx;
+      const float alpha = exp2f(m[g] - ms);  // m = -inf -> 0
+      m[g] = mx;
+      l[g] *= alpha;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[g][i] *= alpha;
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const float p = exp2f(s[g][u] - ms);
+        l[g] += p;
+        float fv[8];
+        unpack8(vv[u], fv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[g][i] = fmaf(p, fv[i], o[g][i]);
+      }
+    }
+  }
+
+  // merge the KPL lane groups of the warp
+#pragma unroll
+  for (int off = LPK; off < 32; off <<= 1) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m[g], off);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l[g], off);
+      const float mx = fmaxf(m[g], m2);
+      const float ms = (mx == -INFINITY) ? 0.f : mx;
+      const float a1 = exp2f(m[g] - ms), a2 = exp2f(m2 - ms);
+      l[g] = l[g] * a1 + l2 * a2;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float o2 = __shfl_xor_sync(0xffffffffu, o[g][i], off);
+        o[g][i] = o[g][i] * a1 + o2 * a2;
+      }
+      m[g] = mx;
+    }
+  }
+  if (sub == 0) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      if (dl == 0) {
+        sm_m[warp][g] = m[g];
+        sm_l[warp][g] = l[g];
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sm_o[warp][g][dl * 8 + i] = o[g][i];
+    }
+  }
+  __syncthreads();
+
+  for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
+    const int g = idx / D, i = idx - g * D;
+    float mx = sm_m[0][g];
+#pragma unroll
+    for (int w = 1; w < kAttnDecWarps; ++w) mx = fmaxf(mx, sm_m[w][g]);
+    const float ms = (mx == -INFINITY) ? 0.f : mx;
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnDecWarps; ++w) {
+      const float al = exp2f(sm_m[w][g] - ms);
+      L += sm_l[w][g] * al;
+      O += sm_o[w][g][i] * al;
+    }
+    const int h = h0 + g;
+    if (a.splits == 1) {
+      a.out[(static_cast<size_t>(b) * a.n_q_heads + h) * D + i] = __float2half_rn(O / L);
+    } else {
+      const size_t p = (static_cast<size_t>(b) * a.n_q_heads + h) * a.splits + split;
+      a.part_o[p * D + i] = O;
+      if (i == 0) {
+        a.part_ml[p * 2] = mx;
+        a.part_ml[p * 2 + 1] = L;
+      }
+    }
+  }
+}
+
+// Merges the split-KV partials: out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
+template <int D>
+__global__ void __launch_bounds__(D) attn_decode_combine_kernel(const AttnDecArgs a) {
+  const size_t bh = blockIdx.x;  // (request, query head)
+  const int i = threadIdx.x;
+  float mx = -INFINITY;
+  for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, a.part_ml[(bh * a.splits + s) * 2]);
+  float L = 0.f, O = 0.f;
+  for (int s = 0; s < a.splits; ++s) {
+    const size_t p = bh * a.splits + s;
+    const float al = exp2f(a.part_ml[p * 2] - mx);
+    L += a.part_ml[p * 2 + 1] * al;
+    O += a.part_o[p * D + i] * al;
+  }
+  a.out[bh * D + i] = __float2half_rn(O / L);
+}
+
+}  // namespace thinfer

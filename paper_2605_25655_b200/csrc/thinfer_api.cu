@@ -1,0 +1,965 @@
+// C ABI of the library (include/thinfer.h): context, argument validation, the
+// per-layer launch sequences of prefill and decode, the bounded KV slot ring of
+// the Prefill-Buffer-Decode pipeline (Section 3.4.2), and the single-operator
+// entry points.  Host code only launches kernels; every step of the path runs
+// in the kernels of this directory.
+#include "../../include/thinfer.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "decode_attn.cuh"
+#include "decode_gemv.cuh"
+#include "misc_kernels.cuh"
+#include "prefill_attn.cuh"
+#include "tc_gemm.cuh"
+
+using namespace thinfer;
+
+namespace {
+
+// ----------------------------------------------------------------------------
+// driver entry point for tensor-map encoding (no link-time dependency on libcuda)
+// ----------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// FP16 tensor [d2][d1][d0] (d0 contiguous), box [1][box1][64], 128-byte swizzle, zero fill outside.
+// stride1 / stride2 in elements.
+bool make_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1,
+              uint64_t stride2, uint32_t box1, int rank) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1 * 2, stride2 * 2};
+  cuuint32_t box[3] = {64, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base), dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+bool make_map_2d(CUtensorMap* m, const void* base, uint64_t k, uint64_t rows, uint32_t box_rows) {
+  return make_map(m, base, k, rows, 1, k, 0, box_rows, 2);
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct LayerMaps {
+  CUtensorMap wq, wk, wv, wo, wg, wu, wd;
+};
+
+struct Slot {
+  int batch = 0, cur_len = 0;
+  bool busy = false;
+};
+
+struct ProfEvent {
+  cudaEvent_t beg, end;
+};
+
+}  // namespace
+
+struct thinfer_ctx {
+  thinfer_config cfg{};
+  std::vector<thinfer_layer_weights> layers;
+  const __half *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+  std::vector<LayerMaps> maps;
+  CUtensorMap map_head{};
+  uint8_t* kv = nullptr;
+  size_t kv_layer_bytes = 0;  // one of K or V for one layer of one slot
+  std::vector<Slot> slots;
+  // scratch carve-up
+  float *rope_cos = nullptr, *rope_sin = nullptr;
+  __half *h = nullptr, *qbuf = nullptr, *attn = nullptr, *x1 = nullptr, *act = nullptr, *xa = nullptr, *xb = nullptr;
+  __half* last = nullptr;
+  float* logits = nullptr;
+  int32_t* ids_out = nullptr;
+  float *part_o = nullptr, *part_ml = nullptr;
+  uint8_t *stage_in = nullptr, *stage_out = nullptr;
+  int max_splits = 1;
+  // status word (pinned, mapped)
+  int* status_host = nullptr;
+  int* status_dev = nullptr;
+  int launch_mode = 0;
+  int64_t launches = 0;
+  int prof_kernel = -1;
+  std::vector<ProfEvent> prof_events;
+  size_t prof_used = 0;
+  std::string err;
+  int sm_count = 148;
+};
+
+namespace {
+
+int fail(thinfer_ctx* c, int code, const char* fmt, ...) {
+  if (c != nullptr) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    c->err = buf;
+  }
+  return code;
+}
+
+thread_local std::string g_global_err;
+
+int validate_config(const thinfer_config* c, std::string* why) {
+  auto bad = [&](int code, const char* s) {
+    if (why) *why = s;
+    return code;
+  };
+  if (c == nullptr) return bad(THINFER_EINVAL, "config is NULL");
+  if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 || c->ffn <= 0 ||
+      c->n_layers <= 0 || c->vocab < 0 || c->max_batch <= 0 || c->max_seq <= 0 || c->buf_slots <= 0)
+    return bad(THINFER_EINVAL, "config has a non-positive size");
+  if (!(c->rms_eps >= 0.f) || !(c->rope_base > 0.f)) return bad(THINFER_EINVAL, "rms_eps or rope_base out of range");
+  if (c->head_dim != 64 && c->head_dim != 128) return bad(THINFER_EUNSUPPORTED, "head_dim must be 64 or 128");
+  if (c->n_q_heads % c->n_kv_heads != 0) return bad(THINFER_EUNSUPPORTED, "n_q_heads must be a multiple of n_kv_heads");
+  if (c->hidden % 8 != 0 || c->ffn % 8 != 0) return bad(THINFER_EUNSUPPORTED, "hidden and ffn must be multiples of 8");
+  if (c->max_batch > 64) return bad(THINFER_EUNSUPPORTED, "max_batch must be <= 64");
+  if (c->vocab % 2 != 0) return bad(THINFER_EUNSUPPORTED, "vocab must be even");
+  return THINFER_OK;
+}
+
+struct ScratchPlan {
+  size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, stage_in, stage_out,
+      total;
+  int max_splits;
+};
+
+ScratchPlan plan_scratch(const thinfer_config& c) {
+  ScratchPlan p{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 1024);
+    return o;
+  };
+  const size_t M = static_cast<size_t>(c.max_batch) * c.max_seq;
+  const size_t qd = static_cast<size_t>(c.n_q_heads) * c.head_dim;
+  p.max_splits = 32;
+  p.rope_cos = take(static_cast<size_t>(c.max_seq) * (c.head_dim / 2) * 4);
+  p.rope_sin = take(static_cast<size_t>(c.max_seq) * (c.head_dim / 2) * 4);
+  p.h = take(M * c.hidden * 2);
+  p.qbuf = take(M * qd * 2);
+  p.attn = take(M * qd * 2);
+  p.x1 = take(M * c.hidden * 2);
+  p.act = take(M * c.ffn * 2);
+  p.xa = take(M * c.hidden * 2);
+  p.xb = take(M * c.hidden * 2);
+  p.last = take(static_cast<size_t>(c.max_batch) * c.hidden * 2);
+  p.logits = take(static_cast<size_t>(c.max_batch) * (c.vocab > 0 ? c.vocab : 1) * 4);
+  p.ids_out = take(static_cast<size_t>(c.max_batch) * 4);
+  p.part_o = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * p.max_splits * c.head_dim * 4);
+  p.part_ml = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * p.max_splits * 2 * 4);
+  const size_t in_bytes = c.vocab > 0 ? M * 4 : M * c.hidden * 2;
+  const size_t out_bytes = c.vocab > 0 ? static_cast<size_t>(c.max_batch) * (4 + static_cast<size_t>(c.vocab) * 4)
+                                       : M * c.hidden * 2;
+  p.stage_in = take(in_bytes);
+  p.stage_out = take(out_bytes);
+  p.total = off;
+  return p;
+}
+
+size_t kv_layer_bytes_of(const thinfer_config& c) {
+  return align_up(static_cast<size_t>(c.max_batch) * c.n_kv_heads * c.max_seq * c.head_dim * 2, 1024);
+}
+
+// ----------------------------------------------------------------------------
+// launch helper: counts, optional event bracketing, error check
+// ----------------------------------------------------------------------------
+struct Launcher {
+  thinfer_ctx* c;
+  cudaStream_t st;
+  int rc = THINFER_OK;
+
+  template <typename... KArgs, typename... Args>
+  void go(int kid, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+    if (rc != THINFER_OK) return;
+    const bool prof = c != nullptr && c->prof_kernel == kid;
+    ProfEvent ev{};
+    if (prof) {
+      if (c->prof_used == c->prof_events.size()) {
+        ProfEvent n{};
+        if (cudaEventCreate(&n.beg) != cudaSuccess || cudaEventCreate(&n.end) != cudaSuccess) {
+          rc = fail(c, THINFER_ECUDA, "cudaEventCreate failed");
+          return;
+        }
+        c->prof_events.push_back(n);
+      }
+      ev = c->prof_events[c->prof_used++];
+      cudaEventRecord(ev.beg, st);
+    }
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    lc.attrs = attr;
+    lc.numAttrs = 0;
+    cudaError_t e = cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+    if (prof) cudaEventRecord(ev.end, st);
+    if (e != cudaSuccess) {
+      rc = fail(c, THINFER_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+      if (c == nullptr) g_global_err = cudaGetErrorString(e);
+      return;
+    }
+    if (c != nullptr) ++c->launches;
+  }
+};
+
+template <typename K>
+bool opt_in_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// ----------------------------------------------------------------------------
+// tcgen05 GEMM dispatch
+// ----------------------------------------------------------------------------
+template <int BN, int EPI>
+void launch_tc(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
+               const CUtensorMap& x, const TcGemmArgs& a) {
+  static bool ready = false;  // per instantiation; contexts are created from one thread at a time
+  constexpr int smem = tc_smem_bytes(BN, EPI);
+  if (!ready) {
+    if (!opt_in_smem(tc_gemm_kernel<BN, EPI>, smem)) {
+      L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+      return;
+    }
+    ready = true;
+  }
+  const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
+  const int n_tt = (a.rows + BN - 1) / BN;
+  L.go(kid, tc_gemm_kernel<BN, EPI>, dim3(n_ft * n_tt), dim3(kTcThreads), smem, w0, w1, w2, x, a);
+}
+
+int pick_bn(int rows) {
+  if (rows <= 16) return 16;
+  if (rows <= 32) return 32;
+  if (rows <= 64) return 64;
+  if (rows <= 128) return 128;
+  return 256;
+}
+
+template <int EPI>
+void launch_tc_bn(Launcher& L, int kid, int bn, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
+                  const CUtensorMap& x, const TcGemmArgs& a) {
+  switch (bn) {
+    case 16: launch_tc<16, EPI>(L, kid, w0, w1, w2, x, a); break;
+    case 32: launch_tc<32, EPI>(L, kid, w0, w1, w2, x, a); break;
+    case 64: launch_tc<64, EPI>(L, kid, w0, w1, w2, x, a); break;
+    case 128: launch_tc<128, EPI>(L, kid, w0, w1, w2, x, a); break;
+    default: launch_tc<256, EPI>(L, kid, w0, w1, w2, x, a); break;
+  }
+}
+
+// x: activations [rows][k]; the token-side tensor map is encoded per call (host only, no device work)
+template <int EPI>
+void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
+               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e) {
+  if (L.rc != THINFER_OK) return;
+  const int bn = pick_bn(rows);
+  CUtensorMap mx;
+  if (!make_map_2d(&mx, x, k, rows, bn)) {
+    L.rc = fail(L.c, THINFER_ECUDA, "cuTensorMapEncodeTiled failed for an activation operand");
+    return;
+  }
+  TcGemmArgs a{};
+  for (int i = 0; i < 3; ++i) {
+    a.n_feat[i] = n_feat[i];
+    a.tiles[i] = (n_feat[i] + kTcBM - 1) / kTcBM;
+  }
+  if (EPI == EPI_SWIGLU) a.tiles[1] = 0;  // gate and up tiles are processed together
+  a.rows = rows;
+  a.k = k;
+  a.status = L.c ? L.c->status_dev : nullptr;
+  a.e = e;
+  launch_tc_bn<EPI>(L, kid, bn, w0, w1, w2, mx, a);
+}
+
+// ----------------------------------------------------------------------------
+// streaming GEMV dispatch (decode)
+// ----------------------------------------------------------------------------
+int pick_kslices(int n_pairs, int k, int sm_count) {
+  // enough independent warps to cover the machine several times; never slice below 512 elements
+  int ks = 1;
+  while (ks < 8 && static_cast<long long>(n_pairs) * ks < 32LL * sm_count && k / (ks * 2) >= 512) ks *= 2;
+  return ks;
+}
+
+template <int EPI, bool NORM>
+void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
+          const __half* x, int ldx, int rows, const __half* gamma, float eps, const EpiArgs& e) {
+  if (L.rc != THINFER_OK) return;
+  GemvArgs a{};
+  a.w[0] = w0;
+  a.w[1] = w1;
+  a.w[2] = w2;
+  for (int i = 0; i < 3; ++i) a.n[i] = n[i];
+  a.k = k;
+  a.rows = rows;
+  a.x = x;
+  a.ldx = ldx;
+  a.gamma = gamma;
+  a.eps = eps;
+  a.e = e;
+  const int n_pairs = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
+  a.kslices = pick_kslices(n_pairs, k, L.c ? L.c->sm_count : 148);
+  const int pairs_per_cta = kGemvWarps / a.kslices;
+  const int gx = (n_pairs + pairs_per_cta - 1) / pairs_per_cta;
+  const dim3 block(kGemvWarps * 32);
+  if (rows == 1) {
+    L.go(kid, gemv_stream_kernel<1, EPI, NORM>, dim3(gx, 1), block, 0, a);
+  } else if (rows == 2) {
+    L.go(kid, gemv_stream_kernel<2, EPI, NORM>, dim3(gx, 1), block, 0, a);
+  } else {
+    L.go(kid, gemv_stream_kernel<4, EPI, NORM>, dim3(gx, (rows + 3) / 4), block, 0, a);
+  }
+}
+
+// ----------------------------------------------------------------------------
+// attention dispatch
+// ----------------------------------------------------------------------------
+template <int D>
+void attn_decode_d(Launcher& L, const AttnDecArgs& a, int batch, int ratio) {
+  int g = 1;
+  if (ratio % 8 == 0) g = 8;
+  else if (ratio % 4 == 0) g = 4;
+  else if (ratio % 2 == 0) g = 2;
+  const dim3 grid(a.splits, a.n_q_heads / g, batch), block(kAttnDecWarps * 32);
+  switch (g) {
+    case 8: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 8>, grid, block, 0, a); break;
+    case 4: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 4>, grid, block, 0, a); break;
+    case 2: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 2>, grid, block, 0, a); break;
+    default: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 1>, grid, block, 0, a); break;
+  }
+  if (a.splits > 1)
+    L.go(THINFER_K_ATTN_COMBINE, attn_decode_combine_kernel<D>, dim3(batch * a.n_q_heads), dim3(D), 0, a);
+}
+
+void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc, const __half* vc, __half* out,
+                 int batch, int t_len) {
+  const thinfer_config& cf = c->cfg;
+  AttnDecArgs a{};
+  a.q = q;
+  a.k_cache = kc;
+  a.v_cache = vc;
+  a.out = out;
+  a.part_o = c->part_o;
+  a.part_ml = c->part_ml;
+  a.n_q_heads = cf.n_q_heads;
+  a.n_kv_heads = cf.n_kv_heads;
+  a.t_len = t_len;
+  a.t_max = cf.max_seq;
+  const int ratio = cf.n_q_heads / cf.n_kv_heads;
+  int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
+  const int ctas = batch * (cf.n_q_heads / g);
+  int splits = (2 * c->sm_count + ctas - 1) / ctas;
+  const int by_len = (t_len + 127) / 128;  // at least 128 keys per split
+  if (splits > by_len) splits = by_len;
+  if (splits > c->max_splits) splits = c->max_splits;
+  if (splits < 1) splits = 1;
+  a.chunk = (t_len + splits - 1) / splits;
+  a.splits = (t_len + a.chunk - 1) / a.chunk;
+  a.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(cf.head_dim));
+  if (cf.head_dim == 128) attn_decode_d<128>(L, a, batch, ratio);
+  else attn_decode_d<64>(L, a, batch, ratio);
+}
+
+template <int D>
+void attn_prefill_d(Launcher& L, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                    const AttnPreArgs& a, int batch) {
+  static bool ready = false;
+  constexpr int smem = attn_pre_smem_bytes(D);
+  if (!ready) {
+    if (!opt_in_smem(attn_prefill_kernel<D>, smem)) {
+      L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+      return;
+    }
+    ready = true;
+  }
+  const int n_qt = (a.seq_len + kAttnBQ - 1) / kAttnBQ;
+  L.go(THINFER_K_ATTN, attn_prefill_kernel<D>, dim3(n_qt, a.n_q_heads, batch), dim3(kAttnThreads), smem, mq, mk, mv, a);
+}
+
+void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v, __half* out, int batch, int n_q_heads,
+                  int n_kv_heads, int seq, int kv_stride, int head_dim, int* status) {
+  if (L.rc != THINFER_OK) return;
+  CUtensorMap mq, mk, mv;
+  const uint64_t d = head_dim;
+  bool ok = make_map(&mq, q, d, seq, static_cast<uint64_t>(batch) * n_q_heads, d, static_cast<uint64_t>(seq) * d, 128, 3);
+  ok = ok && make_map(&mk, k, d, seq, static_cast<uint64_t>(batch) * n_kv_heads, d, static_cast<uint64_t>(kv_stride) * d,
+                      128, 3);
+  ok = ok && make_map(&mv, v, d, seq, static_cast<uint64_t>(batch) * n_kv_heads, d, static_cast<uint64_t>(kv_stride) * d,
+                      128, 3);
+  if (!ok) {
+    L.rc = fail(L.c, THINFER_ECUDA, "cuTensorMapEncodeTiled failed for an attention operand");
+    return;
+  }
+  AttnPreArgs a{};
+  a.out = out;
+  a.n_q_heads = n_q_heads;
+  a.n_kv_heads = n_kv_heads;
+  a.seq_len = seq;
+  a.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(head_dim));
+  a.status = status;
+  if (head_dim == 128) attn_prefill_d<128>(L, mq, mk, mv, a, batch);
+  else attn_prefill_d<64>(L, mq, mk, mv, a, batch);
+}
+
+void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int rows, int n, float eps) {
+  L.go(THINFER_K_RMSNORM, rmsnorm_rows_kernel, dim3((rows + 7) / 8), dim3(256), 0, x, g, y, rows, n, eps);
+}
+
+// ----------------------------------------------------------------------------
+// the layer sequences
+// ----------------------------------------------------------------------------
+EpiArgs qkv_epi(thinfer_ctx* c, __half* kc, __half* vc, int seq_len, int pos0) {
+  const thinfer_config& cf = c->cfg;
+  EpiArgs e{};
+  e.q_out = c->qbuf;
+  e.k_cache = kc;
+  e.v_cache = vc;
+  e.rope_cos = c->rope_cos;
+  e.rope_sin = c->rope_sin;
+  e.n_q = cf.n_q_heads * cf.head_dim;
+  e.n_kv = cf.n_kv_heads * cf.head_dim;
+  e.head_dim = cf.head_dim;
+  e.n_q_heads = cf.n_q_heads;
+  e.n_kv_heads = cf.n_kv_heads;
+  e.seq_len = seq_len;
+  e.pos0 = pos0;
+  e.t_max = cf.max_seq;
+  return e;
+}
+
+__half* kv_ptr(thinfer_ctx* c, int slot, int layer, int which) {
+  const size_t idx = (static_cast<size_t>(slot) * c->cfg.n_layers + layer) * 2 + which;
+  return reinterpret_cast<__half*>(c->kv + idx * c->kv_layer_bytes);
+}
+
+void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half* x_in, __half* x_out, int batch,
+                   int seq) {
+  const thinfer_config& cf = c->cfg;
+  const thinfer_layer_weights& w = c->layers[layer];
+  const LayerMaps& m = c->maps[layer];
+  const int rows = batch * seq;
+  const int qd = cf.n_q_heads * cf.head_dim, kvd = cf.n_kv_heads * cf.head_dim;
+  __half* kc = kv_ptr(c, slot, layer, 0);
+  __half* vc = kv_ptr(c, slot, layer, 1);
+
+  rmsnorm_rows(L, x_in, static_cast<const __half*>(w.attn_norm), c->h, rows, cf.hidden, cf.rms_eps);
+  {
+    const int nf[3] = {qd, kvd, kvd};
+    tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, rows, cf.hidden, nf, qkv_epi(c, kc, vc, seq, 0));
+  }
+  attn_prefill(L, c->qbuf, kc, vc, c->attn, batch, cf.n_q_heads, cf.n_kv_heads, seq, cf.max_seq, cf.head_dim,
+               c->status_dev);
+  {
+    EpiArgs e{};
+    e.out = c->x1;
+    e.resid = x_in;
+    e.ld_out = cf.hidden;
+    const int nf[3] = {cf.hidden, 0, 0};
+    tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->attn, rows, qd, nf, e);
+  }
+  rmsnorm_rows(L, c->x1, static_cast<const __half*>(w.ffn_norm), c->h, rows, cf.hidden, cf.rms_eps);
+  {
+    EpiArgs e{};
+    e.out = c->act;
+    e.ld_out = cf.ffn;
+    const int nf[3] = {cf.ffn, cf.ffn, 0};
+    tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->h, rows, cf.hidden, nf, e);
+  }
+  {
+    EpiArgs e{};
+    e.out = x_out;
+    e.resid = c->x1;
+    e.ld_out = cf.hidden;
+    const int nf[3] = {cf.hidden, 0, 0};
+    tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->act, rows, cf.ffn, nf, e);
+  }
+}
+
+void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half* x_in, __half* x_out, int batch,
+                  int pos) {
+  const thinfer_config& cf = c->cfg;
+  const thinfer_layer_weights& w = c->layers[layer];
+  const int qd = cf.n_q_heads * cf.head_dim, kvd = cf.n_kv_heads * cf.head_dim;
+  __half* kc = kv_ptr(c, slot, layer, 0);
+  __half* vc = kv_ptr(c, slot, layer, 1);
+  auto H = [](const void* p) { return static_cast<const __half*>(p); };
+  {
+    const int n[3] = {qd, kvd, kvd};
+    gemv<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch,
+                             H(w.attn_norm), cf.rms_eps, qkv_epi(c, kc, vc, 1, pos));
+  }
+  attn_decode(L, c, c->qbuf, kc, vc, c->attn, batch, pos + 1);
+  {
+    EpiArgs e{};
+    e.out = c->x1;
+    e.resid = x_in;
+    e.ld_out = cf.hidden;
+    const int n[3] = {cf.hidden, 0, 0};
+    gemv<EPI_RESID, false>(L, THINFER_K_OPROJ, H(w.wo), nullptr, nullptr, n, qd, c->attn, qd, batch, nullptr, 0.f, e);
+  }
+  {
+    EpiArgs e{};
+    e.out = c->act;
+    e.ld_out = cf.ffn;
+    const int n[3] = {cf.ffn, cf.ffn, 0};
+    gemv<EPI_SWIGLU, true>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->x1, cf.hidden, batch,
+                           H(w.ffn_norm), cf.rms_eps, e);
+  }
+  {
+    EpiArgs e{};
+    e.out = x_out;
+    e.resid = c->x1;
+    e.ld_out = cf.hidden;
+    const int n[3] = {cf.hidden, 0, 0};
+    gemv<EPI_RESID, false>(L, THINFER_K_DOWN, H(w.w_down), nullptr, nullptr, n, cf.ffn, c->act, cf.ffn, batch, nullptr,
+                           0.f, e);
+  }
+}
+
+// final RMSNorm + LM head + greedy argmax on `batch` rows of x [batch][hidden]
+void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, int32_t* ids_out, float* logits_out) {
+  const thinfer_config& cf = c->cfg;
+  float* lg = logits_out != nullptr ? logits_out : c->logits;
+  EpiArgs e{};
+  e.out = lg;
+  e.ld_out = cf.vocab;
+  const int n[3] = {cf.vocab, 0, 0};
+  gemv<EPI_PLAIN_F32, true>(L, THINFER_K_HEAD, c->lm_head, nullptr, nullptr, n, cf.hidden, x, cf.hidden, batch,
+                            c->final_norm, cf.rms_eps, e);
+  if (ids_out != nullptr)
+    L.go(THINFER_K_ARGMAX, argmax_rows_kernel, dim3(batch), dim3(1024), 0, static_cast<const float*>(lg), ids_out,
+         cf.vocab);
+}
+
+int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq, void* out_primary, void* out_logits,
+                cudaStream_t st) {
+  const thinfer_config& cf = c->cfg;
+  Launcher L{c, st};
+  const int rows = batch * seq;
+  const __half* x = nullptr;
+  if (cf.vocab > 0) {
+    L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((rows + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
+         c->embed, c->xa, rows, cf.hidden, cf.vocab);
+    x = c->xa;
+  } else {
+    x = static_cast<const __half*>(input);
+  }
+  __half* pong[2] = {c->xb, c->xa};
+  for (int l = 0; l < cf.n_layers; ++l) {
+    __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
+    layer_prefill(L, c, slot, l, x, dst, batch, seq);
+    x = dst;
+  }
+  if (cf.vocab > 0) {
+    L.go(THINFER_K_EMBED, gather_last_rows_kernel, dim3((batch + 7) / 8), dim3(256), 0, x, c->last, batch, seq,
+         cf.hidden);
+    head_and_argmax(L, c, c->last, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits));
+  }
+  return L.rc;
+}
+
+int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, void* out_primary, void* out_logits,
+               cudaStream_t st) {
+  const thinfer_config& cf = c->cfg;
+  Launcher L{c, st};
+  const __half* x = nullptr;
+  if (cf.vocab > 0) {
+    L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((batch + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
+         c->embed, c->xa, batch, cf.hidden, cf.vocab);
+    x = c->xa;
+  } else {
+    x = static_cast<const __half*>(input);
+  }
+  __half* pong[2] = {c->xb, c->xa};
+  for (int l = 0; l < cf.n_layers; ++l) {
+    __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
+    layer_decode(L, c, slot, l, x, dst, batch, pos);
+    x = dst;
+  }
+  if (cf.vocab > 0) head_and_argmax(L, c, x, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits));
+  return L.rc;
+}
+
+int check_prefill_args(thinfer_ctx* c, int slot, const void* input, int batch, int seq, void* out_primary,
+                       void* out_logits) {
+  if (c == nullptr) return THINFER_EINVAL;
+  const thinfer_config& cf = c->cfg;
+  if (slot < 0 || slot >= cf.buf_slots) return fail(c, THINFER_EINVAL, "slot %d outside [0, %d)", slot, cf.buf_slots);
+  if (input == nullptr) return fail(c, THINFER_EINVAL, "input is NULL");
+  if (batch <= 0 || seq <= 0) return fail(c, THINFER_EINVAL, "batch and seq_len must be positive");
+  if (batch > cf.max_batch) return fail(c, THINFER_ECAPACITY, "batch %d > max_batch %d", batch, cf.max_batch);
+  if (seq > cf.max_seq) return fail(c, THINFER_ECAPACITY, "seq_len %d > max_seq %d", seq, cf.max_seq);
+  if (cf.vocab == 0) {
+    if (out_primary == nullptr) return fail(c, THINFER_EINVAL, "out_primary is NULL");
+    if (out_logits != nullptr) return fail(c, THINFER_EINVAL, "out_logits must be NULL in layer-only mode");
+  } else if (out_primary == nullptr && out_logits == nullptr) {
+    return fail(c, THINFER_EINVAL, "both outputs are NULL");
+  }
+  if (c->slots[slot].busy) return fail(c, THINFER_EBUSY, "slot %d holds an unreleased sequence", slot);
+  return THINFER_OK;
+}
+
+int check_decode_args(thinfer_ctx* c, int slot, const void* input, void* out_primary, void* out_logits) {
+  if (c == nullptr) return THINFER_EINVAL;
+  const thinfer_config& cf = c->cfg;
+  if (slot < 0 || slot >= cf.buf_slots) return fail(c, THINFER_EINVAL, "slot %d outside [0, %d)", slot, cf.buf_slots);
+  if (input == nullptr) return fail(c, THINFER_EINVAL, "input is NULL");
+  if (!c->slots[slot].busy) return fail(c, THINFER_EINVAL, "slot %d is empty: prefill first", slot);
+  if (c->slots[slot].cur_len >= cf.max_seq)
+    return fail(c, THINFER_ECAPACITY, "slot %d is full (%d positions)", slot, cf.max_seq);
+  if (cf.vocab == 0) {
+    if (out_primary == nullptr) return fail(c, THINFER_EINVAL, "out_primary is NULL");
+    if (out_logits != nullptr) return fail(c, THINFER_EINVAL, "out_logits must be NULL in layer-only mode");
+  } else if (out_primary == nullptr && out_logits == nullptr) {
+    return fail(c, THINFER_EINVAL, "both outputs are NULL");
+  }
+  return THINFER_OK;
+}
+
+}  // namespace
+
+// ============================================================================
+// exported functions
+// ============================================================================
+extern "C" {
+
+int thinfer_workspace_bytes(const thinfer_config* cfg, size_t* kv_bytes, size_t* scratch_bytes) {
+  int rc = validate_config(cfg, &g_global_err);
+  if (rc != THINFER_OK) return rc;
+  if (kv_bytes == nullptr || scratch_bytes == nullptr) return THINFER_EINVAL;
+  *kv_bytes = kv_layer_bytes_of(*cfg) * 2 * static_cast<size_t>(cfg->n_layers) * cfg->buf_slots;
+  *scratch_bytes = plan_scratch(*cfg).total;
+  return THINFER_OK;
+}
+
+int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, void* kv_workspace, size_t kv_bytes,
+                   void* scratch, size_t scratch_bytes, thinfer_ctx** out) {
+  int rc = validate_config(cfg, &g_global_err);
+  if (rc != THINFER_OK) return rc;
+  if (weights == nullptr || weights->layers == nullptr || kv_workspace == nullptr || scratch == nullptr ||
+      out == nullptr)
+    return THINFER_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(kv_workspace) & 255) != 0 || (reinterpret_cast<uintptr_t>(scratch) & 255) != 0)
+    return THINFER_EINVAL;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const thinfer_layer_weights& w = weights->layers[l];
+    const void* ps[9] = {w.attn_norm, w.wq, w.wk, w.wv, w.wo, w.ffn_norm, w.w_gate, w.w_up, w.w_down};
+    for (const void* p : ps)
+      if (p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15) != 0) return THINFER_EINVAL;
+  }
+  if (cfg->vocab > 0 && (weights->embed == nullptr || weights->final_norm == nullptr || weights->lm_head == nullptr))
+    return THINFER_EINVAL;
+  size_t need_kv = 0, need_scratch = 0;
+  thinfer_workspace_bytes(cfg, &need_kv, &need_scratch);
+  if (kv_bytes < need_kv || scratch_bytes < need_scratch) return THINFER_ECAPACITY;
+
+  int dev = 0;
+  cudaDeviceProp prop{};
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return THINFER_ECUDA;
+  if (prop.major != 10) {
+    g_global_err = "this library runs on sm_100 devices only";
+    return THINFER_EUNSUPPORTED;
+  }
+  if (encode_tiled_fn() == nullptr) return THINFER_ECUDA;
+
+  thinfer_ctx* c = new thinfer_ctx();
+  c->cfg = *cfg;
+  c->sm_count = prop.multiProcessorCount;
+  c->layers.assign(weights->layers, weights->layers + cfg->n_layers);
+  c->embed = static_cast<const __half*>(weights->embed);
+  c->final_norm = static_cast<const __half*>(weights->final_norm);
+  c->lm_head = static_cast<const __half*>(weights->lm_head);
+  c->kv = static_cast<uint8_t*>(kv_workspace);
+  c->kv_layer_bytes = kv_layer_bytes_of(*cfg);
+  c->slots.assign(cfg->buf_slots, Slot{});
+
+  const ScratchPlan p = plan_scratch(*cfg);
+  uint8_t* s = static_cast<uint8_t*>(scratch);
+  c->rope_cos = reinterpret_cast<float*>(s + p.rope_cos);
+  c->rope_sin = reinterpret_cast<float*>(s + p.rope_sin);
+  c->h = reinterpret_cast<__half*>(s + p.h);
+  c->qbuf = reinterpret_cast<__half*>(s + p.qbuf);
+  c->attn = reinterpret_cast<__half*>(s + p.attn);
+  c->x1 = reinterpret_cast<__half*>(s + p.x1);
+  c->act = reinterpret_cast<__half*>(s + p.act);
+  c->xa = reinterpret_cast<__half*>(s + p.xa);
+  c->xb = reinterpret_cast<__half*>(s + p.xb);
+  c->last = reinterpret_cast<__half*>(s + p.last);
+  c->logits = reinterpret_cast<float*>(s + p.logits);
+  c->ids_out = reinterpret_cast<int32_t*>(s + p.ids_out);
+  c->part_o = reinterpret_cast<float*>(s + p.part_o);
+  c->part_ml = reinterpret_cast<float*>(s + p.part_ml);
+  c->stage_in = s + p.stage_in;
+  c->stage_out = s + p.stage_out;
+  c->max_splits = p.max_splits;
+
+  auto cleanup = [&](int code) {
+    if (c->status_host) cudaFreeHost(c->status_host);
+    delete c;
+    return code;
+  };
+  if (cudaHostAlloc(reinterpret_cast<void**>(&c->status_host), 64, cudaHostAllocMapped) != cudaSuccess)
+    return cleanup(THINFER_ECUDA);
+  *c->status_host = 0;
+  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->status_dev), c->status_host, 0) != cudaSuccess)
+    return cleanup(THINFER_ECUDA);
+
+  // tensor maps of the weights: [n_out][k], 128-row x 64-column boxes
+  c->maps.resize(cfg->n_layers);
+  const uint64_t D = cfg->hidden, qd = static_cast<uint64_t>(cfg->n_q_heads) * cfg->head_dim,
+                 kvd = static_cast<uint64_t>(cfg->n_kv_heads) * cfg->head_dim, F = cfg->ffn;
+  bool ok = true;
+  for (int l = 0; l < cfg->n_layers && ok; ++l) {
+    const thinfer_layer_weights& w = c->layers[l];
+    LayerMaps& m = c->maps[l];
+    ok = ok && make_map_2d(&m.wq, w.wq, D, qd, 128) && make_map_2d(&m.wk, w.wk, D, kvd, 128) &&
+         make_map_2d(&m.wv, w.wv, D, kvd, 128) && make_map_2d(&m.wo, w.wo, qd, D, 128) &&
+         make_map_2d(&m.wg, w.w_gate, D, F, 128) && make_map_2d(&m.wu, w.w_up, D, F, 128) &&
+         make_map_2d(&m.wd, w.w_down, F, D, 128);
+  }
+  if (ok && cfg->vocab > 0) ok = make_map_2d(&c->map_head, c->lm_head, D, cfg->vocab, 128);
+  if (!ok) {
+    g_global_err = "cuTensorMapEncodeTiled failed for a weight matrix";
+    return cleanup(THINFER_ECUDA);
+  }
+
+  const int n_tab = cfg->max_seq * (cfg->head_dim / 2);
+  rope_table_kernel<<<(n_tab + 255) / 256, 256>>>(c->rope_cos, c->rope_sin, cfg->max_seq, cfg->head_dim / 2,
+                                                  static_cast<double>(cfg->rope_base));
+  if (cudaDeviceSynchronize() != cudaSuccess) return cleanup(THINFER_ECUDA);
+  *out = c;
+  return THINFER_OK;
+}
+
+int thinfer_prefill(thinfer_ctx* c, int32_t slot, const void* input, int32_t batch, int32_t seq_len, void* out_primary,
+                    void* out_logits, void* cuda_stream) {
+  int rc = check_prefill_args(c, slot, input, batch, seq_len, out_primary, out_logits);
+  if (rc != THINFER_OK) return rc;
+  rc = run_prefill(c, slot, input, batch, seq_len, out_primary, out_logits, static_cast<cudaStream_t>(cuda_stream));
+  if (rc != THINFER_OK) return rc;
+  c->slots[slot].busy = true;
+  c->slots[slot].batch = batch;
+  c->slots[slot].cur_len = seq_len;
+  return THINFER_OK;
+}
+
+int thinfer_decode_step(thinfer_ctx* c, int32_t slot, const void* input, void* out_primary, void* out_logits,
+                        void* cuda_stream) {
+  int rc = check_decode_args(c, slot, input, out_primary, out_logits);
+  if (rc != THINFER_OK) return rc;
+  Slot& s = c->slots[slot];
+  rc = run_decode(c, slot, input, s.batch, s.cur_len, out_primary, out_logits, static_cast<cudaStream_t>(cuda_stream));
+  if (rc != THINFER_OK) return rc;
+  ++s.cur_len;
+  return THINFER_OK;
+}
+
+int thinfer_prefill_host(thinfer_ctx* c, int32_t slot, const void* host_input, int32_t batch, int32_t seq_len,
+                         void* host_out_primary, void* host_out_logits, void* cuda_stream) {
+  int rc = check_prefill_args(c, slot, host_input, batch, seq_len, host_out_primary, host_out_logits);
+  if (rc != THINFER_OK) return rc;
+  const thinfer_config& cf = c->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t rows = static_cast<size_t>(batch) * seq_len;
+  const size_t in_bytes = cf.vocab > 0 ? rows * 4 : rows * cf.hidden * 2;
+  if (cudaMemcpyAsync(c->stage_in, host_input, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return fail(c, THINFER_ECUDA, "host-to-device copy failed");
+  void* d_primary = c->stage_out;
+  float* d_logits = reinterpret_cast<float*>(c->stage_out + static_cast<size_t>(cf.max_batch) * 4);
+  rc = run_prefill(c, slot, c->stage_in, batch, seq_len, (cf.vocab == 0 || host_out_primary) ? d_primary : nullptr,
+                   (cf.vocab > 0 && host_out_logits) ? d_logits : nullptr, st);
+  if (rc != THINFER_OK) return rc;
+  cudaError_t e = cudaSuccess;
+  if (cf.vocab == 0) {
+    e = cudaMemcpyAsync(host_out_primary, d_primary, rows * cf.hidden * 2, cudaMemcpyDeviceToHost, st);
+  } else {
+    if (host_out_primary) e = cudaMemcpyAsync(host_out_primary, d_primary, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && host_out_logits)
+      e = cudaMemcpyAsync(host_out_logits, d_logits, static_cast<size_t>(batch) * cf.vocab * 4, cudaMemcpyDeviceToHost, st);
+  }
+  if (e != cudaSuccess) return fail(c, THINFER_ECUDA, "device-to-host copy failed");
+  c->slots[slot].busy = true;
+  c->slots[slot].batch = batch;
+  c->slots[slot].cur_len = seq_len;
+  return THINFER_OK;
+}
+
+int thinfer_decode_step_host(thinfer_ctx* c, int32_t slot, const void* host_input, void* host_out_primary,
+                             void* host_out_logits, void* cuda_stream) {
+  int rc = check_decode_args(c, slot, host_input, host_out_primary, host_out_logits);
+  if (rc != THINFER_OK) return rc;
+  const thinfer_config& cf = c->cfg;
+  Slot& s = c->slots[slot];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t in_bytes = cf.vocab > 0 ? static_cast<size_t>(s.batch) * 4 : static_cast<size_t>(s.batch) * cf.hidden * 2;
+  if (cudaMemcpyAsync(c->stage_in, host_input, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return fail(c, THINFER_ECUDA, "host-to-device copy failed");
+  void* d_primary = c->stage_out;
+  float* d_logits = reinterpret_cast<float*>(c->stage_out + static_cast<size_t>(cf.max_batch) * 4);
+  rc = run_decode(c, slot, c->stage_in, s.batch, s.cur_len, (cf.vocab == 0 || host_out_primary) ? d_primary : nullptr,
+                  (cf.vocab > 0 && host_out_logits) ? d_logits : nullptr, st);
+  if (rc != THINFER_OK) return rc;
+  cudaError_t e = cudaSuccess;
+  if (cf.vocab == 0) {
+    e = cudaMemcpyAsync(host_out_primary, d_primary, static_cast<size_t>(s.batch) * cf.hidden * 2, cudaMemcpyDeviceToHost, st);
+  } else {
+    if (host_out_primary) e = cudaMemcpyAsync(host_out_primary, d_primary, static_cast<size_t>(s.batch) * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && host_out_logits)
+      e = cudaMemcpyAsync(host_out_logits, d_logits, static_cast<size_t>(s.batch) * cf.vocab * 4, cudaMemcpyDeviceToHost, st);
+  }
+  if (e != cudaSuccess) return fail(c, THINFER_ECUDA, "device-to-host copy failed");
+  ++s.cur_len;
+  return THINFER_OK;
+}
+
+int thinfer_release_slot(thinfer_ctx* c, int32_t slot, void* /*cuda_stream*/) {
+  if (c == nullptr) return THINFER_EINVAL;
+  if (slot < 0 || slot >= c->cfg.buf_slots) return fail(c, THINFER_EINVAL, "slot %d outside [0, %d)", slot, c->cfg.buf_slots);
+  c->slots[slot] = Slot{};
+  return THINFER_OK;
+}
+
+int thinfer_slot_state(const thinfer_ctx* c, int32_t slot, int32_t* batch, int32_t* cur_len) {
+  if (c == nullptr || slot < 0 || slot >= c->cfg.buf_slots) return THINFER_EINVAL;
+  if (batch) *batch = c->slots[slot].batch;
+  if (cur_len) *cur_len = c->slots[slot].cur_len;
+  return THINFER_OK;
+}
+
+int thinfer_kv_pointer(const thinfer_ctx* c, int32_t slot, int32_t layer, int32_t which, void** device_ptr) {
+  if (c == nullptr || device_ptr == nullptr || slot < 0 || slot >= c->cfg.buf_slots || layer < 0 ||
+      layer >= c->cfg.n_layers || which < 0 || which > 1)
+    return THINFER_EINVAL;
+  *device_ptr = kv_ptr(const_cast<thinfer_ctx*>(c), slot, layer, which);
+  return THINFER_OK;
+}
+
+int thinfer_status(thinfer_ctx* c, int32_t* device_status) {
+  if (c == nullptr || device_status == nullptr) return THINFER_EINVAL;
+  *device_status = *reinterpret_cast<volatile int*>(c->status_host);
+  return THINFER_OK;
+}
+
+int thinfer_set_launch_mode(thinfer_ctx* c, int32_t mode) {
+  if (c == nullptr) return THINFER_EINVAL;
+  if (mode != 0) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
+  c->launch_mode = mode;
+  return THINFER_OK;
+}
+
+int thinfer_profile_select(thinfer_ctx* c, int32_t kernel_id) {
+  if (c == nullptr || kernel_id < -1 || kernel_id >= THINFER_K_COUNT) return THINFER_EINVAL;
+  c->prof_kernel = kernel_id;
+  c->prof_used = 0;
+  return THINFER_OK;
+}
+
+int thinfer_profile_read(thinfer_ctx* c, int32_t* launches, float* total_ms) {
+  if (c == nullptr || launches == nullptr || total_ms == nullptr) return THINFER_EINVAL;
+  float sum = 0.f;
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(c->prof_events[i].end) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, c->prof_events[i].beg, c->prof_events[i].end) != cudaSuccess)
+      return fail(c, THINFER_ECUDA, "reading profile events failed");
+    sum += ms;
+  }
+  *launches = static_cast<int32_t>(c->prof_used);
+  *total_ms = sum;
+  c->prof_used = 0;
+  return THINFER_OK;
+}
+
+int64_t thinfer_launch_count(const thinfer_ctx* c) { return c ? c->launches : 0; }
+
+const char* thinfer_last_error(const thinfer_ctx* c) { return c ? c->err.c_str() : g_global_err.c_str(); }
+
+void thinfer_destroy(thinfer_ctx* c) {
+  if (c == nullptr) return;
+  for (ProfEvent& e : c->prof_events) {
+    cudaEventDestroy(e.beg);
+    cudaEventDestroy(e.end);
+  }
+  if (c->status_host) cudaFreeHost(c->status_host);
+  delete c;
+}
+
+// ---------------------------------------------------------------- operators
+int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k, int32_t out_fp32,
+                      int32_t path, void* cuda_stream) {
+  if (x == nullptr || w == nullptr || y == nullptr || rows <= 0 || n_out <= 0 || k <= 0) return THINFER_EINVAL;
+  if (k % 8 != 0 || n_out % 2 != 0) return THINFER_EUNSUPPORTED;
+  Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
+  EpiArgs e{};
+  e.out = y;
+  e.ld_out = n_out;
+  const int n[3] = {n_out, 0, 0};
+  if (path == 1) {
+    if (rows > 16) return THINFER_EUNSUPPORTED;
+    if (out_fp32)
+      gemv<EPI_PLAIN_F32, false>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k,
+                                 static_cast<const __half*>(x), k, rows, nullptr, 0.f, e);
+    else
+      gemv<EPI_PLAIN_F16, false>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k,
+                                 static_cast<const __half*>(x), k, rows, nullptr, 0.f, e);
+  } else if (path == 0) {
+    CUtensorMap mw;
+    if (!make_map_2d(&mw, w, k, n_out, 128)) return THINFER_ECUDA;
+    if (out_fp32) tc_linear<EPI_PLAIN_F32>(L, -2, mw, mw, mw, static_cast<const __half*>(x), rows, k, n, e);
+    else tc_linear<EPI_PLAIN_F16>(L, -2, mw, mw, mw, static_cast<const __half*>(x), rows, k, n, e);
+  } else {
+    return THINFER_EINVAL;
+  }
+  return L.rc;
+}
+
+int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, void* out, int32_t batch,
+                                 int32_t n_q_heads, int32_t n_kv_heads, int32_t seq, int32_t kv_stride,
+                                 int32_t head_dim, void* cuda_stream) {
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || batch <= 0 || n_q_heads <= 0 ||
+      n_kv_heads <= 0 || seq <= 0 || kv_stride < seq)
+    return THINFER_EINVAL;
+  if ((head_dim != 64 && head_dim != 128) || n_q_heads % n_kv_heads != 0) return THINFER_EUNSUPPORTED;
+  Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
+  attn_prefill(L, static_cast<const __half*>(q), static_cast<const __half*>(k), static_cast<const __half*>(v),
+               static_cast<__half*>(out), batch, n_q_heads, n_kv_heads, seq, kv_stride, head_dim, nullptr);
+  return L.rc;
+}
+
+int thinfer_op_rmsnorm(const void* x, const void* gain, void* y, int32_t rows, int32_t n, float eps, void* cuda_stream) {
+  if (x == nullptr || gain == nullptr || y == nullptr || rows <= 0 || n <= 0) return THINFER_EINVAL;
+  if (n % 8 != 0) return THINFER_EUNSUPPORTED;
+  Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
+  rmsnorm_rows(L, static_cast<const __half*>(x), static_cast<const __half*>(gain), static_cast<__half*>(y), rows, n, eps);
+  return L.rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,275 @@
+"""ctypes binding over libthinfer.so (include/thinfer.h).
+
+Argument marshalling only: torch supplies device memory and streams, every step
+of the path runs in the library's CUDA kernels.  There is no CPU fallback: if
+the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libthinfer.so")
+
+OK, EINVAL, EUNSUPPORTED, ECAPACITY, EBUSY, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+ERR_NAMES = {OK: "THINFER_OK", EINVAL: "THINFER_EINVAL", EUNSUPPORTED: "THINFER_EUNSUPPORTED",
+             ECAPACITY: "THINFER_ECAPACITY", EBUSY: "THINFER_EBUSY", ECUDA: "THINFER_ECUDA",
+             ETIMEOUT: "THINFER_ETIMEOUT"}
+K_RMSNORM, K_QKV, K_ATTN, K_ATTN_COMBINE, K_OPROJ, K_GATEUP, K_DOWN, K_HEAD, K_EMBED, K_ARGMAX = range(10)
+
+EXPORTS = (
+    "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_decode_step",
+    "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
+    "thinfer_kv_pointer", "thinfer_status", "thinfer_set_launch_mode", "thinfer_profile_select",
+    "thinfer_profile_read", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
+    "thinfer_op_linear", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
+)
+
+
+class ThinferError(RuntimeError):
+    def __init__(self, code, what=""):
+        self.code = code
+        super().__init__(f"{ERR_NAMES.get(code, code)}: {what}")
+
+
+class Config(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("ffn", C.c_int32), ("n_layers", C.c_int32), ("vocab", C.c_int32),
+                ("rms_eps", C.c_float), ("rope_base", C.c_float), ("max_batch", C.c_int32),
+                ("max_seq", C.c_int32), ("buf_slots", C.c_int32)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")]
+
+
+class Weights(C.Structure):
+    _fields_ = [("layers", C.POINTER(LayerWeights)), ("embed", C.c_void_p), ("final_norm", C.c_void_p),
+                ("lm_head", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library (once).  Fails loudly when it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ThinferError(ECUDA, f"{LIB_PATH} is missing: build it with "
+                                  "`python -m paper_2605_25655_b200._build` (needs nvcc)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    L.thinfer_workspace_bytes.argtypes = [C.POINTER(Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.thinfer_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
+    L.thinfer_prefill.argtypes = [vp, i32, vp, i32, i32, vp, vp, vp]
+    L.thinfer_decode_step.argtypes = [vp, i32, vp, vp, vp, vp]
+    L.thinfer_prefill_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, vp]
+    L.thinfer_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp]
+    L.thinfer_release_slot.argtypes = [vp, i32, vp]
+    L.thinfer_slot_state.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32)]
+    L.thinfer_kv_pointer.argtypes = [vp, i32, i32, i32, C.POINTER(vp)]
+    L.thinfer_status.argtypes = [vp, C.POINTER(i32)]
+    L.thinfer_set_launch_mode.argtypes = [vp, i32]
+    L.thinfer_profile_select.argtypes = [vp, i32]
+    L.thinfer_profile_read.argtypes = [vp, C.POINTER(i32), C.POINTER(C.c_float)]
+    L.thinfer_launch_count.argtypes = [vp]
+    L.thinfer_launch_count.restype = i64
+    L.thinfer_last_error.argtypes = [vp]
+    L.thinfer_last_error.restype = C.c_char_p
+    L.thinfer_destroy.argtypes = [vp]
+    L.thinfer_destroy.restype = None
+    L.thinfer_op_linear.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+    L.thinfer_op_attention_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    L.thinfer_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, C.c_float, vp]
+    _lib = L
+    return L
+
+
+def _check(rc, ctx=None):
+    if rc != OK:
+        msg = lib().thinfer_last_error(ctx)
+        raise ThinferError(rc, msg.decode() if msg else "")
+
+
+def _stream_ptr(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def make_config(shape, max_batch, max_seq, buf_slots=1) -> Config:
+    """shape: any object with the fields of synth.Shape."""
+    return Config(shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn, shape.n_layers,
+                  shape.vocab, shape.rms_eps, shape.rope_base, max_batch, max_seq, buf_slots)
+
+
+def workspace_bytes(cfg: Config):
+    kv, sc = C.c_size_t(0), C.c_size_t(0)
+    _check(lib().thinfer_workspace_bytes(C.byref(cfg), C.byref(kv), C.byref(sc)))
+    return kv.value, sc.value
+
+
+class Context:
+    """One thinfer_ctx plus the torch tensors that back its caller-owned memory.
+
+    layers: list of dicts name -> CUDA FP16 tensor (names of thinfer_layer_weights);
+    stack:  dict with embed / final_norm / lm_head when shape.vocab > 0.
+    """
+
+    def __init__(self, shape, layers, stack=None, max_batch=1, max_seq=128, buf_slots=1, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.shape = shape
+        self.device = torch.device(device)
+        self.cfg = make_config(shape, max_batch, max_seq, buf_slots)
+        kv_bytes, scratch_bytes = workspace_bytes(self.cfg)
+        with torch.cuda.device(self.device):
+            self.kv = torch.empty(kv_bytes, dtype=torch.uint8, device=self.device)
+            self.scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=self.device)
+            self._keep = (layers, stack)
+            arr = (LayerWeights * shape.n_layers)()
+            for l, w in enumerate(layers):
+                for name, _ in LayerWeights._fields_:
+                    t = w[name]
+                    assert t.is_cuda and t.dtype == torch.float16 and t.is_contiguous(), name
+                    setattr(arr[l], name, t.data_ptr())
+            wts = Weights(arr, None, None, None)
+            if shape.vocab > 0:
+                wts.embed, wts.final_norm, wts.lm_head = (stack[n].data_ptr() for n in ("embed", "final_norm", "lm_head"))
+            h = C.c_void_p(None)
+            _check(lib().thinfer_create(C.byref(self.cfg), C.byref(wts), self.kv.data_ptr(), kv_bytes,
+                                        self.scratch.data_ptr(), scratch_bytes, C.byref(h)))
+        self.h = h
+
+    # -- device-buffer calls ------------------------------------------------
+    def prefill(self, inp, slot=0, stream=None, want_logits=False):
+        torch = self.torch
+        batch, seq = int(inp.shape[0]), int(inp.shape[1])
+        assert inp.is_cuda and inp.is_contiguous()
+        if self.shape.vocab == 0:
+            assert inp.dtype == torch.float16
+            out = torch.empty_like(inp)
+            _check(lib().thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, out.data_ptr(), None,
+                                         _stream_ptr(stream)), self.h)
+            return out
+        assert inp.dtype == torch.int32
+        ids = torch.empty(batch, dtype=torch.int32, device=self.device)
+        logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        _check(lib().thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, ids.data_ptr(),
+                                     logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        return (ids, logits) if want_logits else ids
+
+    def decode_step(self, inp, slot=0, stream=None, want_logits=False, out=None):
+        torch = self.torch
+        assert inp.is_cuda and inp.is_contiguous()
+        if self.shape.vocab == 0:
+            out = torch.empty_like(inp) if out is None else out
+            _check(lib().thinfer_decode_step(self.h, slot, inp.data_ptr(), out.data_ptr(), None,
+                                             _stream_ptr(stream)), self.h)
+            return out
+        batch = int(inp.shape[0])
+        ids = torch.empty(batch, dtype=torch.int32, device=self.device) if out is None else out
+        logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        _check(lib().thinfer_decode_step(self.h, slot, inp.data_ptr(), ids.data_ptr(),
+                                         logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        return (ids, logits) if want_logits else ids
+
+    # -- host-buffer calls (pinned tensors make the copies asynchronous) -----
+    def prefill_host(self, host_in, host_out, slot=0, stream=None, host_logits=None):
+        batch, seq = int(host_in.shape[0]), int(host_in.shape[1])
+        _check(lib().thinfer_prefill_host(self.h, slot, host_in.data_ptr(), batch, seq, host_out.data_ptr(),
+                                          host_logits.data_ptr() if host_logits is not None else None,
+                                          _stream_ptr(stream)), self.h)
+
+    def decode_step_host(self, host_in, host_out, slot=0, stream=None, host_logits=None):
+        _check(lib().thinfer_decode_step_host(self.h, slot, host_in.data_ptr(), host_out.data_ptr(),
+                                              host_logits.data_ptr() if host_logits is not None else None,
+                                              _stream_ptr(stream)), self.h)
+
+    # -- bookkeeping ----------------------------------------------------------
+    def release_slot(self, slot=0):
+        _check(lib().thinfer_release_slot(self.h, slot, None), self.h)
+
+    def slot_state(self, slot=0):
+        b, n = C.c_int32(0), C.c_int32(0)
+        _check(lib().thinfer_slot_state(self.h, slot, C.byref(b), C.byref(n)), self.h)
+        return b.value, n.value
+
+    def kv_view(self, slot, layer, which):
+        """Strided torch view [max_batch][n_kv_heads][max_seq][head_dim] of K (0) or V (1)."""
+        p = C.c_void_p(None)
+        _check(lib().thinfer_kv_pointer(self.h, slot, layer, which, C.byref(p)), self.h)
+        off = p.value - self.kv.data_ptr()
+        n = self.cfg.max_batch * self.cfg.n_kv_heads * self.cfg.max_seq * self.cfg.head_dim
+        return self.kv[off:off + 2 * n].view(self.torch.float16).view(
+            self.cfg.max_batch, self.cfg.n_kv_heads, self.cfg.max_seq, self.cfg.head_dim)
+
+    def status(self):
+        v = C.c_int32(0)
+        _check(lib().thinfer_status(self.h, C.byref(v)), self.h)
+        return v.value
+
+    def set_launch_mode(self, mode):
+        _check(lib().thinfer_set_launch_mode(self.h, mode), self.h)
+
+    def profile_select(self, kernel_id):
+        _check(lib().thinfer_profile_select(self.h, kernel_id), self.h)
+
+    def profile_read(self):
+        n, ms = C.c_int32(0), C.c_float(0)
+        _check(lib().thinfer_profile_read(self.h, C.byref(n), C.byref(ms)), self.h)
+        return n.value, ms.value
+
+    def launch_count(self):
+        return int(lib().thinfer_launch_count(self.h))
+
+    def close(self):
+        if self.h is not None and self.h.value:
+            lib().thinfer_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+# ---------------------------------------------------------------- operators
+def op_linear(x, w, out_fp32=False, path=0, stream=None):
+    import torch
+    rows, k = x.shape
+    n_out = w.shape[0]
+    y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else torch.float16, device=x.device)
+    _check(lib().thinfer_op_linear(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k, int(out_fp32), path,
+                                   _stream_ptr(stream)))
+    return y
+
+
+def op_attention_prefill(q, k, v, seq=None, stream=None):
+    """q [B, Hq, S, d]; k, v [B, Hkv, T, d] with T >= S (the first S positions are used) -> [B, S, Hq*d]."""
+    import torch
+    b, hq, s, d = q.shape
+    hkv, t = k.shape[1], k.shape[2]
+    out = torch.empty(b, s, hq * d, dtype=torch.float16, device=q.device)
+    _check(lib().thinfer_op_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), b, hq, hkv,
+                                              s, t, d, _stream_ptr(stream)))
+    return out
+
+
+def op_rmsnorm(x, gain, eps, stream=None):
+    import torch
+    rows, n = x.shape
+    y = torch.empty_like(x)
+    _check(lib().thinfer_op_rmsnorm(x.data_ptr(), gain.data_ptr(), y.data_ptr(), rows, n, eps, _stream_ptr(stream)))
+    return y
+
+
+def to_device_layers(np_layers, device="cuda:0"):
+    """numpy FP16 weight dicts (synth.layer_weights) -> torch CUDA tensors."""
+    import torch
+    return [{k: torch.from_numpy(v).to(device) for k, v in w.items()} for w in np_layers]

@@ -1,0 +1,217 @@
+"""The layer and stack through the C ABI (thinfer_create / prefill / decode_step)
+against the oracle on the same seeded inputs (run with -m gpu on a B200).
+
+Per-layer checks are chained: the oracle is fed the same FP16 inputs as the GPU.
+Tolerance: max |err| <= 2e-2 x row RMS and cosine >= 0.999 (tests/parity.py)."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2605_25655_b200 import synth
+from tests.parity import assert_rows_close, oracle_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def T():
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    thinfer.lib()
+    return torch, thinfer
+
+
+def _ctx(T, shape, np_layers, max_batch, max_seq, stack=None, buf_slots=1):
+    torch, thinfer = T
+    layers = thinfer.to_device_layers(np_layers)
+    st = {k: torch.from_numpy(v).cuda() for k, v in stack.items() if k != "layers"} if stack else None
+    return thinfer.Context(shape, layers, st, max_batch=max_batch, max_seq=max_seq, buf_slots=buf_slots)
+
+
+def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_seq=None):
+    """Prefill `seq` tokens then `n_decode` decode steps on seeded hidden states; compare everything."""
+    torch, thinfer = T
+    cfg = oracle_config(shape)
+    w = synth.layer_weights(shape, seed)
+    x = synth.hidden_states(shape, seed, (batch, seq + n_decode))
+    ctx = _ctx(T, shape, [w], batch, max_seq or (seq + n_decode))
+    xd = torch.from_numpy(x).cuda()
+    out = ctx.prefill(xd[:, :seq].contiguous())
+    dec = [ctx.decode_step(xd[:, seq + i].contiguous()) for i in range(n_decode)]
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    assert ctx.slot_state(0) == (batch, seq + n_decode)
+    bs = list(range(batch)) if check_batches is None else check_batches
+    ref, kc, vc = O.layer_prefill(cfg, w, x[bs, :seq])
+    got = out.cpu().numpy()[bs]
+    stats = [assert_rows_close(got, ref, f"prefill B={batch} S={seq}")]
+    kg = ctx.kv_view(0, 0, 0).cpu().numpy()[bs]
+    vg = ctx.kv_view(0, 0, 1).cpu().numpy()[bs]
+    assert_rows_close(kg[:, :, :seq], kc, "K cache after prefill", max_err=6e-3)
+    assert_rows_close(vg[:, :, :seq], vc, "V cache after prefill", max_err=6e-3)
+    # decode: the oracle continues from the GPU's own FP16 cache (chained check)
+    k_run = kg[:, :, :seq].astype(np.float64)
+    v_run = vg[:, :, :seq].astype(np.float64)
+    for i in range(n_decode):
+        r, k_run, v_run = O.layer_decode(cfg, w, x[bs, seq + i], k_run, v_run, seq + i)
+        stats.append(assert_rows_close(dec[i].cpu().numpy()[bs], r, f"decode step {i} B={batch}"))
+        kg = ctx.kv_view(0, 0, 0).cpu().numpy()[bs]
+        vg = ctx.kv_view(0, 0, 1).cpu().numpy()[bs]
+        assert_rows_close(kg[:, :, seq + i], k_run[:, :, seq + i], f"K append {i}", max_err=6e-3)
+        assert_rows_close(vg[:, :, seq + i], v_run[:, :, seq + i], f"V append {i}", max_err=6e-3)
+        k_run[:, :, seq + i] = kg[:, :, seq + i]
+        v_run[:, :, seq + i] = vg[:, :, seq + i]
+    ctx.close()
+    return stats
+
+
+def test_tiny_config_prefill_then_decode(T):
+    # configuration 1: hidden 256, 4 x 64 heads, FFN 688, batch 1, prompt 32, 8 decode steps
+    _layer_case(T, synth.TINY, batch=1, seq=32, n_decode=8)
+
+
+@pytest.mark.parametrize("batch,seq,n_decode", [(2, 1, 6), (3, 130, 3), (4, 77, 2), (16, 40, 2)])
+def test_tiny_shapes_ragged(T, batch, seq, n_decode):
+    _layer_case(T, synth.TINY, batch=batch, seq=seq, n_decode=n_decode, seed=batch)
+
+
+def test_gqa_layer(T):
+    shape = synth.Shape(hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1024)
+    _layer_case(T, shape, batch=2, seq=150, n_decode=3, seed=4)
+
+
+def test_decode_equals_last_row_of_prefill(T):
+    # the cache is built one token at a time; each step must equal the oracle's full prefill row
+    torch, thinfer = T
+    shape = synth.TINY
+    cfg = oracle_config(shape)
+    w = synth.layer_weights(shape, 2)
+    x = synth.hidden_states(shape, 2, (2, 20))
+    ref, _, _ = O.layer_prefill(cfg, w, x)
+    ctx = _ctx(T, shape, [w], 2, 32)
+    xd = torch.from_numpy(x).cuda()
+    first = ctx.prefill(xd[:, :1].contiguous())
+    assert_rows_close(first.cpu().numpy(), ref[:, :1], "prefill of one token")
+    for t in range(1, 20):
+        out = ctx.decode_step(xd[:, t].contiguous())
+        assert_rows_close(out.cpu().numpy(), ref[:, t], f"incremental decode t={t}")
+    ctx.close()
+
+
+def test_batch_independence(T):
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 0)
+    x = synth.hidden_states(shape, 0, (3, 24))
+    ctx = _ctx(T, shape, [w], 3, 32)
+    xd = torch.from_numpy(x).cuda()
+    base = ctx.prefill(xd.contiguous()).cpu().numpy()
+    ctx.release_slot(0)
+    x2 = x.copy()
+    x2[1] = -x2[1]
+    other = ctx.prefill(torch.from_numpy(x2).cuda()).cpu().numpy()
+    np.testing.assert_array_equal(other[0], base[0])
+    np.testing.assert_array_equal(other[2], base[2])
+    assert not np.array_equal(other[1], base[1])
+    ctx.close()
+
+
+def test_llama7b_layer_batch1_full(T):
+    # configuration 2 at batch 1: 512-token prompt, decode steps at T = 512, 513, 514
+    _layer_case(T, synth.LLAMA_7B_LAYER, batch=1, seq=512, n_decode=3, max_seq=640)
+
+
+@pytest.mark.parametrize("batch", [4, 16])
+def test_llama7b_layer_batched_subset(T, batch):
+    # configuration 2 at batch 4 / 16: first and last request checked (batch independence covers the rest)
+    _layer_case(T, synth.LLAMA_7B_LAYER, batch=batch, seq=512, n_decode=2, check_batches=[0, batch - 1], max_seq=640)
+
+
+def test_stack_teacher_forced(T):
+    torch, thinfer = T
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=688, n_layers=3, vocab=1000)
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, 1)
+    ids = synth.token_ids(shape, 1, (2, 20))
+    ctx = _ctx(T, shape, sw["layers"], 2, 32, stack=sw)
+    idd = torch.from_numpy(ids).cuda()
+    nxt, logits = ctx.prefill(idd[:, :16].contiguous(), want_logits=True)
+    ref_logits, ref_next, caches, _ = O.stack_prefill(cfg, sw, ids[:, :16])
+    assert_rows_close(logits.cpu().numpy(), ref_logits, "prefill logits")
+    _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
+    for t in range(16, 20):                                   # teacher forced: both sides consume the same ids
+        nxt, logits = ctx.decode_step(idd[:, t].contiguous(), want_logits=True)
+        ref_logits, ref_next, caches, _ = O.stack_decode(cfg, sw, ids[:, t], caches, t)
+        assert_rows_close(logits.cpu().numpy(), ref_logits, f"decode logits t={t}")
+        _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
+    assert ctx.status() == 0
+    ctx.close()
+
+
+def _check_greedy(ids, gpu_logits, ref_logits):
+    # the GPU's pick is the lowest-index argmax of its own logits (bit exact), and agrees with the
+    # oracle wherever the oracle's top-2 gap is larger than 4x the logit error
+    np.testing.assert_array_equal(ids, np.argmax(gpu_logits, axis=-1))
+    err = np.max(np.abs(gpu_logits - ref_logits), axis=-1)
+    top2 = np.sort(ref_logits, axis=-1)[:, -2:]
+    clear = (top2[:, 1] - top2[:, 0]) > 4 * err
+    np.testing.assert_array_equal(ids[clear], np.argmax(ref_logits, axis=-1)[clear])
+
+
+def test_errors_and_slots(T):
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 0)
+    ctx = _ctx(T, shape, [w], 2, 8, buf_slots=2)
+    x = torch.from_numpy(synth.hidden_states(shape, 0, (2, 8))).cuda()
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.decode_step(x[:, 0].contiguous())                  # empty slot
+    assert e.value.code == thinfer.EINVAL
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.prefill(torch.cat([x, x], dim=1))                  # 16 > max_seq
+    assert e.value.code == thinfer.ECAPACITY
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.prefill(torch.cat([x, x, x], dim=0))               # batch 6 > max_batch
+    assert e.value.code == thinfer.ECAPACITY
+    a = ctx.prefill(x[:, :7].contiguous(), slot=0)
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.prefill(x[:, :7].contiguous(), slot=0)             # back-pressure: slot not released
+    assert e.value.code == thinfer.EBUSY
+    b = ctx.prefill(x[:, :7].contiguous(), slot=1)             # the second slot is free
+    np.testing.assert_array_equal(a.cpu().numpy(), b.cpu().numpy())
+    ctx.decode_step(x[:, 7].contiguous(), slot=0)
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.decode_step(x[:, 7].contiguous(), slot=0)          # slot full
+    assert e.value.code == thinfer.ECAPACITY
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.prefill(x, slot=5)
+    assert e.value.code == thinfer.EINVAL
+    ctx.release_slot(0)
+    assert ctx.slot_state(0) == (0, 0)
+    ctx.prefill(x[:, :3].contiguous(), slot=0)
+    assert ctx.slot_state(0) == (2, 3) and ctx.slot_state(1) == (2, 7)
+    assert ctx.launch_count() > 0 and ctx.status() == 0
+    ctx.close()
+
+
+def test_host_buffer_calls_match_device_calls(T):
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 3)
+    x = torch.from_numpy(synth.hidden_states(shape, 3, (2, 12)))
+    ctx = _ctx(T, shape, [w], 2, 16, buf_slots=2)
+    dev = ctx.prefill(x[:, :11].contiguous().cuda(), slot=0)
+    dev2 = ctx.decode_step(x[:, 11].contiguous().cuda(), slot=0)
+    hin = x[:, :11].contiguous().pin_memory()
+    hout = torch.empty_like(hin).pin_memory()
+    ctx.prefill_host(hin, hout, slot=1)
+    hin2 = x[:, 11].contiguous().pin_memory()
+    hout2 = torch.empty_like(hin2).pin_memory()
+    ctx.decode_step_host(hin2, hout2, slot=1)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(hout.numpy(), dev.cpu().numpy())
+    np.testing.assert_array_equal(hout2.numpy(), dev2.cpu().numpy())
+    ctx.close()

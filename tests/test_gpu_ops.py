@@ -1,0 +1,105 @@
+"""Single operators through the C ABI against the oracle (run with -m gpu on a B200)."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from tests.parity import assert_rows_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def T():
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    thinfer.lib()
+    return torch, thinfer
+
+
+def _rand16(rng, shape, std):
+    return (rng.standard_normal(shape) * std).astype(np.float16)
+
+
+# rows, n_out, k: multi-tile with ragged tails in every dimension; k = 688 is not a multiple of 64
+LINEAR_SHAPES = [(32, 256, 256), (32, 256, 688), (5, 130, 72), (300, 1376, 256), (512, 384, 4096), (1, 4096, 4096),
+                 (16, 1000, 1024), (129, 128, 64), (700, 300, 520)]
+
+
+@pytest.mark.parametrize("rows,n_out,k", LINEAR_SHAPES)
+@pytest.mark.parametrize("out_fp32", [False, True])
+def test_linear_tensor_core_path(T, rows, n_out, k, out_fp32):
+    torch, thinfer = T
+    rng = np.random.default_rng(rows * 7 + n_out)
+    x, w = _rand16(rng, (rows, k), 1.0), _rand16(rng, (n_out, k), 0.05)
+    y = thinfer.op_linear(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda(), out_fp32=out_fp32, path=0)
+    torch.cuda.synchronize()
+    assert_rows_close(y.cpu().numpy(), O.linear(x, w), f"linear tc {rows}x{n_out}x{k}", max_err=4e-3)
+
+
+@pytest.mark.parametrize("rows,n_out,k", [(1, 256, 256), (2, 130, 72), (3, 1376, 688), (4, 4096, 4096), (7, 256, 11008),
+                                          (16, 512, 1024)])
+def test_linear_streaming_path(T, rows, n_out, k):
+    torch, thinfer = T
+    rng = np.random.default_rng(rows * 11 + k)
+    x, w = _rand16(rng, (rows, k), 1.0), _rand16(rng, (n_out, k), 0.05)
+    for fp32 in (False, True):
+        y = thinfer.op_linear(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda(), out_fp32=fp32, path=1)
+        torch.cuda.synchronize()
+        assert_rows_close(y.cpu().numpy(), O.linear(x, w), f"linear gemv {rows}x{n_out}x{k}", max_err=4e-3)
+
+
+def test_linear_identity_weight_is_exact(T):
+    torch, thinfer = T
+    rng = np.random.default_rng(5)
+    x = _rand16(rng, (40, 192), 1.0)
+    w = np.eye(192, dtype=np.float16)
+    for path in (0, 1):
+        xs = x[:16] if path == 1 else x
+        y = thinfer.op_linear(torch.from_numpy(xs).cuda(), torch.from_numpy(w).cuda(), path=path)
+        np.testing.assert_array_equal(y.cpu().numpy(), xs)
+
+
+@pytest.mark.parametrize("rows,n", [(1, 256), (37, 4096), (300, 8192), (9, 688)])
+def test_rmsnorm(T, rows, n):
+    torch, thinfer = T
+    rng = np.random.default_rng(n)
+    x = _rand16(rng, (rows, n), 2.0)
+    g = (1.0 + 0.1 * rng.standard_normal(n)).astype(np.float16)
+    y = thinfer.op_rmsnorm(torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda(), 1e-5)
+    assert_rows_close(y.cpu().numpy(), O.rmsnorm(x, g, 1e-5), f"rmsnorm {rows}x{n}", max_err=3e-3)
+
+
+# batch, q heads, kv heads, seq, cache stride, head_dim
+ATTN_SHAPES = [(1, 4, 4, 32, 40, 64), (2, 4, 2, 128, 128, 128), (1, 2, 2, 129, 200, 128), (2, 8, 2, 300, 384, 64),
+               (1, 32, 32, 512, 640, 128), (1, 1, 1, 1, 8, 128), (1, 2, 1, 77, 77, 64)]
+
+
+@pytest.mark.parametrize("b,hq,hkv,s,t,d", ATTN_SHAPES)
+def test_attention_prefill(T, b, hq, hkv, s, t, d):
+    torch, thinfer = T
+    rng = np.random.default_rng(s * 3 + d)
+    q, k, v = _rand16(rng, (b, hq, s, d), 1.0), _rand16(rng, (b, hkv, t, d), 1.0), _rand16(rng, (b, hkv, t, d), 1.0)
+    # positions past the sequence hold garbage the kernel must never let through
+    k[:, :, s:, :] = np.float16(np.nan)
+    v[:, :, s:, :] = np.float16(np.inf)
+    out = thinfer.op_attention_prefill(torch.from_numpy(q).cuda(), torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda())
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    for bi in range(b):
+        ref = O.causal_attention(q[bi], k[bi, :, :s], v[bi, :, :s])
+        assert_rows_close(got[bi], ref, f"attention b{bi} S={s} d={d}", max_err=6e-3)
+
+
+def test_attention_first_row_returns_v0_and_uniform_keys_give_running_mean(T):
+    torch, thinfer = T
+    rng = np.random.default_rng(9)
+    s, d = 200, 128
+    q = _rand16(rng, (1, 2, s, d), 1.0)
+    k = np.broadcast_to(_rand16(rng, (1, 2, 1, d), 1.0), (1, 2, s, d)).copy()
+    v = _rand16(rng, (1, 2, s, d), 1.0)
+    out = thinfer.op_attention_prefill(torch.from_numpy(q).cuda(), torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda())
+    got = out.cpu().numpy().reshape(s, 2, d).astype(np.float64)
+    np.testing.assert_allclose(got[0], v[0, :, 0, :].astype(np.float64), rtol=2e-3, atol=2e-3)
+    mean = np.cumsum(v[0].astype(np.float64), axis=1) / np.arange(1, s + 1)[None, :, None]
+    np.testing.assert_allclose(got, mean.transpose(1, 0, 2), rtol=0, atol=4e-3)
