@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: one Llama-7B-shaped decoder layer, FP16, on B200.
+
+A step = one pass of the whole path over one batch of synthetic input:
+prefill of `batch` prompts of 512 tokens, then 128 decode steps over the FP16
+KV cache.  The headline value is decode tokens/s (batch x 128 / decode time);
+prefill tokens/s and both roofline fractions are reported beside it.
+
+  python bench.py --gpus 1 --steps K --warmup W          # this library
+  python bench.py --impl reference ...                    # the CPU oracle, timed on the host cores
+
+With N > 1 (under torchrun) every rank runs an independent replica of the same
+workload on its own GPU: the path has no exchange step, so there is no
+collective on the data path; times are the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_25655_b200 import synth  # noqa: E402
+
+PROMPT = 512
+GEN = 128
+SHAPE = synth.LLAMA_7B_LAYER
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------- #
+# algorithmic bytes / flops (stated in the design doc)
+# --------------------------------------------------------------------------- #
+def layer_weight_elems(s):
+    qd, kvd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    return s.hidden * (qd + 2 * kvd) + qd * s.hidden + 3 * s.ffn * s.hidden
+
+
+def decode_step_bytes(s, batch, t_len):
+    """Weights once + gains, KV read (t_len keys) and append, activations in/out."""
+    kv = batch * 2 * t_len * s.n_kv_heads * s.head_dim * 2
+    app = batch * 2 * s.n_kv_heads * s.head_dim * 2
+    act = batch * s.hidden * 2 * 2
+    return 2 * layer_weight_elems(s) + 2 * 2 * s.hidden + kv + app + act
+
+
+def gateup_gemv_bytes(s, batch):
+    return 2 * (2 * s.ffn * s.hidden) + 2 * s.hidden + batch * s.hidden * 2 + batch * s.ffn * 2
+
+
+def prefill_flops(s, rows, seq):
+    gemm = 2.0 * rows * layer_weight_elems(s)
+    attn = 2.0 * rows * seq * s.head_dim * s.n_q_heads      # causal: QK^T and PV, half of 4*S^2*d
+    return gemm, attn
+
+
+def gateup_gemm_flops(s, rows):
+    return 2.0 * rows * 2 * s.ffn * s.hidden
+
+
+# --------------------------------------------------------------------------- #
+# clocks
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        busy = [s for s, p in zip(sm, power) if p > 250.0] or sm
+        return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- #
+# oracle legs (host cores)
+# --------------------------------------------------------------------------- #
+def _oracle_sample(batch, n_steps, seed=0):
+    """Times the oracle, as it stands, on `n_steps` decode steps of the workload (KV length PROMPT)."""
+    from oracle import oracle as O
+    cfg = O.Config(hidden=SHAPE.hidden, n_q_heads=SHAPE.n_q_heads, n_kv_heads=SHAPE.n_kv_heads,
+                   head_dim=SHAPE.head_dim, ffn=SHAPE.ffn)
+    w = synth.layer_weights(SHAPE, seed)
+    rng = np.random.default_rng(seed)
+    kc = rng.standard_normal((batch, SHAPE.n_kv_heads, PROMPT, SHAPE.head_dim)).astype(np.float16)
+    vc = rng.standard_normal((batch, SHAPE.n_kv_heads, PROMPT, SHAPE.head_dim)).astype(np.float16)
+    x = synth.hidden_states(SHAPE, seed, (batch, n_steps))
+    times = []
+    k, v = kc, vc
+    for i in range(n_steps):
+        t0 = time.perf_counter()
+        _, k, v = O.layer_decode(cfg, w, x[:, i], k, v, PROMPT + i)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info()]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    times = _oracle_sample(args.batch, args.warmup + args.steps)
+    timed = times[args.warmup:]
+    total = sum(timed)
+    value = args.batch * len(timed) / total
+    sample = f"{len(timed)} oracle decode steps of batch {args.batch} at KV length {PROMPT} (one step = {args.batch} tokens)"
+    line = {
+        "impl": "reference", "metric": "decode_tokens_per_s", "value": value, "unit": "tok/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(timed),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args.batch), "batch": args.batch, "prompt": PROMPT, "generate": GEN},
+        "cpu_baseline": {"value": value, "unit": "tok/s", "cores": host_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_name(batch):
+    return (f"Llama-7B-shaped single decoder layer (hidden 4096, 32x128 MHA, FFN 11008), FP16, batch {batch}, "
+            f"prompt {PROMPT}, {GEN} decode steps")
+
+
+# --------------------------------------------------------------------------- #
+# this library
+# --------------------------------------------------------------------------- #
+def run_ours(args):
+    import torch
+    from paper_2605_25655_b200 import thinfer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    B = args.batch
+    peaks, peak_kind = measured_peaks()
+
+    w_np = synth.layer_weights(SHAPE, seed=0)
+    layers = thinfer.to_device_layers([w_np], device=dev)
+    x_np = synth.hidden_states(SHAPE, 0, (B, PROMPT + GEN))
+    x_all = torch.from_numpy(x_np)
+    x_prompt = x_all[:, :PROMPT].contiguous().to(dev)
+    x_dec = [x_all[:, PROMPT + i].contiguous().to(dev) for i in range(GEN)]
+    ctx = thinfer.Context(SHAPE, layers, None, max_batch=B, max_seq=PROMPT + GEN, buf_slots=1, device=dev)
+    out_dec = torch.empty(B, SHAPE.hidden, dtype=torch.float16, device=dev)
+
+    def one_step(events=None):
+        if events:
+            events[0].record()
+        ctx.prefill(x_prompt)
+        if events:
+            events[1].record()
+        for i in range(GEN):
+            ctx.decode_step(x_dec[i], out=out_dec)
+        if events:
+            events[2].record()
+        ctx.release_slot(0)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    sync_all()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = ctx.launch_count()
+    sync_all()
+    wall0 = time.perf_counter()
+    for s in range(args.steps):
+        one_step(evs[s])
+    sync_all()
+    wall = time.perf_counter() - wall0
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if ctx.status() != 0:
+        raise SystemExit(f"device status {ctx.status()} after the timed region")
+    pre_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
+    dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+    tot_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
+    t = torch.tensor([pre_ms, dec_ms, tot_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    pre_ms, dec_ms, tot_ms = (float(v) for v in t.cpu())
+
+    # ---- end to end through the host-buffer entry points (pinned memory, copies inside the timed region)
+    h_prompt = x_all[:, :PROMPT].contiguous().pin_memory()
+    h_prompt_out = torch.empty_like(h_prompt).pin_memory()
+    h_dec = [x_all[:, PROMPT + i].contiguous().pin_memory() for i in range(GEN)]
+    h_dec_out = torch.empty(B, SHAPE.hidden, dtype=torch.float16).pin_memory()
+
+    def one_step_host():
+        ctx.prefill_host(h_prompt, h_prompt_out)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(GEN):
+            ctx.decode_step_host(h_dec[i], h_dec_out)
+            torch.cuda.synchronize()          # the caller reads each step's result before the next one
+        dt = time.perf_counter() - t0
+        ctx.release_slot(0)
+        return dt
+
+    one_step_host()
+    e2e_s = sum(one_step_host() for _ in range(max(1, min(args.steps, 3))))
+    e2e_steps = max(1, min(args.steps, 3))
+    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_s = float(te.cpu()[0])
+
+    # ---- dominant kernels, timed with CUDA events around each of their launches
+    def kernel_time(kid, fn):
+        ctx.profile_select(kid)
+        fn()
+        torch.cuda.synchronize()
+        n, ms = ctx.profile_read()
+        ctx.profile_select(-1)
+        return n, ms
+
+    def decode_only():
+        ctx.prefill(x_prompt)
+        for i in range(GEN):
+            ctx.decode_step(x_dec[i], out=out_dec)
+        ctx.release_slot(0)
+
+    n_gu, ms_gu = kernel_time(thinfer.K_GATEUP, decode_only)     # 1 prefill launch + GEN decode launches
+    ctx.profile_select(thinfer.K_GATEUP)
+    ctx.prefill(x_prompt)
+    torch.cuda.synchronize()
+    n_pre, ms_pre_gu = ctx.profile_read()
+    ctx.profile_select(-1)
+    ctx.release_slot(0)
+    ms_dec_gu = (ms_gu - ms_pre_gu) / max(1, n_gu - n_pre)
+    ms_pre_gu = ms_pre_gu / max(1, n_pre)
+
+    dec_tokens = world * B * GEN * args.steps
+    pre_tokens = world * B * PROMPT * args.steps
+    value = dec_tokens / (dec_ms * 1e-3)
+    dec_bytes = sum(decode_step_bytes(SHAPE, B, PROMPT + i + 1) for i in range(GEN))
+    dec_gbs = dec_bytes * args.steps / (dec_ms * 1e-3) / 1e9
+    gemm_fl, attn_fl = prefill_flops(SHAPE, B * PROMPT, PROMPT)
+    pre_tflops = (gemm_fl + attn_fl) * args.steps / (pre_ms * 1e-3) / 1e12
+    hbm_peak = float(peaks["hbm_gbs"])
+    tc_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    gu_gbs = gateup_gemv_bytes(SHAPE, B) / (ms_dec_gu * 1e-3) / 1e9
+    gu_tflops = gateup_gemm_flops(SHAPE, B * PROMPT) / (ms_pre_gu * 1e-3) / 1e12
+
+    line = {
+        "metric": "decode_tokens_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {"workload": workload_name(B), "batch": B, "prompt": PROMPT, "generate": GEN,
+                   "value_is": "batch x generate / decode-phase time; ms_per_step covers prefill + decode",
+                   "l2": "no flush: the 405 MB of layer weights streamed by every decode step and the prefill "
+                         "activations exceed the 126 MB L2",
+                   "multi_gpu": "independent replicas, no collective"},
+        "decode": {"ms_per_token_step": dec_ms / (args.steps * GEN), "achieved_GBs": dec_gbs,
+                   "frac_of_hbm_peak": dec_gbs / hbm_peak, "peak_GBs": hbm_peak, "peak_kind": peak_kind},
+        "prefill": {"value": pre_tokens / (pre_ms * 1e-3), "unit": "tok/s", "ms": pre_ms / args.steps,
+                    "achieved_TFLOPs": pre_tflops, "frac_of_tensor_peak": pre_tflops / tc_peak,
+                    "peak_TFLOPs": tc_peak, "peak_kind": peak_kind + " bf16 sustained (same tensor-pipe rate as fp16)"},
+        "roofline": {"kernel": "gemv_stream_kernel<SWIGLU> (decode gate/up projection)", "bound": "hbm",
+                     "achieved": gu_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gu_gbs / hbm_peak,
+                     "traffic": None, "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3,
+                     "algorithmic_bytes": gateup_gemv_bytes(SHAPE, B)},
+        "roofline_prefill": {"kernel": "tc_gemm_kernel<SWIGLU> (prefill gate/up projection)", "bound": "tensor",
+                             "achieved": gu_tflops, "peak": tc_peak, "unit": "TFLOP/s", "frac": gu_tflops / tc_peak,
+                             "traffic": None, "peak_kind": peak_kind, "avg_us": ms_pre_gu * 1e3},
+        "e2e": {"value": world * B * GEN * e2e_steps / e2e_s, "unit": "tok/s",
+                "h2d_bytes_per_step": B * SHAPE.hidden * 2, "d2h_bytes_per_step": B * SHAPE.hidden * 2,
+                "note": "per decode step: pinned host input -> device, layer, result -> host, stream synchronised"},
+        "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n = 4
+        times = _oracle_sample(B, n)
+        line["cpu_baseline"] = {"value": B * n / sum(times), "unit": "tok/s", "cores": host_threads(), "kind": "oracle",
+                                "sample": f"{n} oracle decode steps of batch {B} at KV length {PROMPT}"}
+    if rank == 0:
+        print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
