@@ -358,15 +358,43 @@ def run_ours(args):
     return 0
 
 
+def run_profile_case(args):
+    """A small, self-ending case for ncu: one warm-up pass, then one pass of the chosen phase."""
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    B, n_dec = args.batch, args.profile_decode_steps
+    w = thinfer.to_device_layers([synth.layer_weights(SHAPE, seed=0)])
+    x = torch.from_numpy(synth.hidden_states(SHAPE, 0, (B, PROMPT + n_dec)))
+    xp = x[:, :PROMPT].contiguous().cuda()
+    xd = [x[:, PROMPT + i].contiguous().cuda() for i in range(n_dec)]
+    ctx = thinfer.Context(SHAPE, w, None, max_batch=B, max_seq=PROMPT + n_dec)
+    for rep in range(2):
+        ctx.prefill(xp)
+        if args.profile == "decode" or rep == 0:
+            for t in xd:
+                ctx.decode_step(t)
+        ctx.release_slot(0)
+        torch.cuda.synchronize()
+    assert ctx.status() == 0
+    print(json.dumps({"profile_case": args.profile, "batch": B, "launches": ctx.launch_count()}))
+    ctx.close()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile", choices=["prefill", "decode"], default=None,
+                    help="run one small pass of a phase and exit (the case ncu captures)")
+    ap.add_argument("--profile-decode-steps", type=int, default=2)
     args = ap.parse_args()
+    if args.profile:
+        return run_profile_case(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

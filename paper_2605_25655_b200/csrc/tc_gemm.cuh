@@ -1,16 +1,28 @@
-// Tensor-core projection kernel for sm_100a (the large-M Linear of
-// Section 3.2.2, re-designed for Blackwell): TMA feeds a ring of 128-byte
-// swizzled shared-memory stages, one thread issues tcgen05.mma with the FP32
-// accumulator in tensor memory, four warps read the accumulator back with
+// Tensor-core projection kernel for sm_100a (the Linear operator of
+// Section 3.2.2 re-designed for Blackwell): TMA feeds a ring of 128-byte
+// swizzled shared-memory stages, one thread issues tcgen05.mma with FP32
+// accumulators in tensor memory, four warps read the accumulators back with
 // tcgen05.ld and apply the fused epilogue (Section 3.3.1).
 //
 // Orientation: the WEIGHT rows are the M = 128 side of the MMA and the tokens
-// are the N side (16 .. 256), so the same kernel covers prefill (N = 256) and
-// batched decode (N = 16).  Both operands are stored with the contraction
-// index contiguous, which is exactly the K-major layout TMA + tcgen05 want; no
-// copy or re-layout of the caller's weights is made.  An accumulator row (one
-// output feature) lives in one TMEM lane = one epilogue thread; its columns are
-// the tokens.
+// are the N side (16 .. 256), so one kernel covers prefill (N = 128 / 256) and
+// batched decode (N = 16 .. 64).  Both operands are stored with the contraction
+// index contiguous, which is the K-major layout TMA + tcgen05 want; the caller's
+// weights are never copied or re-laid out.  An accumulator row (one output
+// feature) lives in one TMEM lane = one epilogue thread; its columns are tokens.
+//
+// Persistent CTAs, one per SM.  Work is a list of segments (tile, k-block range):
+//   mode 0 (prefill)  whole tiles, round-robin over CTAs, grouped raster
+//   mode 1 (decode)   "stream-K": the (tile, k-block) space is cut into equal
+//                     contiguous ranges so that every SM streams the same
+//                     number of weight bytes whatever the shape (the paper's
+//                     small-M path splits only N; with 128-row tiles that
+//                     would leave most SMs idle).  A tile that spans several
+//                     CTAs is finished by the last CTA to arrive, which adds
+//                     the FP32 partials in a fixed order (deterministic).
+// Two accumulator buffers in tensor memory let the epilogue of segment j
+// overlap the MMAs of segment j+1.  The epilogue stages a chunk of the tile in
+// shared memory and writes it out with 16-byte, fully coalesced stores.
 //
 // Roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA
 // issuer, warps 2..5 = epilogue (warp w may touch TMEM lanes 32*(w%4)..+31).
@@ -21,17 +33,22 @@
 
 namespace thinfer {
 
-constexpr int kTcBM = 128;  // output features per CTA
+constexpr int kTcBM = 128;  // output features per tile
 constexpr int kTcBK = 64;   // contraction elements per stage (128 bytes)
 constexpr int kTcThreads = 192;
-constexpr int kTcGroup = 8;  // feature tiles per raster group (keeps a weight panel and the activations in L2)
+constexpr int kTcGroup = 8;          // feature tiles per raster group (keeps a weight panel and the activations in L2)
+constexpr int kTcStageOut = 16384;   // epilogue staging: 32 tokens x 128 features x 4 bytes
 
 struct TcGemmArgs {
   int n_feat[3];  // rows of each weight matrix (QKV: q, k, v; SWIGLU: ffn for gate and for up; else one)
   int tiles[3];   // 128-row tiles per matrix
   int rows;       // tokens
   int k;          // contraction length
-  int* status;    // device-visible status word
+  int mode;       // 0 = whole tiles round-robin, 1 = stream-K
+  int units_per_cta;  // stream-K: (tile, k-block) units per CTA
+  float* partial_ws;  // stream-K: [n_tiles + grid][NA*BN][128] FP32 partial accumulators
+  int* tile_counters; // stream-K: [n_tiles] arrival counters, zero between launches
+  int* status;        // device-visible status word
   EpiArgs e;
 };
 
@@ -40,52 +57,118 @@ __host__ __device__ constexpr int tc_stage_bytes(int bn, int epi) { return tc_nu
 __host__ __device__ constexpr int tc_stages(int bn, int epi) {
   return (200000 / tc_stage_bytes(bn, epi)) > 8 ? 8 : (200000 / tc_stage_bytes(bn, epi));
 }
+__host__ __device__ constexpr int tc_acc_cols(int bn, int epi) { return tc_num_a(epi) * bn; }
 __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {
-  int need = tc_num_a(epi) * bn, c = 32;
+  int need = 2 * tc_acc_cols(bn, epi), c = 32;
   while (c < need) c <<= 1;
   return c;
 }
 __host__ __device__ constexpr int tc_smem_bytes(int bn, int epi) {
-  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + kTcStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
 }
+__host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) { return epi == EPI_RESID || epi == EPI_PLAIN_F32; }
 
-// ---- epilogue for one chunk of CW token columns held by this thread (feature n) ----
-template <int EPI, int CW>
-__device__ __forceinline__ void tc_epilogue_chunk(const TcGemmArgs& a, const float (&acc)[CW], const float (&acc2)[CW],
-                                                  int n_cat, bool n_valid, int n_local, int tok_base) {
-  const EpiArgs& e = a.e;
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct TcSeg {
+  int tile, kb0, kb1;
+};
+
+// The j-th segment of this CTA; false when there is none.  Every role walks the same sequence.
+struct TcSegIter {
+  int mode, n_tiles, nkb, next_tile, stride;
+  long long u, u_end;
+  __device__ TcSegIter(const TcGemmArgs& a, int n_tiles_, int nkb_) {
+    mode = a.mode;
+    n_tiles = n_tiles_;
+    nkb = nkb_;
+    next_tile = blockIdx.x;
+    stride = gridDim.x;
+    const long long total = static_cast<long long>(n_tiles_) * nkb_;
+    u = static_cast<long long>(blockIdx.x) * a.units_per_cta;
+    u_end = u + a.units_per_cta;
+    if (u_end > total) u_end = total;
+  }
+  __device__ bool next(TcSeg& s) {
+    if (mode == 0) {
+      if (next_tile >= n_tiles) return false;
+      s.tile = next_tile;
+      s.kb0 = 0;
+      s.kb1 = nkb;
+      next_tile += stride;
+      return true;
+    }
+    if (u >= u_end) return false;
+    s.tile = static_cast<int>(u / nkb);
+    s.kb0 = static_cast<int>(u - static_cast<long long>(s.tile) * nkb);
+    const long long left = u_end - u;
+    s.kb1 = (nkb - s.kb0 < left) ? nkb : s.kb0 + static_cast<int>(left);
+    u += s.kb1 - s.kb0;
+    return true;
+  }
+};
+
+struct TcTile {
+  int mat, feat0, feat_off, tok0;
+};
+
+template <int BN, int EPI>
+__device__ __forceinline__ TcTile tc_tile_coords(const TcGemmArgs& a, int tile, int n_ft, int n_tt) {
+  const int per_group = kTcGroup * n_tt;
+  const int gid = tile / per_group;
+  const int first_ft = gid * kTcGroup;
+  const int gsz = min(kTcGroup, n_ft - first_ft);
+  const int in_group = tile - gid * per_group;
+  int ft = first_ft + in_group % gsz;
+  TcTile t;
+  t.tok0 = (in_group / gsz) * BN;
+  t.mat = 0;
+  t.feat_off = 0;
   if (EPI == EPI_QKV_ROPE) {
-    // per-thread constants: which buffer, which head, which element of the head
-    int kind = 0, nn = n_cat;
-    if (nn >= e.n_q) {
-      nn -= e.n_q;
-      kind = 1;
-      if (nn >= e.n_kv) {
-        nn -= e.n_kv;
-        kind = 2;
+    if (ft >= a.tiles[0]) {
+      ft -= a.tiles[0];
+      t.mat = 1;
+      t.feat_off = a.n_feat[0];
+      if (ft >= a.tiles[1]) {
+        ft -= a.tiles[1];
+        t.mat = 2;
+        t.feat_off += a.n_feat[1];
       }
     }
-    const int h = nn / e.head_dim, i = nn - h * e.head_dim;
+  }
+  t.feat0 = ft * kTcBM;
+  return t;
+}
+
+// ---- epilogue of one chunk of CW token columns --------------------------------------------
+// Phase A: thread `row` (one output feature) applies the element-wise part and writes its CW
+// values to the staging tile [token][feature].  Phase B: the 128 threads copy the staged tile
+// out in 16-byte pieces (8 features of one token), fully coalesced.
+template <int EPI, int CW>
+__device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile& t, uint8_t* stage, int row, int ethread,
+                                              const float (&v)[CW], const float (&v2)[CW], int tok_base) {
+  const EpiArgs& e = a.e;
+  constexpr bool F32 = tc_epi_fp32_stage(EPI);
+  __half* st16 = reinterpret_cast<__half*>(stage);
+  float* st32 = reinterpret_cast<float*>(stage);
+
+  // ---------------- phase A
+  if (EPI == EPI_QKV_ROPE) {
+    const int i = (t.feat0 + row) % e.head_dim;  // element inside its head (tiles are 128-aligned, heads 64 or 128)
     const int half = e.head_dim >> 1;
-    __half* dst = kind == 0 ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
+    const bool rotate = t.mat != 2;
     int b = tok_base / e.seq_len, s = tok_base - b * e.seq_len;
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-      float v = acc[c];
-      const float partner = __shfl_xor_sync(0xffffffffu, v, 1);  // the other element of the (2j, 2j+1) pair
-      const int r = tok_base + c;
-      if (n_valid && r < a.rows) {
+      float val = v[c];
+      const float partner = __shfl_xor_sync(0xffffffffu, val, 1);  // the other element of the (2j, 2j+1) pair
+      if (rotate && tok_base + c < a.rows) {
         const int pos = e.pos0 + s;
-        if (kind != 2) {
-          const float cs = __ldg(e.rope_cos + static_cast<size_t>(pos) * half + (i >> 1));
-          const float sn = __ldg(e.rope_sin + static_cast<size_t>(pos) * half + (i >> 1));
-          v = (i & 1) ? fmaf(partner, sn, v * cs) : fmaf(-partner, sn, v * cs);
-        }
-        const size_t off = kind == 0
-                               ? ((static_cast<size_t>(b) * e.n_q_heads + h) * e.seq_len + s) * e.head_dim + i
-                               : ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + pos) * e.head_dim + i;
-        dst[off] = __float2half_rn(v);
+        const float cs = __ldg(e.rope_cos + static_cast<size_t>(pos) * half + (i >> 1));
+        const float sn = __ldg(e.rope_sin + static_cast<size_t>(pos) * half + (i >> 1));
+        val = (i & 1) ? fmaf(partner, sn, val * cs) : fmaf(-partner, sn, val * cs);
       }
+      st16[c * kTcBM + row] = __float2half_rn(val);
       if (++s == e.seq_len) {
         s = 0;
         ++b;
@@ -94,21 +177,79 @@ __device__ __forceinline__ void tc_epilogue_chunk(const TcGemmArgs& a, const flo
   } else {
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-      const int r = tok_base + c;
-      if (n_valid && r < a.rows) {
-        const size_t off = static_cast<size_t>(r) * e.ld_out + n_local;
-        if (EPI == EPI_PLAIN_F16) {
-          reinterpret_cast<__half*>(e.out)[off] = __float2half_rn(acc[c]);
-        } else if (EPI == EPI_PLAIN_F32) {
-          reinterpret_cast<float*>(e.out)[off] = acc[c];
-        } else if (EPI == EPI_RESID) {
-          reinterpret_cast<__half*>(e.out)[off] = __float2half_rn(__half2float(e.resid[off]) + acc[c]);
-        } else {  // EPI_SWIGLU: acc = gate, acc2 = up
-          reinterpret_cast<__half*>(e.out)[off] = __float2half_rn(silu_f(acc[c]) * acc2[c]);
+      if (F32) st32[c * kTcBM + row] = v[c];
+      else if (EPI == EPI_SWIGLU) st16[c * kTcBM + row] = __float2half_rn(silu_f(v[c]) * v2[c]);
+      else st16[c * kTcBM + row] = __float2half_rn(v[c]);
+    }
+  }
+  epi_bar();
+
+  // ---------------- phase B
+  const int n_feat = a.n_feat[t.mat];
+#pragma unroll 1
+  for (int idx = ethread; idx < CW * 16; idx += 128) {
+    const int c = idx >> 4, piece = idx & 15;
+    const int r = tok_base + c;
+    const int n0 = t.feat0 + piece * 8;  // first feature of the piece inside its matrix
+    if (r >= a.rows || n0 >= n_feat) continue;
+    const int valid = min(8, n_feat - n0);
+    if (EPI == EPI_QKV_ROPE) {
+      const int b = r / e.seq_len, s = r - b * e.seq_len;
+      const int h = n0 / e.head_dim, i = n0 - h * e.head_dim;
+      __half* dst;
+      if (t.mat == 0) dst = e.q_out + ((static_cast<size_t>(b) * e.n_q_heads + h) * e.seq_len + s) * e.head_dim + i;
+      else dst = (t.mat == 1 ? e.k_cache : e.v_cache) +
+                 ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + e.pos0 + s) * e.head_dim + i;
+      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(st16 + c * kTcBM + piece * 8);
+    } else {
+      const size_t off = static_cast<size_t>(r) * e.ld_out + n0;
+      const bool vec = valid == 8 && (e.ld_out & 7) == 0;
+      if (EPI == EPI_PLAIN_F32) {
+        float* dst = reinterpret_cast<float*>(e.out) + off;
+        const float* src = st32 + c * kTcBM + piece * 8;
+        if (vec) {
+          reinterpret_cast<float4*>(dst)[0] = reinterpret_cast<const float4*>(src)[0];
+          reinterpret_cast<float4*>(dst)[1] = reinterpret_cast<const float4*>(src)[1];
+        } else {
+          for (int j = 0; j < valid; ++j) dst[j] = src[j];
+        }
+      } else if (EPI == EPI_RESID) {
+        __half* dst = reinterpret_cast<__half*>(e.out) + off;
+        const float* src = st32 + c * kTcBM + piece * 8;
+        if (vec) {
+          float x[8];
+          unpack8(ldg_cached(e.resid + off), x);
+          uint4 o;
+          o.x = pack2(x[0] + src[0], x[1] + src[1]);
+          o.y = pack2(x[2] + src[2], x[3] + src[3]);
+          o.z = pack2(x[4] + src[4], x[5] + src[5]);
+          o.w = pack2(x[6] + src[6], x[7] + src[7]);
+          *reinterpret_cast<uint4*>(dst) = o;
+        } else {
+          for (int j = 0; j < valid; ++j) dst[j] = __float2half_rn(__half2float(e.resid[off + j]) + src[j]);
+        }
+      } else {  // PLAIN_F16, SWIGLU
+        __half* dst = reinterpret_cast<__half*>(e.out) + off;
+        const __half* src = st16 + c * kTcBM + piece * 8;
+        if (vec) {
+          *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        } else {
+          for (int j = 0; j < valid; ++j) dst[j] = src[j];
         }
       }
     }
   }
+  epi_bar();
+}
+
+template <int CW>
+__device__ __forceinline__ void tc_load_acc(uint32_t taddr, float (&f)[CW]) {
+  uint32_t r[CW];
+  if constexpr (CW == 32) tmem_ld32(taddr, r);
+  else tmem_ld16(taddr, r);
+  tmem_ld_wait();
+#pragma unroll
+  for (int c = 0; c < CW; ++c) f[c] = __uint_as_float(r[c]);
 }
 
 template <int BN, int EPI>
@@ -120,44 +261,26 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   constexpr int STAGES = tc_stages(BN, EPI);
   constexpr int STAGE_BYTES = tc_stage_bytes(BN, EPI);
   constexpr int A_BYTES = kTcBM * 128;
+  constexpr int ACC_COLS = tc_acc_cols(BN, EPI);
   constexpr int TMEM_COLS = tc_tmem_cols(BN, EPI);
   constexpr int CW = BN >= 32 ? 32 : 16;
   constexpr uint32_t IDESC = idesc_f16(kTcBM, BN, 0, 0);
+  static_assert(2 * ACC_COLS <= 512, "two accumulator buffers must fit in tensor memory");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* stage_out = smem + STAGES * STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stage_out + kTcStageOut);
   uint64_t* empty_bar = full_bar + STAGES;
-  uint64_t* acc_bar = empty_bar + STAGES;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_bar + 1);
+  uint64_t* tfull_bar = empty_bar + STAGES;   // [2] accumulator ready for the epilogue
+  uint64_t* tempty_bar = tfull_bar + 2;       // [2] accumulator drained by the epilogue
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  int* flag = reinterpret_cast<int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  // ---- tile coordinates (grouped raster: kTcGroup feature tiles x all token tiles) ----
   const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
   const int n_tt = (a.rows + BN - 1) / BN;
-  const int per_group = kTcGroup * n_tt;
-  const int gid = blockIdx.x / per_group;
-  const int first_ft = gid * kTcGroup;
-  const int gsz = min(kTcGroup, n_ft - first_ft);
-  const int in_group = blockIdx.x - gid * per_group;
-  int ft = first_ft + in_group % gsz;
-  const int tt = in_group / gsz;
-  int mat = 0, feat_off = 0;
-  if (EPI == EPI_QKV_ROPE) {
-    if (ft >= a.tiles[0]) {
-      ft -= a.tiles[0];
-      mat = 1;
-      feat_off = a.n_feat[0];
-      if (ft >= a.tiles[1]) {
-        ft -= a.tiles[1];
-        mat = 2;
-        feat_off += a.n_feat[1];
-      }
-    }
-  }
-  const int feat0 = ft * kTcBM;  // first weight row of this tile inside its matrix
-  const int tok0 = tt * BN;
+  const int n_tiles = n_ft * n_tt;
   const int nkb = (a.k + kTcBK - 1) / kTcBK;
 
   if (threadIdx.x == 0) {
@@ -165,7 +288,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(acc_bar, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&tfull_bar[i], 1);
+      mbar_init(&tempty_bar[i], 4);  // one arrival per epilogue warp
+    }
     fence_barrier_init();
   }
   if (warp == 1) tmem_alloc(tmem_holder, TMEM_COLS);
@@ -175,69 +301,140 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
 
   if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (mat == 0 ? &tm_w0 : (mat == 1 ? &tm_w1 : &tm_w2)) : &tm_w0;
-      tma_prefetch_desc(tmw);
+      tma_prefetch_desc(&tm_w0);
       tma_prefetch_desc(&tm_x);
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1u, a.status)) break;
-        uint8_t* st = smem + s * STAGE_BYTES;
-        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-        tma_load_2d(st, tmw, &full_bar[s], kb * kTcBK, feat0);
-        if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[s], kb * kTcBK, feat0);
-        tma_load_2d(st + NA * A_BYTES, &tm_x, &full_bar[s], kb * kTcBK, tok0);
+      TcSegIter it(a, n_tiles, nkb);
+      TcSeg sg;
+      uint32_t n = 0;  // k-blocks issued so far (ring position)
+      bool ok = true;
+      while (ok && it.next(sg)) {
+        const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
+        const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (t.mat == 0 ? &tm_w0 : (t.mat == 1 ? &tm_w1 : &tm_w2)) : &tm_w0;
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
+          const int s = n % STAGES;
+          if (!mbar_wait(&empty_bar[s], ((n / STAGES) & 1) ^ 1u, a.status)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = smem + s * STAGE_BYTES;
+          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          tma_load_2d(st, tmw, &full_bar[s], kb * kTcBK, t.feat0);
+          if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[s], kb * kTcBK, t.feat0);
+          tma_load_2d(st + NA * A_BYTES, &tm_x, &full_bar[s], kb * kTcBK, t.tok0);
+        }
       }
     }
   } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&full_bar[s], ph, a.status)) break;
+      TcSegIter it(a, n_tiles, nkb);
+      TcSeg sg;
+      uint32_t n = 0, j = 0;
+      bool ok = true;
+      while (ok && it.next(sg)) {
+        const uint32_t buf = j & 1, use = j >> 1;
+        if (!mbar_wait(&tempty_bar[buf], (use & 1) ^ 1u, a.status)) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
-        const uint64_t da = smem_desc_sw128(sa, 16, 1024);
-        const uint64_t da2 = smem_desc_sw128(sa + A_BYTES, 16, 1024);
-        const uint64_t db = smem_desc_sw128(sa + NA * A_BYTES, 16, 1024);
+        const uint32_t acc = tmem_base + buf * ACC_COLS;
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
+          const int s = n % STAGES;
+          if (!mbar_wait(&full_bar[s], (n / STAGES) & 1, a.status)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+          const uint64_t da = smem_desc_sw128(sa, 16, 1024);
+          const uint64_t da2 = smem_desc_sw128(sa + A_BYTES, 16, 1024);
+          const uint64_t db = smem_desc_sw128(sa + NA * A_BYTES, 16, 1024);
 #pragma unroll
-        for (int k = 0; k < kTcBK / 16; ++k) {
-          const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-          tc_mma_f16(tmem_base, da + 2 * k, db + 2 * k, IDESC, accum);  // +32 bytes per K=16 step
-          if (NA == 2) tc_mma_f16(tmem_base + BN, da2 + 2 * k, db + 2 * k, IDESC, accum);
+          for (int k = 0; k < kTcBK / 16; ++k) {
+            const uint32_t accum = (kb != sg.kb0 || k != 0) ? 1u : 0u;
+            tc_mma_f16(acc, da + 2 * k, db + 2 * k, IDESC, accum);  // +32 bytes per K=16 step
+            if (NA == 2) tc_mma_f16(acc + BN, da2 + 2 * k, db + 2 * k, IDESC, accum);
+          }
+          tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
         }
-        tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+        if (ok) tc_commit(&tfull_bar[buf]);
+        ++j;
       }
-      tc_commit(acc_bar);
     }
   } else {
+    // ------------------------------------------------------------ epilogue
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;
-    const bool n_valid = feat0 + row < a.n_feat[mat];
-    const int n_local = feat0 + row;
-    const int n_cat = feat_off + n_local;
-    if (mbar_wait(acc_bar, 0, a.status)) {
+    const int ethread = (warp - 2) * 32 + lane;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    TcSegIter it(a, n_tiles, nkb);
+    TcSeg sg;
+    uint32_t j = 0;
+    while (it.next(sg)) {
+      const uint32_t buf = j & 1, use = j >> 1;
+      ++j;
+      if (!mbar_wait(&tfull_bar[buf], use & 1, a.status)) break;
       tc_fence_after();
+      const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
+      const uint32_t acc = lane_base + buf * ACC_COLS;
+      const bool whole = sg.kb0 == 0 && sg.kb1 == nkb;
+      if (whole) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += CW) {
-        uint32_t r1[CW], r2[CW];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + c0;
-        if constexpr (CW == 32) {
-          tmem_ld32(taddr, r1);
-          if (NA == 2) tmem_ld32(taddr + BN, r2);
-        } else {
-          tmem_ld16(taddr, r1);
-          if (NA == 2) tmem_ld16(taddr + BN, r2);
+        for (int c0 = 0; c0 < BN; c0 += CW) {
+          float v[CW], v2[CW];
+          tc_load_acc<CW>(acc + c0, v);
+          if (NA == 2) tc_load_acc<CW>(acc + BN + c0, v2);
+          if (c0 + CW >= BN) {  // accumulator fully read: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty_bar[buf]);
+          }
+          tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
         }
-        tmem_ld_wait();
-        float f1[CW], f2[CW];
+      } else {
+        // stream-K: park the partial accumulator; the last CTA of the tile reduces and finishes it
+        const long long first_unit = static_cast<long long>(sg.tile) * nkb;
+        const int first_cta = static_cast<int>(first_unit / a.units_per_cta);
+        const int last_cta = static_cast<int>((first_unit + nkb - 1) / a.units_per_cta);
+        const int n_seg = last_cta - first_cta + 1;
+        float* slot = a.partial_ws + static_cast<size_t>(sg.tile + blockIdx.x) * (ACC_COLS * kTcBM);
+#pragma unroll 1
+        for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
+          float v[CW];
+          tc_load_acc<CW>(acc + c0, v);
 #pragma unroll
-        for (int c = 0; c < CW; ++c) {
-          f1[c] = __uint_as_float(r1[c]);
-          f2[c] = NA == 2 ? __uint_as_float(r2[c]) : 0.f;
+          for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
         }
-        tc_epilogue_chunk<EPI, CW>(a, f1, f2, n_cat, n_valid, n_local, tok0 + c0);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[buf]);
+        __threadfence();
+        epi_bar();
+        if (ethread == 0) {
+          const int old = atomicAdd(a.tile_counters + sg.tile, 1);
+          *flag = (old == n_seg - 1) ? 1 : 0;
+        }
+        epi_bar();
+        const bool last = *reinterpret_cast<volatile int*>(flag) != 0;
+        if (last) {
+          __threadfence();
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += CW) {
+            float v[CW], v2[CW];
+#pragma unroll
+            for (int c = 0; c < CW; ++c) v[c] = v2[c] = 0.f;
+            for (int sgi = 0; sgi < n_seg; ++sgi) {  // fixed order: the result does not depend on arrival order
+              const float* src = a.partial_ws + static_cast<size_t>(sg.tile + first_cta + sgi) * (ACC_COLS * kTcBM);
+#pragma unroll
+              for (int c = 0; c < CW; ++c) {
+                v[c] += __ldcg(src + (c0 + c) * kTcBM + row);
+                if (NA == 2) v2[c] += __ldcg(src + (BN + c0 + c) * kTcBM + row);
+              }
+            }
+            tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
+          }
+          if (ethread == 0) a.tile_counters[sg.tile] = 0;  // ready for the next launch
+        }
       }
     }
   }

@@ -94,6 +94,8 @@ struct thinfer_ctx {
   float* logits = nullptr;
   int32_t* ids_out = nullptr;
   float *part_o = nullptr, *part_ml = nullptr;
+  float* splitk_ws = nullptr;   // stream-K partial accumulators
+  int* splitk_counters = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
   // status word (pinned, mapped)
@@ -143,10 +145,13 @@ int validate_config(const thinfer_config* c, std::string* why) {
 }
 
 struct ScratchPlan {
-  size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, stage_in, stage_out,
-      total;
-  int max_splits;
+  size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
+      splitk_counters, stage_in, stage_out, total;
+  int max_splits, max_tiles;
 };
+
+constexpr int kTcMaxCtas = 160;      // persistent grid bound (a B200 has 148 SMs)
+constexpr int kTcDecodeMaxBN = 64;   // token tile of the stream-K decode path
 
 ScratchPlan plan_scratch(const thinfer_config& c) {
   ScratchPlan p{};
@@ -173,6 +178,17 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
   p.ids_out = take(static_cast<size_t>(c.max_batch) * 4);
   p.part_o = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * p.max_splits * c.head_dim * 4);
   p.part_ml = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * p.max_splits * 2 * 4);
+  {
+    auto t128 = [](size_t n) { return (n + 127) / 128; };
+    size_t tiles = t128(qd) + 2 * t128(static_cast<size_t>(c.n_kv_heads) * c.head_dim);
+    if (t128(c.ffn) > tiles) tiles = t128(c.ffn);
+    if (t128(c.hidden) > tiles) tiles = t128(c.hidden);
+    if (c.vocab > 0 && t128(c.vocab) > tiles) tiles = t128(c.vocab);
+    p.max_tiles = static_cast<int>(tiles);
+    // one slot per (tile, CTA) pair that can occur: tiles + CTAs; a slot holds 128 rows x (2 x 64) FP32 columns
+    p.splitk_ws = take((tiles + kTcMaxCtas) * static_cast<size_t>(2 * kTcDecodeMaxBN) * 128 * 4);
+    p.splitk_counters = take(tiles * 4);
+  }
   const size_t in_bytes = c.vocab > 0 ? M * 4 : M * c.hidden * 2;
   const size_t out_bytes = c.vocab > 0 ? static_cast<size_t>(c.max_batch) * (4 + static_cast<size_t>(c.vocab) * 4)
                                        : M * c.hidden * 2;
@@ -252,14 +268,24 @@ void launch_tc(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   }
   const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
   const int n_tt = (a.rows + BN - 1) / BN;
-  L.go(kid, tc_gemm_kernel<BN, EPI>, dim3(n_ft * n_tt), dim3(kTcThreads), smem, w0, w1, w2, x, a);
+  const int n_tiles = n_ft * n_tt;
+  int sms = L.c ? L.c->sm_count : 148;
+  if (sms > kTcMaxCtas) sms = kTcMaxCtas;
+  TcGemmArgs b = a;
+  int grid = n_tiles < sms ? n_tiles : sms;
+  if (b.mode == 1) {
+    const long long units = static_cast<long long>(n_tiles) * ((a.k + kTcBK - 1) / kTcBK);
+    grid = units < sms ? static_cast<int>(units) : sms;
+    b.units_per_cta = static_cast<int>((units + grid - 1) / grid);
+  }
+  L.go(kid, tc_gemm_kernel<BN, EPI>, dim3(grid), dim3(kTcThreads), smem, w0, w1, w2, x, b);
 }
 
-int pick_bn(int rows) {
+int pick_bn(int rows, int epi) {
   if (rows <= 16) return 16;
   if (rows <= 32) return 32;
   if (rows <= 64) return 64;
-  if (rows <= 128) return 128;
+  if (rows <= 128 || epi == EPI_SWIGLU) return 128;  // gate + up need two accumulators per buffer
   return 256;
 }
 
@@ -271,16 +297,18 @@ void launch_tc_bn(Launcher& L, int kid, int bn, const CUtensorMap& w0, const CUt
     case 32: launch_tc<32, EPI>(L, kid, w0, w1, w2, x, a); break;
     case 64: launch_tc<64, EPI>(L, kid, w0, w1, w2, x, a); break;
     case 128: launch_tc<128, EPI>(L, kid, w0, w1, w2, x, a); break;
-    default: launch_tc<256, EPI>(L, kid, w0, w1, w2, x, a); break;
+    default:
+      if constexpr (EPI != EPI_SWIGLU) launch_tc<256, EPI>(L, kid, w0, w1, w2, x, a);
+      break;
   }
 }
 
 // x: activations [rows][k]; the token-side tensor map is encoded per call (host only, no device work)
 template <int EPI>
 void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
-               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e) {
+               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e, bool stream_k = false) {
   if (L.rc != THINFER_OK) return;
-  const int bn = pick_bn(rows);
+  const int bn = pick_bn(rows, EPI);
   CUtensorMap mx;
   if (!make_map_2d(&mx, x, k, rows, bn)) {
     L.rc = fail(L.c, THINFER_ECUDA, "cuTensorMapEncodeTiled failed for an activation operand");
@@ -296,6 +324,11 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   a.k = k;
   a.status = L.c ? L.c->status_dev : nullptr;
   a.e = e;
+  if (stream_k && L.c != nullptr && rows <= kTcDecodeMaxBN) {
+    a.mode = 1;
+    a.partial_ws = L.c->splitk_ws;
+    a.tile_counters = L.c->splitk_counters;
+  }
   launch_tc_bn<EPI>(L, kid, bn, w0, w1, w2, mx, a);
 }
 
@@ -511,6 +544,43 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
   __half* kc = kv_ptr(c, slot, layer, 0);
   __half* vc = kv_ptr(c, slot, layer, 1);
   auto H = [](const void* p) { return static_cast<const __half*>(p); };
+  if (batch >= 2) {
+    // batched decode: the weight stream feeds the tensor cores (stream-K over all SMs); plain FMA
+    // cannot keep up with HBM beyond a couple of tokens per weight
+    const LayerMaps& m = c->maps[layer];
+    rmsnorm_rows(L, x_in, H(w.attn_norm), c->h, batch, cf.hidden, cf.rms_eps);
+    {
+      const int nf[3] = {qd, kvd, kvd};
+      tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, batch, cf.hidden, nf, qkv_epi(c, kc, vc, 1, pos),
+                              true);
+    }
+    attn_decode(L, c, c->qbuf, kc, vc, c->attn, batch, pos + 1);
+    {
+      EpiArgs e{};
+      e.out = c->x1;
+      e.resid = x_in;
+      e.ld_out = cf.hidden;
+      const int nf[3] = {cf.hidden, 0, 0};
+      tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->attn, batch, qd, nf, e, true);
+    }
+    rmsnorm_rows(L, c->x1, H(w.ffn_norm), c->h, batch, cf.hidden, cf.rms_eps);
+    {
+      EpiArgs e{};
+      e.out = c->act;
+      e.ld_out = cf.ffn;
+      const int nf[3] = {cf.ffn, cf.ffn, 0};
+      tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->h, batch, cf.hidden, nf, e, true);
+    }
+    {
+      EpiArgs e{};
+      e.out = x_out;
+      e.resid = c->x1;
+      e.ld_out = cf.hidden;
+      const int nf[3] = {cf.hidden, 0, 0};
+      tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->act, batch, cf.ffn, nf, e, true);
+    }
+    return;
+  }
   {
     const int n[3] = {qd, kvd, kvd};
     gemv<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch,
@@ -552,8 +622,13 @@ void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, in
   e.out = lg;
   e.ld_out = cf.vocab;
   const int n[3] = {cf.vocab, 0, 0};
-  gemv<EPI_PLAIN_F32, true>(L, THINFER_K_HEAD, c->lm_head, nullptr, nullptr, n, cf.hidden, x, cf.hidden, batch,
-                            c->final_norm, cf.rms_eps, e);
+  if (batch >= 2) {
+    rmsnorm_rows(L, x, c->final_norm, c->h, batch, cf.hidden, cf.rms_eps);
+    tc_linear<EPI_PLAIN_F32>(L, THINFER_K_HEAD, c->map_head, c->map_head, c->map_head, c->h, batch, cf.hidden, n, e, true);
+  } else {
+    gemv<EPI_PLAIN_F32, true>(L, THINFER_K_HEAD, c->lm_head, nullptr, nullptr, n, cf.hidden, x, cf.hidden, batch,
+                              c->final_norm, cf.rms_eps, e);
+  }
   if (ids_out != nullptr)
     L.go(THINFER_K_ARGMAX, argmax_rows_kernel, dim3(batch), dim3(1024), 0, static_cast<const float*>(lg), ids_out,
          cf.vocab);
@@ -717,6 +792,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->ids_out = reinterpret_cast<int32_t*>(s + p.ids_out);
   c->part_o = reinterpret_cast<float*>(s + p.part_o);
   c->part_ml = reinterpret_cast<float*>(s + p.part_ml);
+  c->splitk_ws = reinterpret_cast<float*>(s + p.splitk_ws);
+  c->splitk_counters = reinterpret_cast<int*>(s + p.splitk_counters);
   c->stage_in = s + p.stage_in;
   c->stage_out = s + p.stage_out;
   c->max_splits = p.max_splits;
@@ -754,6 +831,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   const int n_tab = cfg->max_seq * (cfg->head_dim / 2);
   rope_table_kernel<<<(n_tab + 255) / 256, 256>>>(c->rope_cos, c->rope_sin, cfg->max_seq, cfg->head_dim / 2,
                                                   static_cast<double>(cfg->rope_base));
+  if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 4, 0) != cudaSuccess)
+    return cleanup(THINFER_ECUDA);
   if (cudaDeviceSynchronize() != cudaSuccess) return cleanup(THINFER_ECUDA);
   *out = c;
   return THINFER_OK;
