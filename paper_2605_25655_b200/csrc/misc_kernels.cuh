@@ -38,6 +38,59 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __half* __restr
   }
 }
 
+// The same operator for few rows (decode): one CTA per row, the row is read once into registers.
+// n <= 8 * 256 * kRmsSmallChunks.
+constexpr int kRmsSmallChunks = 8;
+__global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const __half* __restrict__ x,
+                                                               const __half* __restrict__ gain, __half* __restrict__ y,
+                                                               int n, float eps) {
+  __shared__ float red[8];
+  const __half* xr = x + static_cast<size_t>(blockIdx.x) * n;
+  __half* yr = y + static_cast<size_t>(blockIdx.x) * n;
+  const int chunks = n >> 3;
+  uint4 xv[kRmsSmallChunks], gv[kRmsSmallChunks];
+#pragma unroll
+  for (int j = 0; j < kRmsSmallChunks; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < chunks) {
+      xv[j] = ldg_cached(xr + (c << 3));
+      gv[j] = ldg_cached(gain + (c << 3));
+    }
+  }
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < kRmsSmallChunks; ++j) {
+    if (threadIdx.x + j * 256 < chunks) {
+      float f[8];
+      unpack8(xv[j], f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+    }
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float rstd = rsqrtf(tot / static_cast<float>(n) + eps);
+#pragma unroll
+  for (int j = 0; j < kRmsSmallChunks; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < chunks) {
+      float f[8], g[8];
+      unpack8(xv[j], f);
+      unpack8(gv[j], g);
+      uint4 o;
+      o.x = pack2(f[0] * rstd * g[0], f[1] * rstd * g[1]);
+      o.y = pack2(f[2] * rstd * g[2], f[3] * rstd * g[3]);
+      o.z = pack2(f[4] * rstd * g[4], f[5] * rstd * g[5]);
+      o.w = pack2(f[6] * rstd * g[6], f[7] * rstd * g[7]);
+      *reinterpret_cast<uint4*>(yr + (c << 3)) = o;
+    }
+  }
+}
+
 // dst[r][:] = table[ids[r]][:]  (embedding).  One warp per row.
 __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __restrict__ ids,
                                                            const __half* __restrict__ table, __half* __restrict__ dst,

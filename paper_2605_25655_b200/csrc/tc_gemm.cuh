@@ -157,22 +157,28 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
     const int i = (t.feat0 + row) % e.head_dim;  // element inside its head (tiles are 128-aligned, heads 64 or 128)
     const int half = e.head_dim >> 1;
     const bool rotate = t.mat != 2;
-    int b = tok_base / e.seq_len, s = tok_base - b * e.seq_len;
+    // all table reads of the chunk are issued before any is used: one L2 latency per chunk, not per column
+    float cs[CW], sn[CW];
+    {
+      int b = tok_base / e.seq_len, s = tok_base - b * e.seq_len;
+#pragma unroll
+      for (int c = 0; c < CW; ++c) {
+        cs[c] = 1.f;
+        sn[c] = 0.f;
+        if (rotate && tok_base + c < a.rows) {
+          const size_t o = static_cast<size_t>(e.pos0 + s) * half + (i >> 1);
+          cs[c] = __ldg(e.rope_cos + o);
+          sn[c] = __ldg(e.rope_sin + o);
+        }
+        if (++s == e.seq_len) s = 0;
+      }
+    }
+    const float sgn = (i & 1) ? 1.f : -1.f;
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-      float val = v[c];
+      const float val = v[c];
       const float partner = __shfl_xor_sync(0xffffffffu, val, 1);  // the other element of the (2j, 2j+1) pair
-      if (rotate && tok_base + c < a.rows) {
-        const int pos = e.pos0 + s;
-        const float cs = __ldg(e.rope_cos + static_cast<size_t>(pos) * half + (i >> 1));
-        const float sn = __ldg(e.rope_sin + static_cast<size_t>(pos) * half + (i >> 1));
-        val = (i & 1) ? fmaf(partner, sn, val * cs) : fmaf(-partner, sn, val * cs);
-      }
-      st16[c * kTcBM + row] = __float2half_rn(val);
-      if (++s == e.seq_len) {
-        s = 0;
-        ++b;
-      }
+      st16[c * kTcBM + row] = __float2half_rn(fmaf(sgn * partner, sn[c], val * cs[c]));
     }
   } else {
 #pragma unroll
@@ -186,7 +192,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
 
   // ---------------- phase B
   const int n_feat = a.n_feat[t.mat];
-#pragma unroll 1
+#pragma unroll
   for (int idx = ethread; idx < CW * 16; idx += 128) {
     const int c = idx >> 4, piece = idx & 15;
     const int r = tok_base + c;

@@ -463,6 +463,10 @@ void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v
 }
 
 void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int rows, int n, float eps) {
+  if (rows <= 256 && n <= 8 * 256 * kRmsSmallChunks) {
+    L.go(THINFER_K_RMSNORM, rmsnorm_few_rows_kernel, dim3(rows), dim3(256), 0, x, g, y, n, eps);
+    return;
+  }
   L.go(THINFER_K_RMSNORM, rmsnorm_rows_kernel, dim3((rows + 7) / 8), dim3(256), 0, x, g, y, rows, n, eps);
 }
 
