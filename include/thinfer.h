@@ -186,6 +186,30 @@ void thinfer_destroy(thinfer_ctx* ctx);
 int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k,
                       int32_t out_fp32, int32_t path, void* cuda_stream);
 
+/* The same product for callers that must not allocate (the paper has no
+ * counterpart: this entry point exists for the integration, not the method).
+ * Some hosts of this library cannot call cudaMalloc at the point where they
+ * need a projection: code running while a CUDA graph is being captured on
+ * another stream of the process, real-time loops that forbid calls which may
+ * synchronise the device, and allocators that hand a fixed arena to each
+ * plug-in.  For them the split-K partial sums and arrival counters of the
+ * stream-K kernel live in a fixed array inside the library image instead of a
+ * caller workspace; nothing is allocated or freed, by this call or by anything
+ * it uses.
+ *   Limits: rows <= 16, n_out <= 16384, k % 8 == 0, n_out even.  Larger sizes
+ *   return THINFER_ECAPACITY (text in thinfer_last_error(NULL)).  The array is
+ *   about 2.3 MB and stays resident on every GPU that loads the library until
+ *   the process exits.
+ *   The first call on a device resolves the array's device address (with that
+ *   device current) and should therefore come before any stream capture; later
+ *   calls only enqueue a 1 KB clear of the counters and the kernel.
+ *   All calls on a device share the array: calls whose kernels may overlap on
+ *   the GPU (different streams without ordering) race on it.  Keep them on one
+ *   stream or order them with events.
+ * x, w, y: device pointers as for thinfer_op_linear (tensor-core path). */
+int thinfer_op_linear_noalloc(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k,
+                              int32_t out_fp32, void* cuda_stream);
+
 /* Causal attention of Eq. 6 for a batch: q FP16 [batch, n_q_heads, seq, head_dim],
  * k, v FP16 [batch, n_kv_heads, kv_stride, head_dim] (first seq positions used),
  * out FP16 [batch, seq, n_q_heads*head_dim]. */

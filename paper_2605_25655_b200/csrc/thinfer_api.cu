@@ -1024,6 +1024,70 @@ int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32
   return L.rc;
 }
 
+// ---------------------------------------------------------------------------
+// Allocation-free linear.  The stream-K scratch (arrival counters, then one FP32
+// partial-accumulator slot per (tile, CTA) pair) is a fixed array in the library
+// image.  In host code the array's name is only a handle: the kernel needs the
+// device address, which cudaGetSymbolAddress returns for the current device.
+// ---------------------------------------------------------------------------
+namespace {
+constexpr int kNoAllocMaxRows = 16;
+constexpr int kNoAllocMaxNOut = 16384;
+constexpr size_t kNoAllocCounterBytes = 1024;             // 128 tiles x 4 bytes, rounded up
+constexpr size_t kNoAllocSlotBytes = 16 * kTcBM * 4;      // 16 token columns x 128 features, FP32
+constexpr size_t kNoAllocBytes = kNoAllocCounterBytes + (kNoAllocMaxNOut / kTcBM + kTcMaxCtas) * kNoAllocSlotBytes;
+constexpr int kNoAllocMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {};
+}  // namespace
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+int thinfer_op_linear_noalloc(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k,
+                              int32_t out_fp32, void* cuda_stream) {
+  if (x == nullptr || w == nullptr || y == nullptr || rows <= 0 || n_out <= 0 || k <= 0) return THINFER_EINVAL;
+  if (k % 8 != 0 || n_out % 2 != 0) return THINFER_EUNSUPPORTED;
+  if (rows > kNoAllocMaxRows || n_out > kNoAllocMaxNOut) {
+    g_global_err = "thinfer_op_linear_noalloc: rows <= 16 and n_out <= 16384 is the limit of the built-in scratch";
+    return THINFER_ECAPACITY;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) return THINFER_ECUDA;
+  unsigned char* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[dev] == nullptr) {  // set-up, once per device, with that device current
+      void* p = nullptr;
+      const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+      if (e != cudaSuccess || p == nullptr) {
+        g_global_err = std::string("cudaGetSymbolAddress failed: ") + cudaGetErrorString(e);
+        return THINFER_ECUDA;
+      }
+      g_noalloc_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // the counters must start at zero whatever an earlier (possibly failed) call left behind
+  if (cudaMemsetAsync(scratch, 0, kNoAllocCounterBytes, st) != cudaSuccess) return THINFER_ECUDA;
+  CUtensorMap mw, mx;
+  if (!make_map_2d(&mw, w, k, n_out, 128) || !make_map_2d(&mx, x, k, rows, 16)) return THINFER_ECUDA;
+  Launcher L{nullptr, st};
+  TcGemmArgs a{};
+  a.n_feat[0] = n_out;
+  a.tiles[0] = (n_out + kTcBM - 1) / kTcBM;
+  a.rows = rows;
+  a.k = k;
+  a.mode = 1;
+  a.tile_counters = reinterpret_cast<int*>(scratch);
+  a.partial_ws = reinterpret_cast<float*>(scratch + kNoAllocCounterBytes);
+  a.status = nullptr;
+  a.e.out = y;
+  a.e.ld_out = n_out;
+  if (out_fp32) launch_tc<16, EPI_PLAIN_F32>(L, -2, mw, mw, mw, mx, a);
+  else launch_tc<16, EPI_PLAIN_F16>(L, -2, mw, mw, mw, mx, a);
+  return L.rc;
+}
+
 int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, void* out, int32_t batch,
                                  int32_t n_q_heads, int32_t n_kv_heads, int32_t seq, int32_t kv_stride,
                                  int32_t head_dim, void* cuda_stream) {

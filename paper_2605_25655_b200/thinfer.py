@@ -23,7 +23,7 @@ EXPORTS = (
     "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
     "thinfer_kv_pointer", "thinfer_status", "thinfer_set_launch_mode", "thinfer_profile_select",
     "thinfer_profile_read", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
-    "thinfer_op_linear", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
+    "thinfer_op_linear", "thinfer_op_linear_noalloc", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
 )
 
 
@@ -83,6 +83,7 @@ def lib():
     L.thinfer_destroy.argtypes = [vp]
     L.thinfer_destroy.restype = None
     L.thinfer_op_linear.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+    L.thinfer_op_linear_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     L.thinfer_op_attention_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
     L.thinfer_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, C.c_float, vp]
     _lib = L
@@ -247,6 +248,19 @@ def op_linear(x, w, out_fp32=False, path=0, stream=None):
     y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else torch.float16, device=x.device)
     _check(lib().thinfer_op_linear(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k, int(out_fp32), path,
                                    _stream_ptr(stream)))
+    return y
+
+
+def op_linear_noalloc(x, w, y, stream=None):
+    """y[rows, n_out] = x w^T through the entry point that allocates nothing: the caller passes
+    the output (FP16 or FP32 tensor); the split-K scratch is a fixed array inside the library.
+    For hosts that cannot call cudaMalloc where they need the product.  rows <= 16, n_out <= 16384."""
+    import torch
+    rows, k = x.shape
+    n_out = w.shape[0]
+    assert y.shape == (rows, n_out) and y.is_contiguous()
+    _check(lib().thinfer_op_linear_noalloc(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k,
+                                           int(y.dtype == torch.float32), _stream_ptr(stream)))
     return y
 
 
