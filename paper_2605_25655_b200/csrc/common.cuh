@@ -60,6 +60,15 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 
+// ------------------------------------------------ programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while its
+// predecessor in the stream is still running.  pdl_wait() blocks until the predecessor has
+// completed and its memory is visible (a no-op for an ordinary launch); everything a kernel
+// does before it must touch only data no earlier kernel of the step writes (weights, its own
+// shared / tensor memory).  pdl_launch_dependents() lets the successor be scheduled early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // --------------------------------------------------------------- mbarrier
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));

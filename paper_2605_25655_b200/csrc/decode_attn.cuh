@@ -30,6 +30,8 @@ struct AttnDecArgs {
 
 template <int D, int G>
 __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const AttnDecArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int LPK = D / 8;     // lanes that cover one key row
   constexpr int KPL = 32 / LPK;  // keys per warp-wide load
   constexpr int UN = kAttnDecUnroll;
@@ -177,6 +179,8 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
 // Merges the split-KV partials: out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
 template <int D>
 __global__ void __launch_bounds__(D) attn_decode_combine_kernel(const AttnDecArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t bh = blockIdx.x;  // (request, query head)
   const int i = threadIdx.x;
   float mx = -INFINITY;

@@ -32,6 +32,8 @@ struct GemvArgs {
 
 template <int NB, int EPI, bool NORM>
 __global__ void __launch_bounds__(kGemvWarps * 32) gemv_stream_kernel(const GemvArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float red[kGemvWarps][3 * NB];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ks = warp % a.kslices;

@@ -10,6 +10,8 @@ namespace thinfer {
 // One warp per row, 128-bit accesses; n is a multiple of 8.
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __half* __restrict__ x, const __half* __restrict__ gain,
                                                            __half* __restrict__ y, int rows, int n, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -44,6 +46,8 @@ constexpr int kRmsSmallChunks = 8;
 __global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const __half* __restrict__ x,
                                                                const __half* __restrict__ gain, __half* __restrict__ y,
                                                                int n, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float red[8];
   const __half* xr = x + static_cast<size_t>(blockIdx.x) * n;
   __half* yr = y + static_cast<size_t>(blockIdx.x) * n;
@@ -95,6 +99,8 @@ __global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const __half* __r
 __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __restrict__ ids,
                                                            const __half* __restrict__ table, __half* __restrict__ dst,
                                                            int rows, int n, int vocab) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -108,6 +114,8 @@ __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __rest
 // dst[b][:] = src[b][seq_len-1][:]  (the last prompt position feeds the LM head).
 __global__ void __launch_bounds__(256) gather_last_rows_kernel(const __half* __restrict__ src, __half* __restrict__ dst,
                                                                int batch, int seq_len, int n) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= batch) return;
@@ -119,6 +127,8 @@ __global__ void __launch_bounds__(256) gather_last_rows_kernel(const __half* __r
 // ids[r] = argmax_n logits[r][n], exact ties to the lowest index.  One CTA per row.
 __global__ void __launch_bounds__(1024) argmax_rows_kernel(const float* __restrict__ logits, int32_t* __restrict__ ids,
                                                            int n) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float sv[32];
   __shared__ int si[32];
   const float* row = logits + static_cast<size_t>(blockIdx.x) * n;

@@ -39,6 +39,8 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
     attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                         const __grid_constant__ CUtensorMap tm_v, const AttnPreArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int SUB = D / 64;            // 64-wide column blocks of a head
   constexpr int TILE_BYTES = SUB * 16384;
   constexpr int TMEM_COLS = 256;

@@ -37,7 +37,6 @@ constexpr int kTcBM = 128;  // output features per tile
 constexpr int kTcBK = 64;   // contraction elements per stage (128 bytes)
 constexpr int kTcThreads = 192;
 constexpr int kTcGroup = 8;          // feature tiles per raster group (keeps a weight panel and the activations in L2)
-constexpr int kTcStageOut = 16384;   // epilogue staging: 32 tokens x 128 features x 4 bytes
 
 struct TcGemmArgs {
   int n_feat[3];  // rows of each weight matrix (QKV: q, k, v; SWIGLU: ffn for gate and for up; else one)
@@ -54,8 +53,15 @@ struct TcGemmArgs {
 
 __host__ __device__ constexpr int tc_num_a(int epi) { return epi == EPI_SWIGLU ? 2 : 1; }
 __host__ __device__ constexpr int tc_stage_bytes(int bn, int epi) { return tc_num_a(epi) * kTcBM * 128 + bn * 128; }
+// epilogue staging: CW tokens x 128 features x 4 bytes
+__host__ __device__ constexpr int tc_stage_out_bytes(int bn) { return (bn >= 32 ? 32 : 16) * kTcBM * 4; }
+// Token tiles up to 64 are the decode kernels: they are sized so that two CTAs fit on one SM, which
+// lets the next kernel of the step become resident and prefetch its weights while this one finishes.
+__host__ __device__ constexpr int tc_ring_budget(int bn) {
+  return bn <= 64 ? (233472 / 2 - 1024) - tc_stage_out_bytes(bn) - 1280 : 200000;
+}
 __host__ __device__ constexpr int tc_stages(int bn, int epi) {
-  return (200000 / tc_stage_bytes(bn, epi)) > 8 ? 8 : (200000 / tc_stage_bytes(bn, epi));
+  return (tc_ring_budget(bn) / tc_stage_bytes(bn, epi)) > 8 ? 8 : (tc_ring_budget(bn) / tc_stage_bytes(bn, epi));
 }
 __host__ __device__ constexpr int tc_acc_cols(int bn, int epi) { return tc_num_a(epi) * bn; }
 __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {
@@ -64,7 +70,7 @@ __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {
   return c;
 }
 __host__ __device__ constexpr int tc_smem_bytes(int bn, int epi) {
-  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + kTcStageOut + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + tc_stage_out_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 }
 __host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) { return epi == EPI_RESID || epi == EPI_PLAIN_F32; }
 
@@ -276,7 +282,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_out = smem + STAGES * STAGE_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stage_out + kTcStageOut);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stage_out + tc_stage_out_bytes(BN));
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tfull_bar = empty_bar + STAGES;   // [2] accumulator ready for the epilogue
   uint64_t* tempty_bar = tfull_bar + 2;       // [2] accumulator drained by the epilogue
@@ -305,12 +311,32 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_w0);
       tma_prefetch_desc(&tm_x);
+      // Weights do not depend on the previous kernel of the step: in decode the first ring-full of
+      // weight tiles is requested before the dependency wait, the token tiles follow after it.
+      const uint32_t pre = a.mode == 1 ? STAGES : 0;
+      {
+        TcSegIter it(a, n_tiles, nkb);
+        TcSeg sg;
+        uint32_t n = 0;
+        while (n < pre && it.next(sg)) {
+          const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
+          const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (t.mat == 0 ? &tm_w0 : (t.mat == 1 ? &tm_w1 : &tm_w2)) : &tm_w0;
+          for (int kb = sg.kb0; kb < sg.kb1 && n < pre; ++kb, ++n) {
+            uint8_t* st = smem + n * STAGE_BYTES;
+            mbar_expect_tx(&full_bar[n], STAGE_BYTES);
+            tma_load_2d(st, tmw, &full_bar[n], kb * kTcBK, t.feat0);
+            if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[n], kb * kTcBK, t.feat0);
+          }
+        }
+      }
+      pdl_wait();
       TcSegIter it(a, n_tiles, nkb);
       TcSeg sg;
       uint32_t n = 0;  // k-blocks issued so far (ring position)
@@ -320,14 +346,16 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (t.mat == 0 ? &tm_w0 : (t.mat == 1 ? &tm_w1 : &tm_w2)) : &tm_w0;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
           const int s = n % STAGES;
-          if (!mbar_wait(&empty_bar[s], ((n / STAGES) & 1) ^ 1u, a.status)) {
-            ok = false;
-            break;
-          }
           uint8_t* st = smem + s * STAGE_BYTES;
-          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-          tma_load_2d(st, tmw, &full_bar[s], kb * kTcBK, t.feat0);
-          if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[s], kb * kTcBK, t.feat0);
+          if (n >= pre) {
+            if (!mbar_wait(&empty_bar[s], ((n / STAGES) & 1) ^ 1u, a.status)) {
+              ok = false;
+              break;
+            }
+            mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+            tma_load_2d(st, tmw, &full_bar[s], kb * kTcBK, t.feat0);
+            if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[s], kb * kTcBK, t.feat0);
+          }
           tma_load_2d(st + NA * A_BYTES, &tm_x, &full_bar[s], kb * kTcBK, t.tok0);
         }
       }
@@ -373,6 +401,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const int row = q * 32 + lane;
     const int ethread = (warp - 2) * 32 + lane;
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    pdl_wait();  // residual stream, RoPE positions, stream-K scratch: all written by earlier kernels
     TcSegIter it(a, n_tiles, nkb);
     TcSeg sg;
     uint32_t j = 0;

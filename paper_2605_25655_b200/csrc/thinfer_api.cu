@@ -101,7 +101,7 @@ struct thinfer_ctx {
   // status word (pinned, mapped)
   int* status_host = nullptr;
   int* status_dev = nullptr;
-  int launch_mode = 0;
+  int launch_mode = 1;
   int64_t launches = 0;
   int prof_kernel = -1;
   std::vector<ProfEvent> prof_events;
@@ -235,6 +235,11 @@ struct Launcher {
     cudaLaunchAttribute attr[1];
     lc.attrs = attr;
     lc.numAttrs = 0;
+    if (c != nullptr && c->launch_mode >= 1 && !prof) {
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      lc.numAttrs = 1;
+    }
     cudaError_t e = cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
     if (prof) cudaEventRecord(ev.end, st);
     if (e != cudaSuccess) {
@@ -953,7 +958,7 @@ int thinfer_status(thinfer_ctx* c, int32_t* device_status) {
 
 int thinfer_set_launch_mode(thinfer_ctx* c, int32_t mode) {
   if (c == nullptr) return THINFER_EINVAL;
-  if (mode != 0) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
+  if (mode < 0 || mode > 1) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
   c->launch_mode = mode;
   return THINFER_OK;
 }

@@ -215,3 +215,26 @@ def test_host_buffer_calls_match_device_calls(T):
     np.testing.assert_array_equal(hout.numpy(), dev.cpu().numpy())
     np.testing.assert_array_equal(hout2.numpy(), dev2.cpu().numpy())
     ctx.close()
+
+
+@pytest.mark.parametrize("batch", [1, 5])
+def test_launch_modes_agree_bit_for_bit(T, batch):
+    # plain launches and programmatic dependent launch (kernels start early and wait on the device)
+    # run the same arithmetic in the same order: outputs and caches must be identical
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 6)
+    x = torch.from_numpy(synth.hidden_states(shape, 6, (batch, 40))).cuda()
+    outs = []
+    for mode in (0, 1):
+        ctx = _ctx(T, shape, [w], batch, 48)
+        ctx.set_launch_mode(mode)
+        res = [ctx.prefill(x[:, :33].contiguous())]
+        res += [ctx.decode_step(x[:, 33 + i].contiguous()) for i in range(7)]
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        outs.append([r.cpu().numpy() for r in res] + [ctx.kv_view(0, 0, 0).cpu().numpy()[:, :, :40],
+                                                      ctx.kv_view(0, 0, 1).cpu().numpy()[:, :, :40]])
+        ctx.close()
+    for a, b in zip(*outs):
+        np.testing.assert_array_equal(a, b)
