@@ -177,6 +177,20 @@ def run_reference(args):
     return 0
 
 
+def reduce_max_over_ranks(values, dist, device):
+    """Element-wise maximum over ranks of a list of floats (times are reported as the slowest rank's)."""
+    import torch
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_rate(units_per_rank, world, seconds):
+    """Aggregate throughput of `world` independent replicas: all units processed / slowest rank's time."""
+    return world * units_per_rank / seconds
+
+
 def workload_name(batch):
     return (f"Llama-7B-shaped single decoder layer (hidden 4096, 32x128 MHA, FFN 11008), FP16, batch {batch}, "
             f"prompt {PROMPT}, {GEN} decode steps")
@@ -252,10 +266,7 @@ def run_ours(args):
     pre_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
     dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
     tot_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
-    t = torch.tensor([pre_ms, dec_ms, tot_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    pre_ms, dec_ms, tot_ms = (float(v) for v in t.cpu())
+    pre_ms, dec_ms, tot_ms = reduce_max_over_ranks([pre_ms, dec_ms, tot_ms], dist, dev)
 
     # ---- end to end through the host-buffer entry points (pinned memory, copies inside the timed region)
     h_prompt = x_all[:, :PROMPT].contiguous().pin_memory()
@@ -277,10 +288,7 @@ def run_ours(args):
     one_step_host()
     e2e_s = sum(one_step_host() for _ in range(max(1, min(args.steps, 3))))
     e2e_steps = max(1, min(args.steps, 3))
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_s = float(te.cpu()[0])
+    e2e_s = reduce_max_over_ranks([e2e_s], dist, dev)[0]
 
     # ---- dominant kernels, timed with CUDA events around each of their launches
     def kernel_time(kid, fn):
@@ -307,9 +315,8 @@ def run_ours(args):
     ms_dec_gu = (ms_gu - ms_pre_gu) / max(1, n_gu - n_pre)
     ms_pre_gu = ms_pre_gu / max(1, n_pre)
 
-    dec_tokens = world * B * GEN * args.steps
     pre_tokens = world * B * PROMPT * args.steps
-    value = dec_tokens / (dec_ms * 1e-3)
+    value = whole_job_rate(B * GEN * args.steps, world, dec_ms * 1e-3)
     dec_bytes = sum(decode_step_bytes(SHAPE, B, PROMPT + i + 1) for i in range(GEN))
     dec_gbs = dec_bytes * args.steps / (dec_ms * 1e-3) / 1e9
     gemm_fl, attn_fl = prefill_flops(SHAPE, B * PROMPT, PROMPT)

@@ -31,7 +31,7 @@ def _ctx(T, shape, np_layers, max_batch, max_seq, stack=None, buf_slots=1):
     return thinfer.Context(shape, layers, st, max_batch=max_batch, max_seq=max_seq, buf_slots=buf_slots)
 
 
-def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_seq=None):
+def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_seq=None, check_prefill=True):
     """Prefill `seq` tokens then `n_decode` decode steps on seeded hidden states; compare everything."""
     torch, thinfer = T
     cfg = oracle_config(shape)
@@ -45,13 +45,17 @@ def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_
     assert ctx.status() == 0
     assert ctx.slot_state(0) == (batch, seq + n_decode)
     bs = list(range(batch)) if check_batches is None else check_batches
-    ref, kc, vc = O.layer_prefill(cfg, w, x[bs, :seq])
-    got = out.cpu().numpy()[bs]
-    stats = [assert_rows_close(got, ref, f"prefill B={batch} S={seq}")]
+    stats = []
     kg = ctx.kv_view(0, 0, 0).cpu().numpy()[bs]
     vg = ctx.kv_view(0, 0, 1).cpu().numpy()[bs]
-    assert_rows_close(kg[:, :, :seq], kc, "K cache after prefill", max_err=6e-3)
-    assert_rows_close(vg[:, :, :seq], vc, "V cache after prefill", max_err=6e-3)
+    if check_prefill:
+        ref, kc, vc = O.layer_prefill(cfg, w, x[bs, :seq])
+        got = out.cpu().numpy()[bs]
+        stats.append(assert_rows_close(got, ref, f"prefill B={batch} S={seq}"))
+        assert_rows_close(kg[:, :, :seq], kc, "K cache after prefill", max_err=6e-3)
+        assert_rows_close(vg[:, :, :seq], vc, "V cache after prefill", max_err=6e-3)
+    else:
+        assert np.all(np.isfinite(out.cpu().numpy().astype(np.float32)))
     # decode: the oracle continues from the GPU's own FP16 cache (chained check)
     k_run = kg[:, :, :seq].astype(np.float64)
     v_run = vg[:, :, :seq].astype(np.float64)
@@ -128,6 +132,48 @@ def test_llama7b_layer_batch1_full(T):
 def test_llama7b_layer_batched_subset(T, batch):
     # configuration 2 at batch 4 / 16: first and last request checked (batch independence covers the rest)
     _layer_case(T, synth.LLAMA_7B_LAYER, batch=batch, seq=512, n_decode=2, check_batches=[0, batch - 1], max_seq=640)
+
+
+def test_llama7b_layer_long_kv_decode(T):
+    # decode attention over 1279 .. 1281 cached keys (the KV length configuration 4 reaches); the prompt is
+    # processed on the GPU only, the decode steps are checked against the oracle continuing from that cache
+    _layer_case(T, synth.LLAMA_7B_LAYER, batch=2, seq=1279, n_decode=2, max_seq=1281, check_prefill=False, seed=3)
+
+
+def test_llama13b_layer_reduced_budget(T):
+    # configuration 4's layer shape (hidden 5120, 40 x 128 heads, FFN 13824) on a reduced token budget
+    shape = dataclasses.replace(synth.LLAMA_13B, n_layers=1, vocab=0)
+    _layer_case(T, shape, batch=2, seq=64, n_decode=2, seed=13)
+
+
+def test_llama70b_layer_reduced_budget(T):
+    # configuration 5's layer shape (hidden 8192, 64 query / 8 KV heads, FFN 28672) on a reduced token budget
+    shape = dataclasses.replace(synth.LLAMA_70B, n_layers=1, vocab=0)
+    _layer_case(T, shape, batch=2, seq=64, n_decode=2, seed=70)
+    _layer_case(T, shape, batch=1, seq=3, n_decode=2, seed=71)        # batch 1: the FMA streaming path with 8:1 GQA
+
+
+def test_llama7b_two_layer_stack_with_32000_vocab(T):
+    # configuration 3's shapes at reduced depth: embedding, 2 layers, final norm, 32000-way head, greedy pick
+    torch, thinfer = T
+    shape = dataclasses.replace(synth.LLAMA_7B, n_layers=2)
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, 3)
+    for batch in (2, 1):
+        ids = synth.token_ids(shape, 3, (batch, 34))
+        ctx = _ctx(T, shape, sw["layers"], batch, 40, stack=sw)
+        idd = torch.from_numpy(ids).cuda()
+        nxt, logits = ctx.prefill(idd[:, :32].contiguous(), want_logits=True)
+        ref_logits, _, caches, _ = O.stack_prefill(cfg, sw, ids[:, :32])
+        assert_rows_close(logits.cpu().numpy(), ref_logits, "prefill logits")
+        _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
+        for t in range(32, 34):
+            nxt, logits = ctx.decode_step(idd[:, t].contiguous(), want_logits=True)
+            ref_logits, _, caches, _ = O.stack_decode(cfg, sw, ids[:, t], caches, t)
+            assert_rows_close(logits.cpu().numpy(), ref_logits, f"decode logits t={t}")
+            _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
+        assert ctx.status() == 0
+        ctx.close()
 
 
 def test_stack_teacher_forced(T):
