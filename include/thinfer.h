@@ -150,10 +150,13 @@ int thinfer_kv_pointer(const thinfer_ctx* ctx, int32_t slot, int32_t layer, int3
  * synchronising; meaningful after the caller synchronised the stream. */
 int thinfer_status(thinfer_ctx* ctx, int32_t* device_status);
 
-/* Unified launch (Section 3.3.3: one submission for the whole operator graph
- * instead of one per operator).  mode 0: plain launches; 1: launches chained
- * with programmatic dependent launch; 2: each decode step is replayed from a
- * CUDA graph captured on first use per (slot, batch) and updated in place. */
+/* Unified launch (Section 3.3.3: one creation + launch for the whole operator
+ * graph instead of one per operator).  mode 0: one plain launch per fusion
+ * unit; 1: the same launches chained with programmatic dependent launch (each
+ * kernel starts early and waits on the device); 2: a decode step of up to 16
+ * requests runs every unit of every layer in ONE cooperative, persistent
+ * kernel with grid-wide barriers between units (larger batches and prefill
+ * fall back to mode 1). */
 int thinfer_set_launch_mode(thinfer_ctx* ctx, int32_t mode);
 
 /* Per-kernel timing for roofline reports.  When `kernel_id` >= 0 every launch
@@ -163,7 +166,7 @@ int thinfer_set_launch_mode(thinfer_ctx* ctx, int32_t mode);
 typedef enum {
   THINFER_K_RMSNORM = 0, THINFER_K_QKV = 1, THINFER_K_ATTN = 2, THINFER_K_ATTN_COMBINE = 3,
   THINFER_K_OPROJ = 4, THINFER_K_GATEUP = 5, THINFER_K_DOWN = 6, THINFER_K_HEAD = 7,
-  THINFER_K_EMBED = 8, THINFER_K_ARGMAX = 9, THINFER_K_COUNT = 10
+  THINFER_K_EMBED = 8, THINFER_K_ARGMAX = 9, THINFER_K_DECODE_UNIFIED = 10, THINFER_K_COUNT = 11
 } thinfer_kernel_id;
 int thinfer_profile_select(thinfer_ctx* ctx, int32_t kernel_id);
 int thinfer_profile_read(thinfer_ctx* ctx, int32_t* launches, float* total_ms);

@@ -47,6 +47,16 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
                : "l"(p));
   return v;
 }
+// Same streaming read for data that may have been written earlier in the same kernel (the KV row a
+// decode step has just appended): no read-only path.
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p)
+               : "memory");
+  return v;
+}
 __device__ __forceinline__ uint4 ldg_cached(const void* p) {
   return __ldg(reinterpret_cast<const uint4*>(p));
 }
@@ -105,13 +115,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
   const uint64_t t0 = global_ns();
   uint32_t polls = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++polls & 0x3ffu) == 0u) {
-      // a wait that already expired elsewhere poisons the context: give up at once
-      if (status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
-        if (status != nullptr) *reinterpret_cast<volatile int*>(status) = kErrTimeout;
-        return false;
-      }
+    // purely time-based: the warps that wait on one barrier must all take the same decision,
+    // because the ones that pass go on to a CTA-level barrier that has no time limit
+    if ((++polls & 0x3ffu) == 0u && global_ns() - t0 > kWaitLimitNs) {
+      if (status != nullptr) *reinterpret_cast<volatile int*>(status) = kErrTimeout;
+      return false;
     }
   }
   return true;
@@ -119,6 +127,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
+// Orders generic-proxy accesses (ordinary loads / stores) with async-proxy ones (TMA) on any memory.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 // Generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -28,6 +28,93 @@ struct AttnDecArgs {
   float scale_log2;       // log2(e) / sqrt(D)
 };
 
+// Streams keys t_first, t_first + t_step, ... (< t_end) in groups of UN*KPL and folds them into the
+// running (max, sum, output) of this lane group.  kb / vb already point at this lane's 8 head elements.
+template <int D, int G>
+__device__ __forceinline__ void attn_stream_keys(const __half* kb, const __half* vb, const float (&q)[G][8], int t_first,
+                                                 int t_end, int t_step, int sub, float (&m)[G], float (&l)[G],
+                                                 float (&o)[G][8]) {
+  constexpr int LPK = D / 8;
+  constexpr int KPL = 32 / LPK;
+  constexpr int UN = kAttnDecUnroll;
+  for (int tb = t_first; tb < t_end; tb += t_step) {
+    uint4 kv[UN], vv[UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      const int t = tb + u * KPL + sub;
+      if (t < t_end) {
+        kv[u] = ld_stream(kb + static_cast<size_t>(t) * D);
+        vv[u] = ld_stream(vb + static_cast<size_t>(t) * D);
+      } else {
+        kv[u] = make_uint4(0, 0, 0, 0);
+        vv[u] = make_uint4(0, 0, 0, 0);
+      }
+    }
+    float s[G][UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      float fk[8];
+      unpack8(kv[u], fk);
+      const bool valid = (tb + u * KPL + sub) < t_end;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) d = fmaf(q[g][i], fk[i], d);
+#pragma unroll
+        for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        s[g][u] = valid ? d : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float mx = m[g];
+#pragma unroll
+      for (int u = 0; u < UN; ++u) mx = fmaxf(mx, s[g][u]);
+      const float ms = (mx == -INFINITY) ? 0.f : mx;
+      const float alpha = exp2f(m[g] - ms);  // m = -inf -> 0
+      m[g] = mx;
+      l[g] *= alpha;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[g][i] *= alpha;
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const float p = exp2f(s[g][u] - ms);
+        l[g] += p;
+        float fv[8];
+        unpack8(vv[u], fv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[g][i] = fmaf(p, fv[i], o[g][i]);
+      }
+    }
+  }
+}
+
+// Merges the KPL lane groups of a warp by the online-softmax rule; afterwards every lane holds the
+// warp's state for its 8 head elements.
+template <int D, int G>
+__device__ __forceinline__ void attn_merge_lane_groups(float (&m)[G], float (&l)[G], float (&o)[G][8]) {
+  constexpr int LPK = D / 8;
+#pragma unroll
+  for (int off = LPK; off < 32; off <<= 1) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m[g], off);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l[g], off);
+      const float mx = fmaxf(m[g], m2);
+      const float ms = (mx == -INFINITY) ? 0.f : mx;
+      const float a1 = exp2f(m[g] - ms), a2 = exp2f(m2 - ms);
+      l[g] = l[g] * a1 + l2 * a2;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float o2 = __shfl_xor_sync(0xffffffffu, o[g][i], off);
+        o[g][i] = o[g][i] * a1 + o2 * a2;
+      }
+      m[g] = mx;
+    }
+  }
+}
+
 template <int D, int G>
 __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const AttnDecArgs a) {
   pdl_launch_dependents();
@@ -65,77 +152,8 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
     for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
   }
 
-  for (int tb = t0 + warp * (UN * KPL); tb < t1; tb += kAttnDecWarps * UN * KPL) {
-    uint4 kv[UN], vv[UN];
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-      const int t = tb + u * KPL + sub;
-      if (t < t1) {
-        kv[u] = ldg_stream(kb + static_cast<size_t>(t) * D);
-        vv[u] = ldg_stream(vb + static_cast<size_t>(t) * D);
-      } else {
-        kv[u] = make_uint4(0, 0, 0, 0);
-        vv[u] = make_uint4(0, 0, 0, 0);
-      }
-    }
-    float s[G][UN];
-#pragma unroll
-    for (int u = 0; u < UN; ++u) {
-      float fk[8];
-      unpack8(kv[u], fk);
-      const bool valid = (tb + u * KPL + sub) < t1;
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float d = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) d = fmaf(q[g][i], fk[i], d);
-#pragma unroll
-        for (int off = LPK / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-        s[g][u] = valid ? d : -INFINITY;
-      }
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float mx = m[g];
-#pragma unroll
-      for (int u = 0; u < UN; ++u) mx = fmaxf(mx, s[g][u]);
-      const float ms = (mx == -INFINITY) ? 0.f : mx;
-      const float alpha = exp2f(m[g] - ms);  // m = -inf -> 0
-      m[g] = mx;
-      l[g] *= alpha;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) o[g][i] *= alpha;
-#pragma unroll
-      for (int u = 0; u < UN; ++u) {
-        const float p = exp2f(s[g][u] - ms);
-        l[g] += p;
-        float fv[8];
-        unpack8(vv[u], fv);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[g][i] = fmaf(p, fv[i], o[g][i]);
-      }
-    }
-  }
-
-  // merge the KPL lane groups of the warp
-#pragma unroll
-  for (int off = LPK; off < 32; off <<= 1) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float m2 = __shfl_xor_sync(0xffffffffu, m[g], off);
-      const float l2 = __shfl_xor_sync(0xffffffffu, l[g], off);
-      const float mx = fmaxf(m[g], m2);
-      const float ms = (mx == -INFINITY) ? 0.f : mx;
-      const float a1 = exp2f(m[g] - ms), a2 = exp2f(m2 - ms);
-      l[g] = l[g] * a1 + l2 * a2;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float o2 = __shfl_xor_sync(0xffffffffu, o[g][i], off);
-        o[g][i] = o[g][i] * a1 + o2 * a2;
-      }
-      m[g] = mx;
-    }
-  }
+  attn_stream_keys<D, G>(kb, vb, q, t0 + warp * (UN * KPL), t1, kAttnDecWarps * UN * KPL, sub, m, l, o);
+  attn_merge_lane_groups<D, G>(m, l, o);
   if (sub == 0) {
 #pragma unroll
     for (int g = 0; g < G; ++g) {

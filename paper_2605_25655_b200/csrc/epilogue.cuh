@@ -31,6 +31,13 @@ struct EpiArgs {
   int seq_len;          // tokens per request in this call (1 in decode)
   int pos0;             // position of the first token of each request
   int t_max;            // KV positions per request in the cache
+  // RESID only, optional (outg != nullptr): the next RMSNorm is folded into this epilogue.  Beside
+  // y = resid + acc the kernel writes outg = y * gain_next (the operand the next projection reads)
+  // and, per 128-feature tile and token, the sum of y^2 (sumsq[feature_tile][64 tokens]); the next
+  // projection multiplies its result by rsqrt(sum over tiles / n + eps) per token.
+  __half* outg;
+  const __half* gain_next;
+  float* sumsq;
 };
 
 // Destination of element (token r, feature n of the concatenated q|k|v space).

@@ -203,8 +203,10 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
     const int c = idx >> 4, piece = idx & 15;
     const int r = tok_base + c;
     const int n0 = t.feat0 + piece * 8;  // first feature of the piece inside its matrix
-    if (r >= a.rows || n0 >= n_feat) continue;
+    const bool live = r < a.rows && n0 < n_feat;
     const int valid = min(8, n_feat - n0);
+    float sq = 0.f;
+    if (live) {
     if (EPI == EPI_QKV_ROPE) {
       const int b = r / e.seq_len, s = r - b * e.seq_len;
       const int h = n0 / e.head_dim, i = n0 - h * e.head_dim;
@@ -230,15 +232,36 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
         const float* src = st32 + c * kTcBM + piece * 8;
         if (vec) {
           float x[8];
-          unpack8(ldg_cached(e.resid + off), x);
+          unpack8(__ldcg(reinterpret_cast<const uint4*>(e.resid + off)), x);  // L2: may be written earlier in the same kernel
           uint4 o;
           o.x = pack2(x[0] + src[0], x[1] + src[1]);
           o.y = pack2(x[2] + src[2], x[3] + src[3]);
           o.z = pack2(x[4] + src[4], x[5] + src[5]);
           o.w = pack2(x[6] + src[6], x[7] + src[7]);
           *reinterpret_cast<uint4*>(dst) = o;
+          if (e.outg != nullptr) {  // folded RMSNorm of the next sub-layer (gain here, 1/rms there)
+            float y[8], g[8];
+            unpack8(o, y);
+            unpack8(ldg_cached(e.gain_next + n0), g);
+            uint4 og;
+            og.x = pack2(y[0] * g[0], y[1] * g[1]);
+            og.y = pack2(y[2] * g[2], y[3] * g[3]);
+            og.z = pack2(y[4] * g[4], y[5] * g[5]);
+            og.w = pack2(y[6] * g[6], y[7] * g[7]);
+            *reinterpret_cast<uint4*>(e.outg + off) = og;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sq = fmaf(y[j], y[j], sq);
+          }
         } else {
-          for (int j = 0; j < valid; ++j) dst[j] = __float2half_rn(__half2float(e.resid[off + j]) + src[j]);
+          for (int j = 0; j < valid; ++j) {
+            const __half yh = __float2half_rn(__half2float(__ldcg(e.resid + off + j)) + src[j]);
+            dst[j] = yh;
+            if (e.outg != nullptr) {
+              const float y = __half2float(yh);
+              e.outg[off + j] = __float2half_rn(y * __half2float(e.gain_next[n0 + j]));
+              sq = fmaf(y, y, sq);
+            }
+          }
         }
       } else {  // PLAIN_F16, SWIGLU
         __half* dst = reinterpret_cast<__half*>(e.out) + off;
@@ -249,6 +272,14 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
           for (int j = 0; j < valid; ++j) dst[j] = src[j];
         }
       }
+    }
+    }  // live
+    if (EPI == EPI_RESID && e.outg != nullptr) {
+      // the 16 pieces of one token sit in 16 consecutive lanes: add their squares, lane 0 of the group
+      // records the tile's contribution (every lane takes part in the shuffles)
+#pragma unroll
+      for (int off = 8; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+      if (piece == 0 && r < a.rows) e.sumsq[(t.feat0 / kTcBM) * 64 + r] = sq;
     }
   }
   epi_bar();
@@ -262,6 +293,94 @@ __device__ __forceinline__ void tc_load_acc(uint32_t taddr, float (&f)[CW]) {
   tmem_ld_wait();
 #pragma unroll
   for (int c = 0; c < CW; ++c) f[c] = __uint_as_float(r[c]);
+}
+
+// ---- epilogue of one segment ------------------------------------------------------------------
+// Reads the accumulator buffer of the segment from tensor memory.  A whole tile is finished
+// directly; a partial one (stream-K) is parked in the workspace and finished by the last CTA to
+// arrive, which adds the partials in slot order.  `col_scale` (shared memory, one factor per token
+// column of the tile, or nullptr) multiplies the finished sums before the element-wise part: the
+// 1/rms of a folded RMSNorm.  Called by the 128 epilogue threads.
+template <int BN, int EPI>
+__device__ __forceinline__ void tc_epilogue_segment(const TcGemmArgs& a, const TcSeg& sg, const TcTile& t, uint32_t acc,
+                                                    uint64_t* tempty, uint8_t* stage_out, int* flag, int row,
+                                                    int ethread, int lane, int nkb, const float* col_scale) {
+  constexpr int NA = tc_num_a(EPI);
+  constexpr int ACC_COLS = tc_acc_cols(BN, EPI);
+  constexpr int CW = BN >= 32 ? 32 : 16;
+  const bool whole = sg.kb0 == 0 && sg.kb1 == nkb;
+  if (whole) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CW) {
+      float v[CW], v2[CW];
+      tc_load_acc<CW>(acc + c0, v);
+      if (NA == 2) tc_load_acc<CW>(acc + BN + c0, v2);
+      if (c0 + CW >= BN) {  // accumulator fully read: hand it back to the MMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty);
+      }
+      if (col_scale != nullptr) {
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          v[c] *= col_scale[c0 + c];
+          if (NA == 2) v2[c] *= col_scale[c0 + c];
+        }
+      }
+      tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
+    }
+    return;
+  }
+  // stream-K: park the partial accumulator; the last CTA of the tile reduces and finishes it
+  const long long first_unit = static_cast<long long>(sg.tile) * nkb;
+  const int first_cta = static_cast<int>(first_unit / a.units_per_cta);
+  const int last_cta = static_cast<int>((first_unit + nkb - 1) / a.units_per_cta);
+  const int n_seg = last_cta - first_cta + 1;
+  float* slot = a.partial_ws + static_cast<size_t>(sg.tile + blockIdx.x) * (ACC_COLS * kTcBM);
+#pragma unroll 1
+  for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
+    float v[CW];
+    tc_load_acc<CW>(acc + c0, v);
+#pragma unroll
+    for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(tempty);
+  __threadfence();
+  epi_bar();
+  if (ethread == 0) {
+    const int old = atomicAdd(a.tile_counters + sg.tile, 1);
+    *flag = (old == n_seg - 1) ? 1 : 0;
+  }
+  epi_bar();
+  const bool last = *reinterpret_cast<volatile int*>(flag) != 0;
+  if (last) {
+    __threadfence();
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CW) {
+      float v[CW], v2[CW];
+#pragma unroll
+      for (int c = 0; c < CW; ++c) v[c] = v2[c] = 0.f;
+      for (int sgi = 0; sgi < n_seg; ++sgi) {  // fixed order: the result does not depend on arrival order
+        const float* src = a.partial_ws + static_cast<size_t>(sg.tile + first_cta + sgi) * (ACC_COLS * kTcBM);
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          v[c] += __ldcg(src + (c0 + c) * kTcBM + row);
+          if (NA == 2) v2[c] += __ldcg(src + (BN + c0 + c) * kTcBM + row);
+        }
+      }
+      if (col_scale != nullptr) {
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          v[c] *= col_scale[c0 + c];
+          if (NA == 2) v2[c] *= col_scale[c0 + c];
+        }
+      }
+      tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
+    }
+    if (ethread == 0) a.tile_counters[sg.tile] = 0;  // ready for the next launch
+  }
 }
 
 template <int BN, int EPI>
@@ -412,65 +531,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       tc_fence_after();
       const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
       const uint32_t acc = lane_base + buf * ACC_COLS;
-      const bool whole = sg.kb0 == 0 && sg.kb1 == nkb;
-      if (whole) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += CW) {
-          float v[CW], v2[CW];
-          tc_load_acc<CW>(acc + c0, v);
-          if (NA == 2) tc_load_acc<CW>(acc + BN + c0, v2);
-          if (c0 + CW >= BN) {  // accumulator fully read: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty_bar[buf]);
-          }
-          tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
-        }
-      } else {
-        // stream-K: park the partial accumulator; the last CTA of the tile reduces and finishes it
-        const long long first_unit = static_cast<long long>(sg.tile) * nkb;
-        const int first_cta = static_cast<int>(first_unit / a.units_per_cta);
-        const int last_cta = static_cast<int>((first_unit + nkb - 1) / a.units_per_cta);
-        const int n_seg = last_cta - first_cta + 1;
-        float* slot = a.partial_ws + static_cast<size_t>(sg.tile + blockIdx.x) * (ACC_COLS * kTcBM);
-#pragma unroll 1
-        for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
-          float v[CW];
-          tc_load_acc<CW>(acc + c0, v);
-#pragma unroll
-          for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty_bar[buf]);
-        __threadfence();
-        epi_bar();
-        if (ethread == 0) {
-          const int old = atomicAdd(a.tile_counters + sg.tile, 1);
-          *flag = (old == n_seg - 1) ? 1 : 0;
-        }
-        epi_bar();
-        const bool last = *reinterpret_cast<volatile int*>(flag) != 0;
-        if (last) {
-          __threadfence();
-#pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += CW) {
-            float v[CW], v2[CW];
-#pragma unroll
-            for (int c = 0; c < CW; ++c) v[c] = v2[c] = 0.f;
-            for (int sgi = 0; sgi < n_seg; ++sgi) {  // fixed order: the result does not depend on arrival order
-              const float* src = a.partial_ws + static_cast<size_t>(sg.tile + first_cta + sgi) * (ACC_COLS * kTcBM);
-#pragma unroll
-              for (int c = 0; c < CW; ++c) {
-                v[c] += __ldcg(src + (c0 + c) * kTcBM + row);
-                if (NA == 2) v2[c] += __ldcg(src + (BN + c0 + c) * kTcBM + row);
-              }
-            }
-            tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
-          }
-          if (ethread == 0) a.tile_counters[sg.tile] = 0;  // ready for the next launch
-        }
-      }
+      tc_epilogue_segment<BN, EPI>(a, sg, t, acc, &tempty_bar[buf], stage_out, flag, row, ethread, lane, nkb, nullptr);
     }
   }
 

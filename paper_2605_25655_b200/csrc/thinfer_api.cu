@@ -14,6 +14,7 @@
 
 #include "decode_attn.cuh"
 #include "decode_gemv.cuh"
+#include "decode_mega.cuh"
 #include "misc_kernels.cuh"
 #include "prefill_attn.cuh"
 #include "tc_gemm.cuh"
@@ -96,6 +97,14 @@ struct thinfer_ctx {
   float *part_o = nullptr, *part_ml = nullptr;
   float* splitk_ws = nullptr;   // stream-K partial accumulators
   int* splitk_counters = nullptr;
+  // unified decode kernel
+  __half *xg = nullptr, *x1g = nullptr;
+  float *sumsq0 = nullptr, *sumsq1 = nullptr, *attn_partial = nullptr;
+  int* attn_counters = nullptr;
+  unsigned int* grid_bar = nullptr;
+  unsigned int bar_base = 0;
+  MegaCommon* mega_common = nullptr;
+  MegaLayer* mega_layers = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
   // status word (pinned, mapped)
@@ -146,7 +155,8 @@ int validate_config(const thinfer_config* c, std::string* why) {
 
 struct ScratchPlan {
   size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
-      splitk_counters, stage_in, stage_out, total;
+      splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, mega_common, mega_layers,
+      stage_in, stage_out, total;
   int max_splits, max_tiles;
 };
 
@@ -189,6 +199,18 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     p.splitk_ws = take((tiles + kTcMaxCtas) * static_cast<size_t>(2 * kTcDecodeMaxBN) * 128 * 4);
     p.splitk_counters = take(tiles * 4);
   }
+  {
+    const size_t parts = (static_cast<size_t>(c.hidden) + 127) / 128;
+    p.xg = take(static_cast<size_t>(c.max_batch) * c.hidden * 2);
+    p.x1g = take(static_cast<size_t>(c.max_batch) * c.hidden * 2);
+    p.sumsq0 = take(parts * 64 * 4);
+    p.sumsq1 = take(parts * 64 * 4);
+    p.attn_partial = take((static_cast<size_t>(c.max_batch) * c.n_q_heads + kTcMaxCtas * 4) * (c.head_dim + 2) * 4);
+    p.attn_counters = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * 4);
+    p.grid_bar = take(64);
+    p.mega_common = take(sizeof(MegaCommon));
+    p.mega_layers = take(sizeof(MegaLayer) * c.n_layers);
+  }
   const size_t in_bytes = c.vocab > 0 ? M * 4 : M * c.hidden * 2;
   const size_t out_bytes = c.vocab > 0 ? static_cast<size_t>(c.max_batch) * (4 + static_cast<size_t>(c.vocab) * 4)
                                        : M * c.hidden * 2;
@@ -209,6 +231,7 @@ struct Launcher {
   thinfer_ctx* c;
   cudaStream_t st;
   int rc = THINFER_OK;
+  bool cooperative = false;  // next launch only: all CTAs must be co-resident (grid-wide barriers inside)
 
   template <typename... KArgs, typename... Args>
   void go(int kid, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
@@ -235,7 +258,12 @@ struct Launcher {
     cudaLaunchAttribute attr[1];
     lc.attrs = attr;
     lc.numAttrs = 0;
-    if (c != nullptr && c->launch_mode >= 1 && !prof) {
+    if (cooperative) {
+      attr[0].id = cudaLaunchAttributeCooperative;
+      attr[0].val.cooperative = 1;
+      lc.numAttrs = 1;
+      cooperative = false;
+    } else if (c != nullptr && c->launch_mode >= 1 && !prof) {
       attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
       attr[0].val.programmaticStreamSerializationAllowed = 1;
       lc.numAttrs = 1;
@@ -623,6 +651,81 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
   }
 }
 
+// ----------------------------------------------------------------------------
+// unified decode kernel: all layers of a step in one cooperative launch
+// ----------------------------------------------------------------------------
+template <int D, int G>
+void launch_mega(Launcher& L, thinfer_ctx* c, const MegaArgs& a) {
+  static bool ready = false;
+  constexpr int smem = mega_smem_bytes<16, D, G>();
+  if (!ready) {
+    if (!opt_in_smem(decode_mega_kernel<16, D, G>, smem)) {
+      L.rc = fail(c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+      return;
+    }
+    ready = true;
+  }
+  L.cooperative = true;
+  L.go(THINFER_K_DECODE_UNIFIED, decode_mega_kernel<16, D, G>, dim3(c->sm_count < kTcMaxCtas ? c->sm_count : kTcMaxCtas),
+       dim3(kMegaThreads), smem, a);
+}
+
+bool mega_supported(const thinfer_ctx* c, int batch) { return batch <= 16; }
+
+void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* x_in, __half* x_out, int batch, int pos) {
+  const thinfer_config& cf = c->cfg;
+  MegaArgs a{};
+  a.common = c->mega_common;
+  a.layers = c->mega_layers;
+  a.n_layers = cf.n_layers;
+  a.batch = batch;
+  a.pos = pos;
+  a.hidden = cf.hidden;
+  a.ffn = cf.ffn;
+  a.n_q_heads = cf.n_q_heads;
+  a.n_kv_heads = cf.n_kv_heads;
+  a.t_max = cf.max_seq;
+  a.eps = cf.rms_eps;
+  a.x_in = x_in;
+  a.x_out = x_out;
+  a.xa = c->xa;
+  a.xb = c->xb;
+  a.xg = c->xg;
+  a.x1 = c->x1;
+  a.x1g = c->x1g;
+  a.qbuf = c->qbuf;
+  a.attn = c->attn;
+  a.act = c->act;
+  a.sumsq0 = c->sumsq0;
+  a.sumsq1 = c->sumsq1;
+  a.kv_base = c->kv;
+  a.kv_layer_bytes = c->kv_layer_bytes;
+  a.slot = slot;
+  a.rope_cos = c->rope_cos;
+  a.rope_sin = c->rope_sin;
+  a.gemm_partial = c->splitk_ws;
+  a.gemm_counters = c->splitk_counters;
+  a.attn_partial = c->attn_partial;
+  a.attn_counters = c->attn_counters;
+  a.grid_bar = c->grid_bar;
+  a.bar_base = c->bar_base;
+  a.status = c->status_dev;
+  const int ratio = cf.n_q_heads / cf.n_kv_heads;
+  const int g = (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
+  if (cf.head_dim == 128) {
+    if (g == 4) launch_mega<128, 4>(L, c, a);
+    else if (g == 2) launch_mega<128, 2>(L, c, a);
+    else launch_mega<128, 1>(L, c, a);
+  } else {
+    if (g == 4) launch_mega<64, 4>(L, c, a);
+    else if (g == 2) launch_mega<64, 2>(L, c, a);
+    else launch_mega<64, 1>(L, c, a);
+  }
+  // every CTA arrives once per grid barrier: 5 per layer
+  const unsigned int grid = c->sm_count < kTcMaxCtas ? c->sm_count : kTcMaxCtas;
+  c->bar_base += 5u * cf.n_layers * grid;
+}
+
 // final RMSNorm + LM head + greedy argmax on `batch` rows of x [batch][hidden]
 void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, int32_t* ids_out, float* logits_out) {
   const thinfer_config& cf = c->cfg;
@@ -683,10 +786,16 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
     x = static_cast<const __half*>(input);
   }
   __half* pong[2] = {c->xb, c->xa};
-  for (int l = 0; l < cf.n_layers; ++l) {
-    __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
-    layer_decode(L, c, slot, l, x, dst, batch, pos);
+  if (c->launch_mode == 2 && mega_supported(c, batch)) {
+    __half* dst = cf.vocab == 0 ? static_cast<__half*>(out_primary) : pong[(cf.n_layers - 1) & 1];
+    layers_decode_unified(L, c, slot, x, dst, batch, pos);
     x = dst;
+  } else {
+    for (int l = 0; l < cf.n_layers; ++l) {
+      __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
+      layer_decode(L, c, slot, l, x, dst, batch, pos);
+      x = dst;
+    }
   }
   if (cf.vocab > 0) head_and_argmax(L, c, x, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits));
   return L.rc;
@@ -803,6 +912,15 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->part_ml = reinterpret_cast<float*>(s + p.part_ml);
   c->splitk_ws = reinterpret_cast<float*>(s + p.splitk_ws);
   c->splitk_counters = reinterpret_cast<int*>(s + p.splitk_counters);
+  c->xg = reinterpret_cast<__half*>(s + p.xg);
+  c->x1g = reinterpret_cast<__half*>(s + p.x1g);
+  c->sumsq0 = reinterpret_cast<float*>(s + p.sumsq0);
+  c->sumsq1 = reinterpret_cast<float*>(s + p.sumsq1);
+  c->attn_partial = reinterpret_cast<float*>(s + p.attn_partial);
+  c->attn_counters = reinterpret_cast<int*>(s + p.attn_counters);
+  c->grid_bar = reinterpret_cast<unsigned int*>(s + p.grid_bar);
+  c->mega_common = reinterpret_cast<MegaCommon*>(s + p.mega_common);
+  c->mega_layers = reinterpret_cast<MegaLayer*>(s + p.mega_layers);
   c->stage_in = s + p.stage_in;
   c->stage_out = s + p.stage_out;
   c->max_splits = p.max_splits;
@@ -842,6 +960,28 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
                                                   static_cast<double>(cfg->rope_base));
   if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 4, 0) != cudaSuccess)
     return cleanup(THINFER_ECUDA);
+  {
+    // parameter blocks of the unified decode kernel: weight tensor maps per layer, token-operand maps
+    // over the fixed scratch buffers (boxes of 16 token rows; rows beyond the batch are never stored)
+    std::vector<MegaLayer> ml(cfg->n_layers);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      const LayerMaps& m = c->maps[l];
+      ml[l].wq = m.wq; ml[l].wk = m.wk; ml[l].wv = m.wv; ml[l].wo = m.wo; ml[l].wg = m.wg; ml[l].wu = m.wu; ml[l].wd = m.wd;
+      ml[l].attn_norm = static_cast<const __half*>(c->layers[l].attn_norm);
+      ml[l].ffn_norm = static_cast<const __half*>(c->layers[l].ffn_norm);
+      ml[l].next_norm = l + 1 < cfg->n_layers ? static_cast<const __half*>(c->layers[l + 1].attn_norm) : nullptr;
+    }
+    MegaCommon mc;
+    const uint64_t rows = cfg->max_batch;
+    bool mok = make_map_2d(&mc.x_qkv, c->xg, D, rows, 16) && make_map_2d(&mc.x_o, c->attn, qd, rows, 16) &&
+               make_map_2d(&mc.x_gu, c->x1g, D, rows, 16) && make_map_2d(&mc.x_down, c->act, F, rows, 16);
+    if (!mok) return cleanup(THINFER_ECUDA);
+    if (cudaMemcpy(c->mega_layers, ml.data(), sizeof(MegaLayer) * ml.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(c->mega_common, &mc, sizeof(mc), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(c->attn_counters, 0, static_cast<size_t>(cfg->max_batch) * cfg->n_q_heads * 4) != cudaSuccess ||
+        cudaMemset(c->grid_bar, 0, 64) != cudaSuccess)
+      return cleanup(THINFER_ECUDA);
+  }
   if (cudaDeviceSynchronize() != cudaSuccess) return cleanup(THINFER_ECUDA);
   *out = c;
   return THINFER_OK;
@@ -958,7 +1098,7 @@ int thinfer_status(thinfer_ctx* c, int32_t* device_status) {
 
 int thinfer_set_launch_mode(thinfer_ctx* c, int32_t mode) {
   if (c == nullptr) return THINFER_EINVAL;
-  if (mode < 0 || mode > 1) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
+  if (mode < 0 || mode > 2) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
   c->launch_mode = mode;
   return THINFER_OK;
 }

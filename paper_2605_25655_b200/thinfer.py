@@ -16,7 +16,7 @@ OK, EINVAL, EUNSUPPORTED, ECAPACITY, EBUSY, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4,
 ERR_NAMES = {OK: "THINFER_OK", EINVAL: "THINFER_EINVAL", EUNSUPPORTED: "THINFER_EUNSUPPORTED",
              ECAPACITY: "THINFER_ECAPACITY", EBUSY: "THINFER_EBUSY", ECUDA: "THINFER_ECUDA",
              ETIMEOUT: "THINFER_ETIMEOUT"}
-K_RMSNORM, K_QKV, K_ATTN, K_ATTN_COMBINE, K_OPROJ, K_GATEUP, K_DOWN, K_HEAD, K_EMBED, K_ARGMAX = range(10)
+K_RMSNORM, K_QKV, K_ATTN, K_ATTN_COMBINE, K_OPROJ, K_GATEUP, K_DOWN, K_HEAD, K_EMBED, K_ARGMAX, K_DECODE_UNIFIED = range(11)
 
 EXPORTS = (
     "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_decode_step",

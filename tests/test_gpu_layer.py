@@ -31,13 +31,16 @@ def _ctx(T, shape, np_layers, max_batch, max_seq, stack=None, buf_slots=1):
     return thinfer.Context(shape, layers, st, max_batch=max_batch, max_seq=max_seq, buf_slots=buf_slots)
 
 
-def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_seq=None, check_prefill=True):
+def _layer_case(T, shape, batch, seq, n_decode, seed=0, check_batches=None, max_seq=None, check_prefill=True,
+                launch_mode=None):
     """Prefill `seq` tokens then `n_decode` decode steps on seeded hidden states; compare everything."""
     torch, thinfer = T
     cfg = oracle_config(shape)
     w = synth.layer_weights(shape, seed)
     x = synth.hidden_states(shape, seed, (batch, seq + n_decode))
     ctx = _ctx(T, shape, [w], batch, max_seq or (seq + n_decode))
+    if launch_mode is not None:
+        ctx.set_launch_mode(launch_mode)
     xd = torch.from_numpy(x).cuda()
     out = ctx.prefill(xd[:, :seq].contiguous())
     dec = [ctx.decode_step(xd[:, seq + i].contiguous()) for i in range(n_decode)]
@@ -80,6 +83,67 @@ def test_tiny_config_prefill_then_decode(T):
 @pytest.mark.parametrize("batch,seq,n_decode", [(2, 1, 6), (3, 130, 3), (4, 77, 2), (16, 40, 2)])
 def test_tiny_shapes_ragged(T, batch, seq, n_decode):
     _layer_case(T, synth.TINY, batch=batch, seq=seq, n_decode=n_decode, seed=batch)
+
+
+# ---- launch mode 2: the whole decode step in one cooperative persistent kernel ---------------------
+@pytest.mark.parametrize("batch,seq,n_decode", [(1, 32, 8), (2, 1, 6), (3, 130, 3), (16, 40, 3), (7, 5, 12)])
+def test_unified_decode_kernel_tiny(T, batch, seq, n_decode):
+    _layer_case(T, synth.TINY, batch=batch, seq=seq, n_decode=n_decode, seed=batch, launch_mode=2)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 128), (8, 4, 64), (6, 2, 64), (8, 1, 128)])
+def test_unified_decode_kernel_gqa(T, hq, hkv, d):
+    shape = synth.Shape(hidden=512, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, ffn=1024)
+    _layer_case(T, shape, batch=3, seq=150, n_decode=3, seed=4, launch_mode=2)
+
+
+@pytest.mark.parametrize("batch", [1, 4, 16])
+def test_unified_decode_kernel_llama7b_layer(T, batch):
+    _layer_case(T, synth.LLAMA_7B_LAYER, batch=batch, seq=512, n_decode=3, check_batches=[0, batch - 1], max_seq=640,
+                check_prefill=False, launch_mode=2)
+
+
+def test_unified_decode_kernel_multi_layer_stack(T):
+    # four layers in one launch: residual ping-pong, the next layer's norm folded into the down projection
+    torch, thinfer = T
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=688, n_layers=4, vocab=1000)
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, 5)
+    ids = synth.token_ids(shape, 5, (3, 14))
+    ctx = _ctx(T, shape, sw["layers"], 3, 16, stack=sw)
+    ctx.set_launch_mode(2)
+    idd = torch.from_numpy(ids).cuda()
+    nxt, logits = ctx.prefill(idd[:, :9].contiguous(), want_logits=True)
+    ref_logits, _, caches, _ = O.stack_prefill(cfg, sw, ids[:, :9])
+    assert_rows_close(logits.cpu().numpy(), ref_logits, "prefill logits")
+    for t in range(9, 14):
+        nxt, logits = ctx.decode_step(idd[:, t].contiguous(), want_logits=True)
+        ref_logits, _, caches, _ = O.stack_decode(cfg, sw, ids[:, t], caches, t)
+        assert_rows_close(logits.cpu().numpy(), ref_logits, f"decode logits t={t}")
+        _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
+        for l in (0, 3):                                       # caches of the first and last layer
+            kg = ctx.kv_view(0, l, 0).cpu().numpy()[:3, :, :t + 1]
+            assert_rows_close(kg, caches[l][0], f"K cache layer {l} t={t}", max_err=8e-3)
+    assert ctx.status() == 0
+    ctx.close()
+
+
+def test_unified_decode_kernel_is_deterministic(T):
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 6)
+    x = torch.from_numpy(synth.hidden_states(shape, 6, (5, 40))).cuda()
+    outs = []
+    for rep in range(2):
+        ctx = _ctx(T, shape, [w], 5, 48)
+        ctx.set_launch_mode(2)
+        res = [ctx.prefill(x[:, :33].contiguous())] + [ctx.decode_step(x[:, 33 + i].contiguous()) for i in range(7)]
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        outs.append([r.cpu().numpy() for r in res])
+        ctx.close()
+    for a, b in zip(*outs):
+        np.testing.assert_array_equal(a, b)
 
 
 def test_gqa_layer(T):
