@@ -171,6 +171,14 @@ typedef enum {
 int thinfer_profile_select(thinfer_ctx* ctx, int32_t kernel_id);
 int thinfer_profile_read(thinfer_ctx* ctx, int32_t* launches, float* total_ms);
 
+/* Trace of the unified decode kernel (launch mode 2).  enable != 0: CTA 0 of every later unified
+ * launch stores the nanosecond device timer at each unit boundary into a scratch area.  If host_out is
+ * not NULL, the area is copied to it first (synchronous copy; call after synchronising the stream):
+ * entry 0 = kernel end, 1 = start, 2 = prep done, 3 = after the first grid barrier, then per layer
+ * QKV done, barrier, attention done, barrier, O done, barrier, gate/up done, barrier, down done
+ * (, barrier).  max_entries <= 256.  Host pointer; tracing aid, not part of the hot path. */
+int thinfer_trace_unified(thinfer_ctx* ctx, int32_t enable, uint64_t* host_out, int32_t max_entries);
+
 /* Number of kernels this context has launched so far (host counter). */
 int64_t thinfer_launch_count(const thinfer_ctx* ctx);
 

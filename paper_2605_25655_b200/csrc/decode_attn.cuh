@@ -30,13 +30,12 @@ struct AttnDecArgs {
 
 // Streams keys t_first, t_first + t_step, ... (< t_end) in groups of UN*KPL and folds them into the
 // running (max, sum, output) of this lane group.  kb / vb already point at this lane's 8 head elements.
-template <int D, int G>
+template <int D, int G, int UN = kAttnDecUnroll>
 __device__ __forceinline__ void attn_stream_keys(const __half* kb, const __half* vb, const float (&q)[G][8], int t_first,
                                                  int t_end, int t_step, int sub, float (&m)[G], float (&l)[G],
                                                  float (&o)[G][8]) {
   constexpr int LPK = D / 8;
   constexpr int KPL = 32 / LPK;
-  constexpr int UN = kAttnDecUnroll;
   for (int tb = t_first; tb < t_end; tb += t_step) {
     uint4 kv[UN], vv[UN];
 #pragma unroll

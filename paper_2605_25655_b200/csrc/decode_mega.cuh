@@ -30,7 +30,7 @@ namespace thinfer {
 constexpr int kMegaThreads = 384;
 constexpr int kMegaWorkerWarps = 10;  // warps 2..11
 constexpr int kMegaWorkers = kMegaWorkerWarps * 32;
-constexpr int kMegaSlots = 5;
+constexpr int kMegaSlots = 10;  // ring of (one 128 x 64 weight tile + one token tile) slots
 constexpr int kMegaABytes = kTcBM * 128;
 
 struct alignas(64) MegaLayer {
@@ -65,6 +65,8 @@ struct MegaArgs {
   unsigned int* grid_bar;  // arrival counter of the grid barriers; holds bar_base at launch
   unsigned int bar_base;
   int* status;
+  unsigned int prefetch_ahead_bytes;  // how far (per SM) the L2 prefetch walker runs ahead of the loads
+  unsigned long long* timeline;  // optional trace: CTA 0 stores %globaltimer at every unit boundary
 };
 
 template <int D, int G>
@@ -75,7 +77,7 @@ struct MegaAttnSmem {
 
 template <int BN, int D, int G>
 __host__ __device__ constexpr int mega_smem_bytes() {
-  return kMegaSlots * (2 * kMegaABytes + BN * 128) + tc_stage_out_bytes(BN) + static_cast<int>(sizeof(MegaAttnSmem<D, G>)) +
+  return kMegaSlots * (kMegaABytes + BN * 128) + tc_stage_out_bytes(BN) + static_cast<int>(sizeof(MegaAttnSmem<D, G>)) +
          1024 /*alignment slack*/ + 512 /*barriers, flags, 1/rms*/;
 }
 
@@ -108,6 +110,8 @@ __device__ __forceinline__ void mega_gemm_desc(const MegaArgs& a, int layer, int
   g = TcGemmArgs{};
   g.rows = a.batch;
   g.mode = 1;
+  g.static_finisher = 1;  // cooperative launch: all CTAs are resident
+  g.dbg = (a.timeline != nullptr && layer == 0) ? a.timeline + 140 + 8 * phase : nullptr;
   g.partial_ws = a.gemm_partial;
   g.tile_counters = a.gemm_counters;
   g.status = a.status;
@@ -199,15 +203,94 @@ __device__ __forceinline__ bool mega_grid_sync(const MegaArgs& a, const MegaShar
   return *sh.abort == 0;
 }
 
+// ------------------------------------------------------------------ L2 prefetch walker
+// Walks this CTA's weight tiles of ALL projections of ALL layers in the order the producer will load
+// them, and asks the TMA unit to bring them into L2 ahead of time.  The walker stays a fixed number of
+// bytes ahead of the shared-memory loads, across unit boundaries: while epilogues, stream-K fix-ups and
+// grid barriers hold the loads back, HBM keeps delivering the next unit's weights into L2, and the loads
+// that follow the barrier run at L2 speed until the lead is rebuilt.
+constexpr unsigned int kMegaPrefetchAheadBytes = 0;  // off: measured slower at every distance (64 KB .. 1 MB per SM)
+
+template <int BN, int D>
+struct MegaWalker {
+  int layer, phase, kb;
+  bool have_seg, done;
+  MegaGemm m;
+  TcSegIter it;
+  TcSeg sg;
+  __device__ MegaWalker(const MegaArgs& a) : layer(0), phase(0), kb(0), have_seg(false), done(false), it(TcGemmArgs{}, 0, 1) {
+    open(a);
+  }
+  __device__ void open(const MegaArgs& a) {
+    mega_gemm_desc<BN, D>(a, layer, phase, m);
+    it = TcSegIter(m.g, m.n_tiles, m.nkb);
+    have_seg = false;
+  }
+  // Prefetches the next tile; returns its bytes, or 0 when every unit has been walked.
+  __device__ unsigned int step(const MegaArgs& a) {
+    while (!done) {
+      if (!have_seg) {
+        if (it.next(sg)) {
+          have_seg = true;
+          kb = sg.kb0;
+        } else {
+          if (++phase == 4) {
+            phase = 0;
+            if (++layer == a.n_layers) {
+              done = true;
+              return 0;
+            }
+          }
+          open(a);
+          continue;
+        }
+      }
+      // one token tile in decode: the feature tile index is the tile index
+      int ft = sg.tile;
+      const CUtensorMap* w = m.w0;
+      if (phase == 0) {
+        if (ft >= m.g.tiles[0]) {
+          ft -= m.g.tiles[0];
+          w = m.w1;
+          if (ft >= m.g.tiles[1]) {
+            ft -= m.g.tiles[1];
+            w = m.w2;
+          }
+        }
+      }
+      tma_prefetch_l2_2d(w, kb * kTcBK, ft * kTcBM);
+      unsigned int bytes = kMegaABytes;
+      if (phase == 2) {
+        tma_prefetch_l2_2d(m.w1, kb * kTcBK, ft * kTcBM);
+        bytes += kMegaABytes;
+      }
+      if (++kb == sg.kb1) have_seg = false;
+      return bytes;
+    }
+    return 0;
+  }
+};
+
 // ------------------------------------------------------------------ producer of one projection
 template <int BN, int D, int EPI>
-__device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared& sh, int layer, int phase, uint32_t& n) {
+__device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared& sh, int layer, int phase, uint32_t& n,
+                                             MegaWalker<BN, D>& walker, unsigned int& pf_bytes, unsigned int& ld_bytes) {
   constexpr int NA = tc_num_a(EPI);
-  constexpr int SLOT = 2 * kMegaABytes + BN * 128;
-  constexpr uint32_t TX = NA * kMegaABytes + BN * 128;
+  constexpr int SLOT = kMegaABytes + BN * 128;
+  constexpr uint32_t TX = SLOT;
+  auto keep_ahead = [&]() {
+    ld_bytes += kMegaABytes;
+    while (static_cast<int>(pf_bytes - ld_bytes) < static_cast<int>(a.prefetch_ahead_bytes)) {
+      const unsigned int b = walker.step(a);
+      if (b == 0) break;
+      pf_bytes += b;
+    }
+  };
   MegaGemm m;
   mega_gemm_desc<BN, D>(a, layer, phase, m);
-  // pass 1: weight tiles of the first ring-full of k-blocks, as slots come free
+  // A ring slot holds one weight tile and the token tile it is multiplied with; the gate and the up tile
+  // of a k-block are two consecutive slots.  Pass 1: the weight tiles of the first ring-full of slots are
+  // requested as slots come free, before the previous unit has finished (weights depend on nothing).
   uint32_t pre = 0;
   {
     TcSegIter it(m.g, m.n_tiles, m.nkb);
@@ -215,19 +298,19 @@ __device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared
     while (pre < kMegaSlots && it.next(sg)) {
       const TcTile t = tc_tile_coords<BN, EPI>(m.g, sg.tile, m.n_tiles, 1);
       const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (t.mat == 0 ? m.w0 : (t.mat == 1 ? m.w1 : m.w2)) : m.w0;
-      for (int kb = sg.kb0; kb < sg.kb1 && pre < kMegaSlots; ++kb, ++pre) {
+      for (int u = sg.kb0 * NA; u < sg.kb1 * NA && pre < kMegaSlots; ++u, ++pre) {
         const uint32_t q = n + pre;
         const int s = q % kMegaSlots;
         if (!mbar_wait(&sh.empty_bar[s], ((q / kMegaSlots) & 1) ^ 1u, a.status)) return false;
-        uint8_t* st = sh.ring + s * SLOT;
+        keep_ahead();
         mbar_expect_tx(&sh.full_bar[s], TX);
-        tma_load_2d(st, tmw, &sh.full_bar[s], kb * kTcBK, t.feat0);
-        if (NA == 2) tma_load_2d(st + kMegaABytes, m.w1, &sh.full_bar[s], kb * kTcBK, t.feat0);
+        tma_load_2d(sh.ring + s * SLOT, (NA == 2 && (u & 1)) ? m.w1 : tmw, &sh.full_bar[s], (u / NA) * kTcBK, t.feat0);
       }
     }
   }
   // the token operand is written by the unit before the preceding grid barrier
   if (!mega_wait_sync(sh, mega_need_sync(layer, phase), a.status)) return false;
+  if (a.timeline != nullptr && blockIdx.x == 0 && layer == 0) a.timeline[110 + phase] = global_ns();
   // pass 2
   TcSegIter it(m.g, m.n_tiles, m.nkb);
   TcSeg sg;
@@ -235,20 +318,21 @@ __device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared
   while (it.next(sg)) {
     const TcTile t = tc_tile_coords<BN, EPI>(m.g, sg.tile, m.n_tiles, 1);
     const CUtensorMap* tmw = (EPI == EPI_QKV_ROPE) ? (t.mat == 0 ? m.w0 : (t.mat == 1 ? m.w1 : m.w2)) : m.w0;
-    for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++i) {
+    for (int u = sg.kb0 * NA; u < sg.kb1 * NA; ++u, ++i) {
       const uint32_t q = n + i;
       const int s = q % kMegaSlots;
       uint8_t* st = sh.ring + s * SLOT;
       if (i >= pre) {
         if (!mbar_wait(&sh.empty_bar[s], ((q / kMegaSlots) & 1) ^ 1u, a.status)) return false;
+        keep_ahead();
         mbar_expect_tx(&sh.full_bar[s], TX);
-        tma_load_2d(st, tmw, &sh.full_bar[s], kb * kTcBK, t.feat0);
-        if (NA == 2) tma_load_2d(st + kMegaABytes, m.w1, &sh.full_bar[s], kb * kTcBK, t.feat0);
+        tma_load_2d(st, (NA == 2 && (u & 1)) ? m.w1 : tmw, &sh.full_bar[s], (u / NA) * kTcBK, t.feat0);
       }
-      tma_load_2d(st + 2 * kMegaABytes, m.x, &sh.full_bar[s], kb * kTcBK, t.tok0);
+      tma_load_2d(st + kMegaABytes, m.x, &sh.full_bar[s], (u / NA) * kTcBK, t.tok0);
     }
   }
   n += i;
+  if (a.timeline != nullptr && blockIdx.x == 0 && layer == 0) a.timeline[120 + phase] = global_ns();
   return true;
 }
 
@@ -257,7 +341,7 @@ template <int BN, int D, int EPI>
 __device__ __forceinline__ bool mega_mma(const MegaArgs& a, const MegaShared& sh, int layer, int phase, uint32_t tmem_base,
                                          uint32_t& n, uint32_t& j) {
   constexpr int NA = tc_num_a(EPI);
-  constexpr int SLOT = 2 * kMegaABytes + BN * 128;
+  constexpr int SLOT = kMegaABytes + BN * 128;
   constexpr uint32_t IDESC = idesc_f16(kTcBM, BN, 0, 0);
   MegaGemm m;
   mega_gemm_desc<BN, D>(a, layer, phase, m);
@@ -268,20 +352,17 @@ __device__ __forceinline__ bool mega_mma(const MegaArgs& a, const MegaShared& sh
     if (!mbar_wait(&sh.tempty_bar[buf], (use & 1) ^ 1u, a.status)) return false;
     tc_fence_after();
     const uint32_t acc = tmem_base + buf * (2 * BN);
-    for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
+    for (int u = sg.kb0 * NA; u < sg.kb1 * NA; ++u, ++n) {
       const int s = n % kMegaSlots;
       if (!mbar_wait(&sh.full_bar[s], (n / kMegaSlots) & 1, a.status)) return false;
       tc_fence_after();
       const uint32_t sa = smem_u32(sh.ring + s * SLOT);
       const uint64_t da = smem_desc_sw128(sa, 16, 1024);
-      const uint64_t da2 = smem_desc_sw128(sa + kMegaABytes, 16, 1024);
-      const uint64_t db = smem_desc_sw128(sa + 2 * kMegaABytes, 16, 1024);
+      const uint64_t db = smem_desc_sw128(sa + kMegaABytes, 16, 1024);
+      const uint32_t dst = acc + ((NA == 2 && (u & 1)) ? BN : 0);  // gate -> first accumulator, up -> second
+      const bool first_kb = (u / NA) == sg.kb0;
 #pragma unroll
-      for (int k = 0; k < kTcBK / 16; ++k) {
-        const uint32_t accum = (kb != sg.kb0 || k != 0) ? 1u : 0u;
-        tc_mma_f16(acc, da + 2 * k, db + 2 * k, IDESC, accum);
-        if (NA == 2) tc_mma_f16(acc + BN, da2 + 2 * k, db + 2 * k, IDESC, accum);
-      }
+      for (int k = 0; k < kTcBK / 16; ++k) tc_mma_f16(dst, da + 2 * k, db + 2 * k, IDESC, (!first_kb || k != 0) ? 1u : 0u);
       tc_commit(&sh.empty_bar[s]);
     }
     tc_commit(&sh.tfull_bar[buf]);
@@ -307,6 +388,7 @@ __device__ __forceinline__ bool mega_epilogue(const MegaArgs& a, const MegaShare
     ++j;
     if (!mbar_wait(&sh.tfull_bar[buf], use & 1, a.status)) return false;
     tc_fence_after();
+    if (a.timeline != nullptr && blockIdx.x == 0 && ethread == 0 && layer == 0) a.timeline[100 + phase] = global_ns();
     const TcTile t = tc_tile_coords<BN, EPI>(m.g, sg.tile, m.n_tiles, 1);
     tc_epilogue_segment<BN, EPI>(m.g, sg, t, lane_base + buf * (2 * BN), &sh.tempty_bar[buf], sh.stage_out, sh.flag, row,
                                  ethread, lane, m.nkb, col_scale);
@@ -372,7 +454,8 @@ __device__ __forceinline__ void mega_prep(const MegaArgs& a, float* red, int wti
 template <int D, int G>
 __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShared& sh, MegaAttnSmem<D, G>& sm,
                                                uint8_t* kc_bytes, int wtid) {
-  constexpr int LPK = D / 8, KPL = 32 / LPK, UN = kAttnDecUnroll;
+  // 10 warps per SM must keep ~80 KB of K/V rows in flight to cover the loaded DRAM latency
+  constexpr int LPK = D / 8, KPL = 32 / LPK, UN = G == 1 ? 8 : (G == 2 ? 6 : 4);
   const int wwarp = wtid >> 5, lane = wtid & 31;
   const int sub = lane / LPK, dl = lane % LPK;
   const int T = a.pos + 1;
@@ -409,7 +492,7 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
 #pragma unroll
       for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
     }
-    attn_stream_keys<D, G>(kcache + head_off, vcache + head_off, q, t0 + wwarp * (UN * KPL), t1,
+    attn_stream_keys<D, G, UN>(kcache + head_off, vcache + head_off, q, t0 + wwarp * (UN * KPL), t1,
                            kMegaWorkerWarps * UN * KPL, sub, m, l, o);
     attn_merge_lane_groups<D, G>(m, l, o);
     if (sub == 0) {
@@ -453,30 +536,50 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
       }
     }
     if (n_seg > 1) {
-      __threadfence();
-      worker_bar();
-      if (wtid == 0) {
-        const int old = atomicAdd(a.attn_counters + item, 1);
-        *sh.flag = (old == n_seg - 1) ? 1 : 0;
-      }
-      worker_bar();
-      if (*reinterpret_cast<volatile int*>(sh.flag) != 0) {
+      // The head keys of a split item are the LAST share its CTA works on; every other share of the item is
+      // the FIRST one of a later CTA and was parked long ago.  The head CTA merges, the others only park.
+      if (t0 != 0) {
         __threadfence();
-        for (int idx = wtid; idx < G * D; idx += kMegaWorkers) {
-          const int g = idx / D, i = idx - g * D;
-          float mx = -INFINITY;
-          for (int s = 0; s < n_seg; ++s)
-            mx = fmaxf(mx, __ldcg(a.attn_partial + static_cast<size_t>(item + first_cta + s) * (G * (D + 2)) + g * (D + 2) + D));
-          float L = 0.f, O = 0.f;
-          for (int s = 0; s < n_seg; ++s) {
-            const float* p = a.attn_partial + static_cast<size_t>(item + first_cta + s) * (G * (D + 2)) + g * (D + 2);
-            const float al = exp2f(__ldcg(p + D) - mx);
-            L += __ldcg(p + D + 1) * al;
-            O += __ldcg(p + i) * al;
+        worker_bar();
+        if (wtid == 0) atomicAdd(a.attn_counters + item, 1);
+      } else {
+        worker_bar();  // this CTA's own partial is complete in global memory for its own threads
+        if (wtid == 0) {
+          const uint64_t ts = global_ns();
+          uint32_t polls = 0;
+          int ok = 1;
+          for (;;) {
+            int seen;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.attn_counters + item) : "memory");
+            if (seen >= n_seg - 1) break;
+            if ((++polls & 0xffu) == 0u && global_ns() - ts > kWaitLimitNs) {
+              *reinterpret_cast<volatile int*>(a.status) = kErrTimeout;
+              ok = 0;
+              break;
+            }
           }
-          a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = __float2half_rn(O / L);
+          *sh.flag = ok;
         }
-        if (wtid == 0) a.attn_counters[item] = 0;
+        worker_bar();
+        if (*reinterpret_cast<volatile int*>(sh.flag) != 0) {
+          for (int idx = wtid; idx < G * D; idx += kMegaWorkers) {
+            const int g = idx / D, i = idx - g * D;
+            float mx = -INFINITY;
+            for (int s = 0; s < n_seg; ++s)
+              mx = fmaxf(mx, __ldcg(a.attn_partial + static_cast<size_t>(item + first_cta + s) * (G * (D + 2)) + g * (D + 2) + D));
+            float L = 0.f, O = 0.f;
+            for (int s = 0; s < n_seg; ++s) {
+              const float* p = a.attn_partial + static_cast<size_t>(item + first_cta + s) * (G * (D + 2)) + g * (D + 2);
+              const float al = exp2f(__ldcg(p + D) - mx);
+              L += __ldcg(p + D + 1) * al;
+              O += __ldcg(p + i) * al;
+            }
+            a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = __float2half_rn(O / L);
+          }
+          if (wtid == 0) a.attn_counters[item] = 0;
+        } else {
+          *sh.abort = 1;
+        }
       }
     }
     worker_bar();  // the merge area is reused by the next share
@@ -486,7 +589,7 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
 // ==================================================================== the kernel
 template <int BN, int D, int G>
 __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const MegaArgs a) {
-  constexpr int SLOT = 2 * kMegaABytes + BN * 128;
+  constexpr int SLOT = kMegaABytes + BN * 128;
   constexpr int TMEM_COLS = (4 * BN) < 32 ? 32 : (4 * BN);  // two buffers of up to two accumulators
   static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0 && TMEM_COLS <= 512, "tensor memory columns");
 
@@ -531,12 +634,14 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
   if (warp == 0) {
     if (lane == 0) {
       uint32_t n = 0;
+      unsigned int pf_bytes = 0, ld_bytes = 0;
+      MegaWalker<BN, D> walker(a);
       bool ok = true;
       for (int l = 0; l < a.n_layers && ok; ++l) {
-        ok = mega_produce<BN, D, EPI_QKV_ROPE>(a, sh, l, 0, n);
-        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 1, n);
-        ok = ok && mega_produce<BN, D, EPI_SWIGLU>(a, sh, l, 2, n);
-        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 3, n);
+        ok = mega_produce<BN, D, EPI_QKV_ROPE>(a, sh, l, 0, n, walker, pf_bytes, ld_bytes);
+        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 1, n, walker, pf_bytes, ld_bytes);
+        ok = ok && mega_produce<BN, D, EPI_SWIGLU>(a, sh, l, 2, n, walker, pf_bytes, ld_bytes);
+        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 3, n, walker, pf_bytes, ld_bytes);
       }
     }
   } else if (warp == 1) {
@@ -553,39 +658,57 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
   } else {
     const int wtid = threadIdx.x - 64;
     const bool epi = warp < 6;
+    int ts_n = 0;
+    auto stamp = [&]() {
+      if (a.timeline != nullptr && blockIdx.x == 0 && wtid == 0 && ts_n < 250) a.timeline[1 + ts_n++] = global_ns();
+    };
+    stamp();
     const int ethread = wtid;  // epilogue warps are the first four worker warps
     int epoch = 0;
     uint32_t j = 0;
     bool ok = true;
     mega_prep(a, red, wtid);
+    stamp();
     ok = mega_grid_sync(a, sh, epoch, wtid);                                   // S1
+    stamp();
     for (int l = 0; l < a.n_layers && ok; ++l) {
       if (epi) {
         mega_rstd<BN>(a, sh, a.sumsq0, ethread);
         if (!mega_epilogue<BN, D, EPI_QKV_ROPE>(a, sh, l, 0, tmem_base, j, warp, lane, sh.rstd)) *sh.abort = 1;
       }
+      stamp();
       ok = mega_grid_sync(a, sh, epoch, wtid);                                 // S2: q, K, V written
+      stamp();
       if (!ok) break;
       mega_attention<D, G>(a, sh, attn_sm,
                            a.kv_base + (static_cast<size_t>(a.slot) * a.n_layers + l) * 2 * a.kv_layer_bytes, wtid);
+      stamp();
       ok = mega_grid_sync(a, sh, epoch, wtid);                                 // S3: attention output written
+      stamp();
       if (!ok) break;
       if (epi && !mega_epilogue<BN, D, EPI_RESID>(a, sh, l, 1, tmem_base, j, warp, lane, nullptr)) *sh.abort = 1;
+      stamp();
       ok = mega_grid_sync(a, sh, epoch, wtid);                                 // S4: x1, x1g, sums written
+      stamp();
       if (!ok) break;
       if (epi) {
         mega_rstd<BN>(a, sh, a.sumsq1, ethread);
         if (!mega_epilogue<BN, D, EPI_SWIGLU>(a, sh, l, 2, tmem_base, j, warp, lane, sh.rstd)) *sh.abort = 1;
       }
+      stamp();
       ok = mega_grid_sync(a, sh, epoch, wtid);                                 // S5: act written
+      stamp();
       if (!ok) break;
       if (epi && !mega_epilogue<BN, D, EPI_RESID>(a, sh, l, 3, tmem_base, j, warp, lane, nullptr)) *sh.abort = 1;
+      stamp();
       if (l + 1 < a.n_layers) ok = mega_grid_sync(a, sh, epoch, wtid);         // S6 = S1 of the next layer
+      stamp();
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (a.timeline != nullptr && blockIdx.x == 0 && threadIdx.x == 0) a.timeline[0] = global_ns();  // kernel end
   if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 

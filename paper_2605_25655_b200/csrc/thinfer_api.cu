@@ -7,6 +7,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <string>
@@ -103,6 +104,8 @@ struct thinfer_ctx {
   int* attn_counters = nullptr;
   unsigned int* grid_bar = nullptr;
   unsigned int bar_base = 0;
+  unsigned long long* timeline = nullptr;
+  bool trace_unified = false;
   MegaCommon* mega_common = nullptr;
   MegaLayer* mega_layers = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
@@ -155,7 +158,7 @@ int validate_config(const thinfer_config* c, std::string* why) {
 
 struct ScratchPlan {
   size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
-      splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, mega_common, mega_layers,
+      splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, timeline, mega_common, mega_layers,
       stage_in, stage_out, total;
   int max_splits, max_tiles;
 };
@@ -208,6 +211,7 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     p.attn_partial = take((static_cast<size_t>(c.max_batch) * c.n_q_heads + kTcMaxCtas * 4) * (c.head_dim + 2) * 4);
     p.attn_counters = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * 4);
     p.grid_bar = take(64);
+    p.timeline = take(256 * 8);
     p.mega_common = take(sizeof(MegaCommon));
     p.mega_layers = take(sizeof(MegaLayer) * c.n_layers);
   }
@@ -710,6 +714,15 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
   a.grid_bar = c->grid_bar;
   a.bar_base = c->bar_base;
   a.status = c->status_dev;
+  a.timeline = c->trace_unified ? c->timeline : nullptr;
+  {
+    // debug knob: THINFER_UNIFIED_PREFETCH_KB overrides the L2 prefetch distance (0 switches it off)
+    static const long kb = [] {
+      const char* e = getenv("THINFER_UNIFIED_PREFETCH_KB");
+      return e ? atol(e) : static_cast<long>(kMegaPrefetchAheadBytes / 1024);
+    }();
+    a.prefetch_ahead_bytes = static_cast<unsigned int>(kb < 0 ? 0 : kb) * 1024u;
+  }
   const int ratio = cf.n_q_heads / cf.n_kv_heads;
   const int g = (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
   if (cf.head_dim == 128) {
@@ -919,6 +932,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->attn_partial = reinterpret_cast<float*>(s + p.attn_partial);
   c->attn_counters = reinterpret_cast<int*>(s + p.attn_counters);
   c->grid_bar = reinterpret_cast<unsigned int*>(s + p.grid_bar);
+  c->timeline = reinterpret_cast<unsigned long long*>(s + p.timeline);
   c->mega_common = reinterpret_cast<MegaCommon*>(s + p.mega_common);
   c->mega_layers = reinterpret_cast<MegaLayer*>(s + p.mega_layers);
   c->stage_in = s + p.stage_in;
@@ -1123,6 +1137,17 @@ int thinfer_profile_read(thinfer_ctx* c, int32_t* launches, float* total_ms) {
   *launches = static_cast<int32_t>(c->prof_used);
   *total_ms = sum;
   c->prof_used = 0;
+  return THINFER_OK;
+}
+
+int thinfer_trace_unified(thinfer_ctx* c, int32_t enable, uint64_t* host_out, int32_t max_entries) {
+  if (c == nullptr) return THINFER_EINVAL;
+  c->trace_unified = enable != 0;
+  if (host_out != nullptr && max_entries > 0) {
+    const int n = max_entries < 256 ? max_entries : 256;
+    if (cudaMemcpy(host_out, c->timeline, static_cast<size_t>(n) * 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return fail(c, THINFER_ECUDA, "reading the timeline failed");
+  }
   return THINFER_OK;
 }
 

@@ -22,7 +22,7 @@ EXPORTS = (
     "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_decode_step",
     "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
     "thinfer_kv_pointer", "thinfer_status", "thinfer_set_launch_mode", "thinfer_profile_select",
-    "thinfer_profile_read", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
+    "thinfer_profile_read", "thinfer_trace_unified", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
     "thinfer_op_linear", "thinfer_op_linear_noalloc", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
 )
 
@@ -76,6 +76,7 @@ def lib():
     L.thinfer_set_launch_mode.argtypes = [vp, i32]
     L.thinfer_profile_select.argtypes = [vp, i32]
     L.thinfer_profile_read.argtypes = [vp, C.POINTER(i32), C.POINTER(C.c_float)]
+    L.thinfer_trace_unified.argtypes = [vp, i32, C.POINTER(C.c_uint64), i32]
     L.thinfer_launch_count.argtypes = [vp]
     L.thinfer_launch_count.restype = i64
     L.thinfer_last_error.argtypes = [vp]
@@ -224,6 +225,12 @@ class Context:
         n, ms = C.c_int32(0), C.c_float(0)
         _check(lib().thinfer_profile_read(self.h, C.byref(n), C.byref(ms)), self.h)
         return n.value, ms.value
+
+    def trace_unified(self, enable=True, read=0):
+        """Switches the unit-boundary trace of the unified decode kernel on/off; returns `read` entries (ns)."""
+        buf = (C.c_uint64 * max(read, 1))()
+        _check(lib().thinfer_trace_unified(self.h, int(enable), buf if read else None, read), self.h)
+        return list(buf)[:read]
 
     def launch_count(self):
         return int(lib().thinfer_launch_count(self.h))
