@@ -30,25 +30,32 @@ struct AttnDecArgs {
 
 // Streams keys t_first, t_first + t_step, ... (< t_end) in groups of UN*KPL and folds them into the
 // running (max, sum, output) of this lane group.  kb / vb already point at this lane's 8 head elements.
-template <int D, int G, int UN = kAttnDecUnroll>
+template <int D, int G, int UN = kAttnDecUnroll, bool PIPELINED = true>
 __device__ __forceinline__ void attn_stream_keys(const __half* kb, const __half* vb, const float (&q)[G][8], int t_first,
                                                  int t_end, int t_step, int sub, float (&m)[G], float (&l)[G],
                                                  float (&o)[G][8]) {
   constexpr int LPK = D / 8;
   constexpr int KPL = 32 / LPK;
-  for (int tb = t_first; tb < t_end; tb += t_step) {
-    uint4 kv[UN], vv[UN];
+  // software pipeline: the K/V rows of the next group are requested before the current group is
+  // consumed, so loads are in flight during the arithmetic
+  uint4 kv[UN], vv[UN];
+  auto fetch = [&](int tb, uint4 (&k)[UN], uint4 (&v)[UN]) {
 #pragma unroll
     for (int u = 0; u < UN; ++u) {
       const int t = tb + u * KPL + sub;
       if (t < t_end) {
-        kv[u] = ld_stream(kb + static_cast<size_t>(t) * D);
-        vv[u] = ld_stream(vb + static_cast<size_t>(t) * D);
+        k[u] = ld_stream(kb + static_cast<size_t>(t) * D);
+        v[u] = ld_stream(vb + static_cast<size_t>(t) * D);
       } else {
-        kv[u] = make_uint4(0, 0, 0, 0);
-        vv[u] = make_uint4(0, 0, 0, 0);
+        k[u] = make_uint4(0, 0, 0, 0);
+        v[u] = make_uint4(0, 0, 0, 0);
       }
     }
+  };
+  if (t_first < t_end) fetch(t_first, kv, vv);
+  for (int tb = t_first; tb < t_end; tb += t_step) {
+    uint4 kn[UN], vn[UN];
+    if (PIPELINED && tb + t_step < t_end) fetch(tb + t_step, kn, vn);
     float s[G][UN];
 #pragma unroll
     for (int u = 0; u < UN; ++u) {
@@ -85,6 +92,15 @@ __device__ __forceinline__ void attn_stream_keys(const __half* kb, const __half*
 #pragma unroll
         for (int i = 0; i < 8; ++i) o[g][i] = fmaf(p, fv[i], o[g][i]);
       }
+    }
+    if (PIPELINED) {
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        kv[u] = kn[u];
+        vv[u] = vn[u];
+      }
+    } else if (tb + t_step < t_end) {
+      fetch(tb + t_step, kv, vv);
     }
   }
 }

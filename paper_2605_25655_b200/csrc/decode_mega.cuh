@@ -28,7 +28,7 @@
 namespace thinfer {
 
 constexpr int kMegaThreads = 384;
-constexpr int kMegaWorkerWarps = 10;  // warps 2..11
+constexpr int kMegaWorkerWarps = 10;  // warps 2..11 (384 threads: 168 registers per thread)
 constexpr int kMegaWorkers = kMegaWorkerWarps * 32;
 constexpr int kMegaSlots = 10;  // ring of (one 128 x 64 weight tile + one token tile) slots
 constexpr int kMegaABytes = kTcBM * 128;
@@ -81,7 +81,7 @@ __host__ __device__ constexpr int mega_smem_bytes() {
          1024 /*alignment slack*/ + 512 /*barriers, flags, 1/rms*/;
 }
 
-__device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 2, 320;" ::: "memory"); }
+__device__ __forceinline__ void worker_bar() { asm volatile("bar.sync 2, %0;" ::"n"(kMegaWorkers) : "memory"); }
 
 struct MegaShared {
   uint8_t* ring;
@@ -454,8 +454,7 @@ __device__ __forceinline__ void mega_prep(const MegaArgs& a, float* red, int wti
 template <int D, int G>
 __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShared& sh, MegaAttnSmem<D, G>& sm,
                                                uint8_t* kc_bytes, int wtid) {
-  // 10 warps per SM must keep ~80 KB of K/V rows in flight to cover the loaded DRAM latency
-  constexpr int LPK = D / 8, KPL = 32 / LPK, UN = G == 1 ? 8 : (G == 2 ? 6 : 4);
+  constexpr int LPK = D / 8, KPL = 32 / LPK, UN = 4;
   const int wwarp = wtid >> 5, lane = wtid & 31;
   const int sub = lane / LPK, dl = lane % LPK;
   const int T = a.pos + 1;
@@ -492,7 +491,8 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
 #pragma unroll
       for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
     }
-    attn_stream_keys<D, G, UN>(kcache + head_off, vcache + head_off, q, t0 + wwarp * (UN * KPL), t1,
+    attn_stream_keys<D, G, UN, false>(kcache + head_off,  // not pipelined: 168 registers per thread here
+                                      vcache + head_off, q, t0 + wwarp * (UN * KPL), t1,
                            kMegaWorkerWarps * UN * KPL, sub, m, l, o);
     attn_merge_lane_groups<D, G>(m, l, o);
     if (sub == 0) {
@@ -608,7 +608,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
   sh.flag = reinterpret_cast<int*>(tmem_holder + 1);
   sh.sync_count = sh.flag + 1;
   sh.abort = sh.flag + 2;
-  float* red = reinterpret_cast<float*>(sh.flag + 4);  // [10]
+  float* red = reinterpret_cast<float*>(sh.flag + 4);  // [worker warps]
   sh.rstd = red + 12;                                   // [BN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -48,6 +48,9 @@ struct TcGemmArgs {
   float* partial_ws;  // stream-K: [n_tiles + grid][NA*BN][128] FP32 partial accumulators
   int* tile_counters; // stream-K: [n_tiles] arrival counters, zero between launches
   unsigned long long* dbg;  // optional trace slots
+  const float* sumsq_in;  // folded RMSNorm (see EpiArgs): per-tile sums of squares of the token operand, or nullptr
+  int norm_dim;           // length of the normalised rows
+  float norm_eps;
   int static_finisher;  // stream-K inside a cooperative launch: the CTA that holds the head of a tile finishes it
   int* status;        // device-visible status word
   EpiArgs e;
@@ -72,7 +75,7 @@ __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {
   return c;
 }
 __host__ __device__ constexpr int tc_smem_bytes(int bn, int epi) {
-  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + tc_stage_out_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + tc_stage_out_bytes(bn) + 1024 /*alignment slack*/ + 512 /*barriers, 1/rms*/;
 }
 __host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) { return epi == EPI_RESID || epi == EPI_PLAIN_F32; }
 
@@ -486,6 +489,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   uint64_t* tempty_bar = tfull_bar + 2;       // [2] accumulator drained by the epilogue
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   int* flag = reinterpret_cast<int*>(tmem_holder + 1);
+  float* rstd_sm = reinterpret_cast<float*>(flag + 1);  // [BN] 1/rms per token column when the norm is folded
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
@@ -600,6 +604,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const int ethread = (warp - 2) * 32 + lane;
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     pdl_wait();  // residual stream, RoPE positions, stream-K scratch: all written by earlier kernels
+    if (a.sumsq_in != nullptr) {
+      // one token tile (decode): 1/rms per token from the per-tile sums the previous projection left
+      if (ethread < BN) {
+        float r = 0.f;
+        if (ethread < a.rows) {
+          const int parts = (a.norm_dim + kTcBM - 1) / kTcBM;
+          float ssum = 0.f;
+          for (int p = 0; p < parts; ++p) ssum += __ldcg(a.sumsq_in + p * 64 + ethread);
+          r = rsqrtf(ssum / static_cast<float>(a.norm_dim) + a.norm_eps);
+        }
+        rstd_sm[ethread] = r;
+      }
+      epi_bar();
+    }
+    const float* col_scale = a.sumsq_in != nullptr ? rstd_sm : nullptr;
     TcSegIter it(a, n_tiles, nkb);
     TcSeg sg;
     uint32_t j = 0;
@@ -610,7 +629,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       tc_fence_after();
       const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
       const uint32_t acc = lane_base + buf * ACC_COLS;
-      tc_epilogue_segment<BN, EPI>(a, sg, t, acc, &tempty_bar[buf], stage_out, flag, row, ethread, lane, nkb, nullptr);
+      tc_epilogue_segment<BN, EPI>(a, sg, t, acc, &tempty_bar[buf], stage_out, flag, row, ethread, lane, nkb, col_scale);
     }
   }
 

@@ -343,7 +343,8 @@ void launch_tc_bn(Launcher& L, int kid, int bn, const CUtensorMap& w0, const CUt
 // x: activations [rows][k]; the token-side tensor map is encoded per call (host only, no device work)
 template <int EPI>
 void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
-               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e, bool stream_k = false) {
+               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e, bool stream_k = false,
+               const float* sumsq_in = nullptr, float norm_eps = 0.f) {
   if (L.rc != THINFER_OK) return;
   const int bn = pick_bn(rows, EPI);
   CUtensorMap mx;
@@ -361,6 +362,9 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   a.k = k;
   a.status = L.c ? L.c->status_dev : nullptr;
   a.e = e;
+  a.sumsq_in = sumsq_in;
+  a.norm_dim = k;
+  a.norm_eps = norm_eps;
   if (stream_k && L.c != nullptr && rows <= kTcDecodeMaxBN) {
     a.mode = 1;
     a.partial_ws = L.c->splitk_ws;
@@ -589,11 +593,16 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     // batched decode: the weight stream feeds the tensor cores (stream-K over all SMs); plain FMA
     // cannot keep up with HBM beyond a couple of tokens per weight
     const LayerMaps& m = c->maps[layer];
-    rmsnorm_rows(L, x_in, H(w.attn_norm), c->h, batch, cf.hidden, cf.rms_eps);
+    // The RMSNorm in front of a projection is folded into the projection before it: that one's residual
+    // epilogue also writes (output x next gain) and the per-tile sums of squares; the consumer multiplies
+    // its sums by 1/rms.  Only the first norm of a step still needs its own small kernel.
+    const bool first_norm_folded = layer > 0;
+    const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
+    if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->h, batch, cf.hidden, cf.rms_eps);
     {
       const int nf[3] = {qd, kvd, kvd};
-      tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, batch, cf.hidden, nf, qkv_epi(c, kc, vc, 1, pos),
-                              true);
+      tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, first_norm_folded ? c->xg : c->h, batch, cf.hidden, nf,
+                              qkv_epi(c, kc, vc, 1, pos), true, first_norm_folded ? c->sumsq0 : nullptr, cf.rms_eps);
     }
     attn_decode(L, c, c->qbuf, kc, vc, c->attn, batch, pos + 1);
     {
@@ -601,22 +610,30 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
       e.out = c->x1;
       e.resid = x_in;
       e.ld_out = cf.hidden;
+      e.outg = c->x1g;
+      e.gain_next = H(w.ffn_norm);
+      e.sumsq = c->sumsq1;
       const int nf[3] = {cf.hidden, 0, 0};
       tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->attn, batch, qd, nf, e, true);
     }
-    rmsnorm_rows(L, c->x1, H(w.ffn_norm), c->h, batch, cf.hidden, cf.rms_eps);
     {
       EpiArgs e{};
       e.out = c->act;
       e.ld_out = cf.ffn;
       const int nf[3] = {cf.ffn, cf.ffn, 0};
-      tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->h, batch, cf.hidden, nf, e, true);
+      tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->x1g, batch, cf.hidden, nf, e, true, c->sumsq1,
+                            cf.rms_eps);
     }
     {
       EpiArgs e{};
       e.out = x_out;
       e.resid = c->x1;
       e.ld_out = cf.hidden;
+      if (next_gain != nullptr) {
+        e.outg = c->xg;
+        e.gain_next = next_gain;
+        e.sumsq = c->sumsq0;
+      }
       const int nf[3] = {cf.hidden, 0, 0};
       tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->act, batch, cf.ffn, nf, e, true);
     }
