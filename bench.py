@@ -389,6 +389,65 @@ def run_profile_case(args):
     return 0
 
 
+# Operator latencies the paper prints for MT-3000 (one cluster for Linear; cluster count not stated for
+# attention), quoted for context beside the B200 numbers: Table 8 (FP16 Linear, input dim 4096, ms) and
+# Table 9 ("MT Attention", batch 4, head_dim 128, ms).
+PAPER_TABLE8_FP16_MS = {
+    1024: [0.52, 0.64, 0.90, 1.62, 2.03, 2.93, 3.88], 2048: [0.66, 1.05, 1.45, 1.95, 3.38, 5.05, 6.53],
+    4096: [1.59, 2.19, 3.28, 3.62, 6.80, 9.54, 12.52], 8192: [3.05, 4.45, 5.81, 7.67, 12.93, 18.47, 24.17]}
+TABLE8_OUT = [256, 512, 768, 1024, 2048, 3072, 4096]
+PAPER_TABLE9_MT_MS = {32: [9.72, 25.13, 32.45, 79.00, 107.61, 119.39, 191.98, 248.26],
+                      64: [18.20, 49.29, 63.20, 156.56, 212.08, 236.59, 381.52, 496.23]}
+TABLE9_SEQ = [512, 1024, 1536, 2048, 2560, 3072, 3584, 4096]
+
+
+def run_tables(args):
+    """Operator micro-benchmarks at the shapes of the paper's Tables 8 and 9 (context, not the headline)."""
+    import torch
+    from paper_2605_25655_b200 import thinfer
+
+    def timed(fn, reps=5, inner=20):
+        # `inner` back-to-back launches per measurement so that the device, not the host call path, is timed
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(inner):
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / inner)
+        return float(np.median(ts))
+
+    g = torch.Generator(device="cuda").manual_seed(0)
+    rows = []
+    for s_len in (1024, 2048, 4096, 8192):
+        x = torch.randn(s_len, 4096, device="cuda", dtype=torch.float16, generator=g)
+        for j, n_out in enumerate(TABLE8_OUT):
+            w = torch.randn(n_out, 4096, device="cuda", dtype=torch.float16, generator=g) * 0.02
+            y = torch.empty(s_len, n_out, device="cuda", dtype=torch.float16)
+            ms = timed(lambda: thinfer.op_linear(x, w, path=0, out=y))
+            rows.append({"op": "linear_fp16", "rows": s_len, "in": 4096, "out": n_out, "ms": ms,
+                         "tflops": 2.0 * s_len * 4096 * n_out / (ms * 1e-3) / 1e12,
+                         "paper_mt3000_ms": PAPER_TABLE8_FP16_MS[s_len][j]})
+    for heads in (32, 64):
+        for j, s_len in enumerate(TABLE9_SEQ):
+            q = torch.randn(4, heads, s_len, 128, device="cuda", dtype=torch.float16, generator=g)
+            k = torch.randn(4, heads, s_len, 128, device="cuda", dtype=torch.float16, generator=g)
+            v = torch.randn(4, heads, s_len, 128, device="cuda", dtype=torch.float16, generator=g)
+            o = torch.empty(4, s_len, heads * 128, device="cuda", dtype=torch.float16)
+            ms = timed(lambda: thinfer.op_attention_prefill(q, k, v, out=o))
+            rows.append({"op": "attention_causal_fp16", "batch": 4, "heads": heads, "seq": s_len, "head_dim": 128,
+                         "ms": ms, "tflops": 2.0 * 4 * heads * s_len * s_len * 128 / (ms * 1e-3) / 1e12,
+                         "paper_mt3000_ms": PAPER_TABLE9_MT_MS[heads][j]})
+            del q, k, v
+    print(json.dumps({"tables": rows, "note": "B200 latencies at the shapes of the paper's Tables 8 and 9; the paper "
+                      "column is MT-3000 hardware (context only); attention FLOPs counted causal (2*S^2*d per head)"}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,7 +459,10 @@ def main():
     ap.add_argument("--profile", choices=["prefill", "decode"], default=None,
                     help="run one small pass of a phase and exit (the case ncu captures)")
     ap.add_argument("--profile-decode-steps", type=int, default=2)
+    ap.add_argument("--tables", action="store_true", help="operator micro-benchmarks at the paper's Table 8 / 9 shapes")
     args = ap.parse_args()
+    if args.tables:
+        return run_tables(args)
     if args.profile:
         return run_profile_case(args)
     if args.impl == "reference":

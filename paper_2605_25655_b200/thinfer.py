@@ -248,11 +248,14 @@ class Context:
 
 
 # ---------------------------------------------------------------- operators
-def op_linear(x, w, out_fp32=False, path=0, stream=None):
+def op_linear(x, w, out_fp32=False, path=0, stream=None, out=None):
     import torch
     rows, k = x.shape
     n_out = w.shape[0]
-    y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else torch.float16, device=x.device)
+    if out is not None:
+        y, out_fp32 = out, out.dtype == torch.float32
+    else:
+        y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else torch.float16, device=x.device)
     _check(lib().thinfer_op_linear(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k, int(out_fp32), path,
                                    _stream_ptr(stream)))
     return y
@@ -271,12 +274,13 @@ def op_linear_noalloc(x, w, y, stream=None):
     return y
 
 
-def op_attention_prefill(q, k, v, seq=None, stream=None):
+def op_attention_prefill(q, k, v, seq=None, stream=None, out=None):
     """q [B, Hq, S, d]; k, v [B, Hkv, T, d] with T >= S (the first S positions are used) -> [B, S, Hq*d]."""
     import torch
     b, hq, s, d = q.shape
     hkv, t = k.shape[1], k.shape[2]
-    out = torch.empty(b, s, hq * d, dtype=torch.float16, device=q.device)
+    if out is None:
+        out = torch.empty(b, s, hq * d, dtype=torch.float16, device=q.device)
     _check(lib().thinfer_op_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), b, hq, hkv,
                                               s, t, d, _stream_ptr(stream)))
     return out

@@ -146,6 +146,14 @@ def test_unified_decode_kernel_is_deterministic(T):
         np.testing.assert_array_equal(a, b)
 
 
+@pytest.mark.parametrize("batch", [17, 33, 64])
+def test_decode_with_more_than_16_requests(T, batch):
+    # token tiles of 32 and 64 in the stream-K decode projections; launch mode 2 falls back to per-unit kernels
+    for mode in (1, 2):
+        _layer_case(T, synth.TINY, batch=batch, seq=9, n_decode=2, seed=batch, launch_mode=mode,
+                    check_batches=[0, batch // 2, batch - 1])
+
+
 def test_gqa_layer(T):
     shape = synth.Shape(hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1024)
     _layer_case(T, shape, batch=2, seq=150, n_decode=3, seed=4)
