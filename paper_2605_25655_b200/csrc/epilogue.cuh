@@ -12,7 +12,8 @@ enum Epi : int {
   EPI_PLAIN_F32 = 1,  // y[r][n] = acc                         (FP32 store: logits)
   EPI_QKV_ROPE = 2,   // RoPE on q and k rows, q -> q buffer, k/v -> KV cache (Algorithm 1)
   EPI_RESID = 3,      // y[r][n] = resid[r][n] + acc           (O and down projections)
-  EPI_SWIGLU = 4      // a[r][f] = silu(acc_gate) * acc_up     (gate/up projection)
+  EPI_SWIGLU = 4,     // a[r][f] = silu(acc_gate) * acc_up     (gate/up projection; two accumulators per tile)
+  EPI_SWIGLU_IL = 5   // the same with 64 gate rows and 64 up rows interleaved in ONE 128-row tile (prefill)
 };
 
 struct EpiArgs {

@@ -77,7 +77,11 @@ __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {
 __host__ __device__ constexpr int tc_smem_bytes(int bn, int epi) {
   return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + tc_stage_out_bytes(bn) + 1024 /*alignment slack*/ + 512 /*barriers, 1/rms*/;
 }
-__host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) { return epi == EPI_RESID || epi == EPI_PLAIN_F32; }
+__host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) {
+  return epi == EPI_RESID || epi == EPI_PLAIN_F32 || epi == EPI_SWIGLU_IL;
+}
+// output features per tile: the interleaved gate/up tile produces 64 (its 128 rows are 64 gate + 64 up rows)
+__host__ __device__ constexpr int tc_tile_feats(int epi) { return epi == EPI_SWIGLU_IL ? 64 : kTcBM; }
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -148,7 +152,7 @@ __device__ __forceinline__ TcTile tc_tile_coords(const TcGemmArgs& a, int tile, 
       }
     }
   }
-  t.feat0 = ft * kTcBM;
+  t.feat0 = ft * tc_tile_feats(EPI);
   return t;
 }
 
@@ -204,6 +208,32 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
 
   // ---------------- phase B
   const int n_feat = a.n_feat[t.mat];
+  if (EPI == EPI_SWIGLU_IL) {
+    // rows 0..63 of the tile are gate features f0..f0+63, rows 64..127 the up rows of the same features
+#pragma unroll
+    for (int idx = ethread; idx < CW * 8; idx += 128) {
+      const int c = idx >> 3, piece = idx & 7;
+      const int r = tok_base + c;
+      const int n0 = t.feat0 + piece * 8;
+      if (r < a.rows && n0 < n_feat) {
+        const float* g = st32 + c * kTcBM + piece * 8;
+        const float* u = g + 64;
+        __half* dst = reinterpret_cast<__half*>(e.out) + static_cast<size_t>(r) * e.ld_out + n0;
+        if (n_feat - n0 >= 8 && (e.ld_out & 7) == 0) {
+          uint4 o;
+          o.x = pack2(silu_f(g[0]) * u[0], silu_f(g[1]) * u[1]);
+          o.y = pack2(silu_f(g[2]) * u[2], silu_f(g[3]) * u[3]);
+          o.z = pack2(silu_f(g[4]) * u[4], silu_f(g[5]) * u[5]);
+          o.w = pack2(silu_f(g[6]) * u[6], silu_f(g[7]) * u[7]);
+          *reinterpret_cast<uint4*>(dst) = o;
+        } else {
+          for (int j = 0; j < min(8, n_feat - n0); ++j) dst[j] = __float2half_rn(silu_f(g[j]) * u[j]);
+        }
+      }
+    }
+    epi_bar();
+    return;
+  }
 #pragma unroll
   for (int idx = ethread; idx < CW * 16; idx += 128) {
     const int c = idx >> 4, piece = idx & 15;
@@ -535,6 +565,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             mbar_expect_tx(&full_bar[n], STAGE_BYTES);
             tma_load_2d(st, tmw, &full_bar[n], kb * kTcBK, t.feat0);
             if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[n], kb * kTcBK, t.feat0);
+            if (EPI == EPI_SWIGLU_IL) tma_load_2d(st + A_BYTES / 2, &tm_w1, &full_bar[n], kb * kTcBK, t.feat0);
           }
         }
       }
@@ -557,6 +588,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             mbar_expect_tx(&full_bar[s], STAGE_BYTES);
             tma_load_2d(st, tmw, &full_bar[s], kb * kTcBK, t.feat0);
             if (NA == 2) tma_load_2d(st + A_BYTES, &tm_w1, &full_bar[s], kb * kTcBK, t.feat0);
+            if (EPI == EPI_SWIGLU_IL) tma_load_2d(st + A_BYTES / 2, &tm_w1, &full_bar[s], kb * kTcBK, t.feat0);
           }
           tma_load_2d(st + NA * A_BYTES, &tm_x, &full_bar[s], kb * kTcBK, t.tok0);
         }

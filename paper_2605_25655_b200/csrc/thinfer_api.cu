@@ -67,6 +67,7 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct LayerMaps {
   CUtensorMap wq, wk, wv, wo, wg, wu, wd;
+  CUtensorMap wg64, wu64;  // 64-row boxes: gate and up rows share one 128-row tile in prefill
 };
 
 struct Slot {
@@ -355,9 +356,9 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   TcGemmArgs a{};
   for (int i = 0; i < 3; ++i) {
     a.n_feat[i] = n_feat[i];
-    a.tiles[i] = (n_feat[i] + kTcBM - 1) / kTcBM;
+    a.tiles[i] = (n_feat[i] + tc_tile_feats(EPI) - 1) / tc_tile_feats(EPI);
   }
-  if (EPI == EPI_SWIGLU) a.tiles[1] = 0;  // gate and up tiles are processed together
+  if (EPI == EPI_SWIGLU || EPI == EPI_SWIGLU_IL) a.tiles[1] = 0;  // gate and up rows are processed together
   a.rows = rows;
   a.k = k;
   a.status = L.c ? L.c->status_dev : nullptr;
@@ -569,7 +570,8 @@ void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __hal
     e.out = c->act;
     e.ld_out = cf.ffn;
     const int nf[3] = {cf.ffn, cf.ffn, 0};
-    tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->h, rows, cf.hidden, nf, e);
+    if (rows > 64) tc_linear<EPI_SWIGLU_IL>(L, THINFER_K_GATEUP, m.wg64, m.wu64, m.wu64, c->h, rows, cf.hidden, nf, e);
+    else tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->h, rows, cf.hidden, nf, e);
   }
   {
     EpiArgs e{};
@@ -978,7 +980,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     ok = ok && make_map_2d(&m.wq, w.wq, D, qd, 128) && make_map_2d(&m.wk, w.wk, D, kvd, 128) &&
          make_map_2d(&m.wv, w.wv, D, kvd, 128) && make_map_2d(&m.wo, w.wo, qd, D, 128) &&
          make_map_2d(&m.wg, w.w_gate, D, F, 128) && make_map_2d(&m.wu, w.w_up, D, F, 128) &&
-         make_map_2d(&m.wd, w.w_down, F, D, 128);
+         make_map_2d(&m.wd, w.w_down, F, D, 128) && make_map_2d(&m.wg64, w.w_gate, D, F, 64) &&
+         make_map_2d(&m.wu64, w.w_up, D, F, 64);
   }
   if (ok && cfg->vocab > 0) ok = make_map_2d(&c->map_head, c->lm_head, D, cfg->vocab, 128);
   if (!ok) {
