@@ -46,7 +46,7 @@ struct TcGemmArgs {
   int mode;       // 0 = whole tiles round-robin, 1 = stream-K
   int units_per_cta;  // stream-K: (tile, k-block) units per CTA
   float* partial_ws;  // stream-K: [n_tiles + grid][NA*BN][128] FP32 partial accumulators
-  int* tile_counters; // stream-K: [n_tiles] arrival counters, zero between launches
+  int* tile_counters; // stream-K: [n_tiles][2] arrival counters (claimed, parked), zero between launches
   unsigned long long* dbg;  // optional trace slots
   const float* sumsq_in;  // folded RMSNorm (see EpiArgs): per-tile sums of squares of the token operand, or nullptr
   int norm_dim;           // length of the normalised rows
@@ -367,22 +367,26 @@ __device__ __forceinline__ void tc_epilogue_segment(const TcGemmArgs& a, const T
     }
     return;
   }
-  // stream-K
+  // stream-K: the tile is split over CTAs first_cta .. last_cta; one of them (the finisher) adds the FP32
+  // partial accumulators of the others to its own, in CTA order, and runs the element-wise epilogue.
   const long long first_unit = static_cast<long long>(sg.tile) * nkb;
   const int first_cta = static_cast<int>(first_unit / a.units_per_cta);
   const int last_cta = static_cast<int>((first_unit + nkb - 1) / a.units_per_cta);
   const int n_seg = last_cta - first_cta + 1;
+  const int mine = static_cast<int>(blockIdx.x) - first_cta;
   float* slot = a.partial_ws + static_cast<size_t>(sg.tile + blockIdx.x) * (ACC_COLS * kTcBM);
+  int* claimed = a.tile_counters + 2 * sg.tile;  // CTAs that have reached their epilogue of this tile
+  int* parked = claimed + 1;                     // CTAs whose partial is complete in the workspace
 
-  // Adds the parked partials of segments [s_begin, n_seg) for chunk c0 in slot order; the loads of up to
-  // four segments are in flight together (one L2 round trip instead of one per segment).
-  auto add_partials = [&](int s_begin, int c0, float (&v)[CW], float (&v2)[CW]) {
-    constexpr int PB = CW == 16 ? 4 : 1;  // segments whose loads are in flight together
-    for (int s0 = s_begin; s0 < n_seg; s0 += PB) {
+  // Adds the parked partials of segments [s_begin, s_end) for chunk c0, in order; the loads of up to four
+  // segments are in flight together (one L2 round trip instead of one per segment).
+  auto add_partials = [&](int s_begin, int s_end, int c0, float (&v)[CW], float (&v2)[CW]) {
+    constexpr int PB = CW == 16 ? 4 : 1;
+    for (int s0 = s_begin; s0 < s_end; s0 += PB) {
       float p[PB][CW], p2[PB][CW];
 #pragma unroll
       for (int u = 0; u < PB; ++u) {
-        const bool on = s0 + u < n_seg;
+        const bool on = s0 + u < s_end;
         const float* src = a.partial_ws + static_cast<size_t>(sg.tile + first_cta + (on ? s0 + u : s_begin)) * (ACC_COLS * kTcBM);
 #pragma unroll
         for (int c = 0; c < CW; ++c) {
@@ -400,98 +404,91 @@ __device__ __forceinline__ void tc_epilogue_segment(const TcGemmArgs& a, const T
       }
     }
   };
-  auto scale_cols = [&](int c0, float (&v)[CW], float (&v2)[CW]) {
-    if (col_scale != nullptr) {
-#pragma unroll
-      for (int c = 0; c < CW; ++c) {
-        v[c] *= col_scale[c0 + c];
-        if (NA == 2) v2[c] *= col_scale[c0 + c];
-      }
-    }
-  };
 
-  if (a.static_finisher && sg.kb0 == 0) {
-    // Cooperative launch: the head of a tile is the LAST segment its CTA works on, while every other
-    // segment of the tile is the FIRST one of another CTA, parked long ago.  The head CTA therefore
-    // finishes the tile from its own accumulator plus the parked partials, without parking its own.
-    if (ethread == 0) {
-      const uint64_t t0 = global_ns();
-      uint32_t polls = 0;
-      int ok = 1;
-      for (;;) {
-        int seen;
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.tile_counters + sg.tile) : "memory");
-        if (seen >= n_seg - 1) break;
-        if ((++polls & 0xffu) == 0u && global_ns() - t0 > kWaitLimitNs) {
-          if (a.status != nullptr) *reinterpret_cast<volatile int*>(a.status) = kErrTimeout;
-          ok = 0;
-          break;
-        }
-      }
-      *flag = ok;
-    }
-    epi_bar();
-    if (a.dbg && blockIdx.x == 0 && ethread == 0) a.dbg[0] = global_ns();
-    const bool ok = *reinterpret_cast<volatile int*>(flag) != 0;
-#pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += CW) {
-      float v[CW], v2[CW];
-      tc_load_acc<CW>(acc + c0, v);
-      if (NA == 2) tc_load_acc<CW>(acc + BN + c0, v2);
-      if (c0 + CW >= BN) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tempty);
-      }
-      if (a.dbg && blockIdx.x == 0 && ethread == 0) a.dbg[1] = global_ns();
-      if (ok) {
-        add_partials(1, c0, v, v2);
-        if (a.dbg && blockIdx.x == 0 && ethread == 0) a.dbg[2] = global_ns();
-        scale_cols(c0, v, v2);
-        tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
-        if (a.dbg && blockIdx.x == 0 && ethread == 0) a.dbg[3] = global_ns();
-      }
-    }
-    if (ethread == 0) a.tile_counters[sg.tile] = 0;  // ready for the next unit / launch
-    return;
-  }
-
-  // park the partial accumulator
-#pragma unroll 1
-  for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
-    float v[CW];
-    tc_load_acc<CW>(acc + c0, v);
-#pragma unroll
-    for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
-  }
-  tc_fence_before();
-  __syncwarp();
-  if (lane == 0) mbar_arrive(tempty);
-  __threadfence();
-  epi_bar();
+  // Who finishes?  Cooperative launch (all CTAs resident): the CTA that holds the head of the tile - the
+  // head is the LAST segment it works on, every other segment is the FIRST one of another CTA.  Ordinary
+  // launch: whoever reaches this point last (decided by an atomic claim), so nobody waits for a CTA that
+  // may not be running yet.
+  bool finisher;
   if (a.static_finisher) {
-    if (ethread == 0) atomicAdd(a.tile_counters + sg.tile, 1);  // the head CTA collects
+    finisher = sg.kb0 == 0;
+  } else {
+    if (ethread == 0) *flag = atomicAdd(claimed, 1) == n_seg - 1 ? 1 : 0;
+    epi_bar();
+    finisher = *reinterpret_cast<volatile int*>(flag) != 0;
+    epi_bar();  // flag is reused below
+  }
+
+  if (!finisher) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
+      float v[CW];
+      tc_load_acc<CW>(acc + c0, v);
+#pragma unroll
+      for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(tempty);
+    __threadfence();
+    epi_bar();
+    if (ethread == 0) atomicAdd(parked, 1);
     return;
   }
-  // ordinary launch: the last CTA of the tile to arrive reduces and finishes it
+
+  // finisher: the others have claimed before (or are known to be ahead); wait for their partials (bounded)
   if (ethread == 0) {
-    const int old = atomicAdd(a.tile_counters + sg.tile, 1);
-    *flag = (old == n_seg - 1) ? 1 : 0;
+    const uint64_t t0 = global_ns();
+    uint32_t polls = 0;
+    int ok = 1;
+    for (;;) {
+      int seen;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(parked) : "memory");
+      if (seen >= n_seg - 1) break;
+      if ((++polls & 0xffu) == 0u && global_ns() - t0 > kWaitLimitNs) {
+        if (a.status != nullptr) *reinterpret_cast<volatile int*>(a.status) = kErrTimeout;
+        ok = 0;
+        break;
+      }
+    }
+    *flag = ok;
   }
   epi_bar();
-  const bool last = *reinterpret_cast<volatile int*>(flag) != 0;
-  if (last) {
-    __threadfence();
+  const bool ok = *reinterpret_cast<volatile int*>(flag) != 0;
 #pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += CW) {
-      float v[CW], v2[CW];
+  for (int c0 = 0; c0 < BN; c0 += CW) {
+    float own[CW], own2[CW], v[CW], v2[CW];
+    tc_load_acc<CW>(acc + c0, own);
+    if (NA == 2) tc_load_acc<CW>(acc + BN + c0, own2);
+    if (c0 + CW >= BN) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty);
+    }
+    if (ok) {
+      // sum in CTA order whoever finishes: the result does not depend on arrival order
 #pragma unroll
       for (int c = 0; c < CW; ++c) v[c] = v2[c] = 0.f;
-      add_partials(0, c0, v, v2);  // slot order: the result does not depend on arrival order
-      scale_cols(c0, v, v2);
+      add_partials(0, mine, c0, v, v2);
+#pragma unroll
+      for (int c = 0; c < CW; ++c) {
+        v[c] += own[c];
+        if (NA == 2) v2[c] += own2[c];
+      }
+      add_partials(mine + 1, n_seg, c0, v, v2);
+      if (col_scale != nullptr) {
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          v[c] *= col_scale[c0 + c];
+          if (NA == 2) v2[c] *= col_scale[c0 + c];
+        }
+      }
       tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
     }
-    if (ethread == 0) a.tile_counters[sg.tile] = 0;  // ready for the next launch
+  }
+  if (ethread == 0) {  // ready for the next unit / launch
+    *claimed = 0;
+    *parked = 0;
   }
 }
 

@@ -201,7 +201,7 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     p.max_tiles = static_cast<int>(tiles);
     // one slot per (tile, CTA) pair that can occur: tiles + CTAs; a slot holds 128 rows x (2 x 64) FP32 columns
     p.splitk_ws = take((tiles + kTcMaxCtas) * static_cast<size_t>(2 * kTcDecodeMaxBN) * 128 * 4);
-    p.splitk_counters = take(tiles * 4);
+    p.splitk_counters = take(tiles * 8);
   }
   {
     const size_t parts = (static_cast<size_t>(c.hidden) + 127) / 128;
@@ -992,7 +992,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   const int n_tab = cfg->max_seq * (cfg->head_dim / 2);
   rope_table_kernel<<<(n_tab + 255) / 256, 256>>>(c->rope_cos, c->rope_sin, cfg->max_seq, cfg->head_dim / 2,
                                                   static_cast<double>(cfg->rope_base));
-  if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 4, 0) != cudaSuccess)
+  if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 8, 0) != cudaSuccess)
     return cleanup(THINFER_ECUDA);
   {
     // parameter blocks of the unified decode kernel: weight tensor maps per layer, token-operand maps
@@ -1223,7 +1223,7 @@ int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32
 namespace {
 constexpr int kNoAllocMaxRows = 16;
 constexpr int kNoAllocMaxNOut = 16384;
-constexpr size_t kNoAllocCounterBytes = 1024;             // 128 tiles x 4 bytes, rounded up
+constexpr size_t kNoAllocCounterBytes = 1024;             // 128 tiles x 2 counters x 4 bytes
 constexpr size_t kNoAllocSlotBytes = 16 * kTcBM * 4;      // 16 token columns x 128 features, FP32
 constexpr size_t kNoAllocBytes = kNoAllocCounterBytes + (kNoAllocMaxNOut / kTcBM + kTcMaxCtas) * kNoAllocSlotBytes;
 constexpr int kNoAllocMaxDevices = 64;
