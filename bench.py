@@ -36,6 +36,14 @@ SHAPE = synth.LLAMA_7B_LAYER
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def captured_traffic(key, batch):
+    """DRAM bytes per launch from the committed ncu capture (batch 16 only; None otherwise)."""
+    path = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+    if batch != 16 or not os.path.exists(path):
+        return None
+    return json.load(open(path)).get(key, {}).get("traffic_bytes")
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -343,11 +351,11 @@ def run_ours(args):
         "roofline": {"kernel": ("gemv_stream_kernel<SWIGLU>" if B == 1 else "tc_gemm_kernel<16..64, SWIGLU> stream-K")
                      + " (decode gate/up projection)", "bound": "hbm",
                      "achieved": gu_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gu_gbs / hbm_peak,
-                     "traffic": None, "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3,
+                     "traffic": captured_traffic("decode_gateup_b16", B), "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3,
                      "algorithmic_bytes": gateup_gemv_bytes(SHAPE, B)},
-        "roofline_prefill": {"kernel": "tc_gemm_kernel<SWIGLU> (prefill gate/up projection)", "bound": "tensor",
+        "roofline_prefill": {"kernel": "tc_gemm_kernel<256, SWIGLU interleaved> (prefill gate/up projection)", "bound": "tensor",
                              "achieved": gu_tflops, "peak": tc_peak, "unit": "TFLOP/s", "frac": gu_tflops / tc_peak,
-                             "traffic": None, "peak_kind": peak_kind, "avg_us": ms_pre_gu * 1e3},
+                             "traffic": captured_traffic("prefill_gateup_b16", B), "peak_kind": peak_kind, "avg_us": ms_pre_gu * 1e3},
         "e2e": {"value": world * B * GEN * e2e_steps / e2e_s, "unit": "tok/s",
                 "h2d_bytes_per_step": B * SHAPE.hidden * 2, "d2h_bytes_per_step": B * SHAPE.hidden * 2,
                 "note": "per decode step: pinned host input -> device, layer, result -> host, stream synchronised"},
