@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 def captured_traffic(key, batch):
     """DRAM bytes per launch from the committed ncu capture (batch 16 only; None otherwise)."""
-    path = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+    path = os.path.join(ROOT, "paper_2605_25655_b200", "ncu_traffic.json")
     if batch != 16 or not os.path.exists(path):
         return None
     return json.load(open(path)).get(key, {}).get("traffic_bytes")
