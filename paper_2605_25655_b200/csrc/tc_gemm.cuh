@@ -36,6 +36,10 @@ namespace thinfer {
 constexpr int kTcBM = 128;  // output features per tile
 constexpr int kTcBK = 64;   // contraction elements per stage (128 bytes)
 constexpr int kTcThreads = 192;
+#ifndef THINFER_TC_MAX_STAGES
+#define THINFER_TC_MAX_STAGES 8
+#endif
+constexpr int kTcMaxStages = THINFER_TC_MAX_STAGES;  // ring depth cap (small token tiles would allow more)
 constexpr int kTcGroup = 8;          // feature tiles per raster group (keeps a weight panel and the activations in L2)
 
 struct TcGemmArgs {
@@ -60,13 +64,11 @@ __host__ __device__ constexpr int tc_num_a(int epi) { return epi == EPI_SWIGLU ?
 __host__ __device__ constexpr int tc_stage_bytes(int bn, int epi) { return tc_num_a(epi) * kTcBM * 128 + bn * 128; }
 // epilogue staging: CW tokens x 128 features x 4 bytes
 __host__ __device__ constexpr int tc_stage_out_bytes(int bn) { return (bn >= 32 ? 32 : 16) * kTcBM * 4; }
-// Token tiles up to 64 are the decode kernels: they are sized so that two CTAs fit on one SM, which
-// lets the next kernel of the step become resident and prefetch its weights while this one finishes.
-__host__ __device__ constexpr int tc_ring_budget(int bn) {
-  return bn <= 64 ? (233472 / 2 - 1024) - tc_stage_out_bytes(bn) - 1280 : 200000;
-}
+// Kernels that allocate tensor memory run one CTA per SM on this part (the occupancy query returns 1 for
+// them whatever their register and shared-memory footprint), so the ring simply takes what one CTA can have.
+__host__ __device__ constexpr int tc_ring_budget(int bn) { return 200000 - tc_stage_out_bytes(bn) + 16384; }
 __host__ __device__ constexpr int tc_stages(int bn, int epi) {
-  return (tc_ring_budget(bn) / tc_stage_bytes(bn, epi)) > 8 ? 8 : (tc_ring_budget(bn) / tc_stage_bytes(bn, epi));
+  return (tc_ring_budget(bn) / tc_stage_bytes(bn, epi)) > kTcMaxStages ? kTcMaxStages : (tc_ring_budget(bn) / tc_stage_bytes(bn, epi));
 }
 __host__ __device__ constexpr int tc_acc_cols(int bn, int epi) { return tc_num_a(epi) * bn; }
 __host__ __device__ constexpr int tc_tmem_cols(int bn, int epi) {

@@ -484,11 +484,12 @@ void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v
   if (L.rc != THINFER_OK) return;
   CUtensorMap mq, mk, mv;
   const uint64_t d = head_dim;
-  bool ok = make_map(&mq, q, d, seq, static_cast<uint64_t>(batch) * n_q_heads, d, static_cast<uint64_t>(seq) * d, 128, 3);
+  bool ok = make_map(&mq, q, d, seq, static_cast<uint64_t>(batch) * n_q_heads, d, static_cast<uint64_t>(seq) * d,
+                     kAttnBQ, 3);
   ok = ok && make_map(&mk, k, d, seq, static_cast<uint64_t>(batch) * n_kv_heads, d, static_cast<uint64_t>(kv_stride) * d,
-                      128, 3);
+                      kAttnBK, 3);
   ok = ok && make_map(&mv, v, d, seq, static_cast<uint64_t>(batch) * n_kv_heads, d, static_cast<uint64_t>(kv_stride) * d,
-                      128, 3);
+                      kAttnBK, 3);
   if (!ok) {
     L.rc = fail(L.c, THINFER_ECUDA, "cuTensorMapEncodeTiled failed for an attention operand");
     return;
