@@ -476,7 +476,7 @@ void attn_prefill_d(Launcher& L, const CUtensorMap& mq, const CUtensorMap& mk, c
     ready = true;
   }
   const int n_qt = (a.seq_len + kAttnBQ - 1) / kAttnBQ;
-  L.go(THINFER_K_ATTN, attn_prefill_kernel<D>, dim3(n_qt, a.n_q_heads, batch), dim3(kAttnThreads), smem, mq, mk, mv, a);
+  L.go(THINFER_K_ATTN, attn_prefill_kernel<D>, dim3((n_qt + 1) / 2, a.n_q_heads, batch), dim3(kAttnThreads), smem, mq, mk, mv, a);
 }
 
 void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v, __half* out, int batch, int n_q_heads,
