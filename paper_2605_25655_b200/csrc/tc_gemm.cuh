@@ -270,7 +270,9 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
         const float* src = st32 + c * kTcBM + piece * 8;
         if (vec) {
           float x[8];
-          unpack8(__ldcg(reinterpret_cast<const uint4*>(e.resid + off)), x);  // L2: may be written earlier in the same kernel
+          unpack8(a.static_finisher ? __ldcg(reinterpret_cast<const uint4*>(e.resid + off))  // written earlier in the same kernel
+                                   : *reinterpret_cast<const uint4*>(e.resid + off),   // written by an earlier kernel: L1 is fine
+                  x);
           uint4 o;
           o.x = pack2(x[0] + src[0], x[1] + src[1]);
           o.y = pack2(x[2] + src[2], x[3] + src[3]);
@@ -407,20 +409,69 @@ __device__ __forceinline__ void tc_epilogue_segment(const TcGemmArgs& a, const T
     }
   };
 
-  // Who finishes?  Cooperative launch (all CTAs resident): the CTA that holds the head of the tile - the
-  // head is the LAST segment it works on, every other segment is the FIRST one of another CTA.  Ordinary
-  // launch: whoever reaches this point last (decided by an atomic claim), so nobody waits for a CTA that
-  // may not be running yet.
-  bool finisher;
-  if (a.static_finisher) {
-    finisher = sg.kb0 == 0;
-  } else {
-    if (ethread == 0) *flag = atomicAdd(claimed, 1) == n_seg - 1 ? 1 : 0;
+  if (!a.static_finisher) {
+    // Everybody parks its partial at once and claims a ticket while the stores drain; whoever holds the last
+    // ticket adds all slots in CTA order (its own included) once they are all marked complete.
+#pragma unroll 1
+    for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
+      float v[CW];
+      tc_load_acc<CW>(acc + c0, v);
+#pragma unroll
+      for (int c = 0; c < CW; ++c) slot[(c0 + c) * kTcBM + row] = v[c];
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(tempty);
+    int ticket = 0;
+    if (ethread == 0) ticket = atomicAdd(claimed, 1);  // travels while the other threads' fences complete
+    __threadfence();
     epi_bar();
-    finisher = *reinterpret_cast<volatile int*>(flag) != 0;
-    epi_bar();  // flag is reused below
+    if (ethread == 0) {
+      atomicAdd(parked, 1);
+      int ok = ticket == n_seg - 1 ? 1 : 0;
+      if (ok) {  // last ticket: wait (bounded) until every slot is complete
+        const uint64_t t0 = global_ns();
+        uint32_t polls = 0;
+        for (;;) {
+          int seen;
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(parked) : "memory");
+          if (seen >= n_seg) break;
+          if ((++polls & 0xffu) == 0u && global_ns() - t0 > kWaitLimitNs) {
+            if (a.status != nullptr) *reinterpret_cast<volatile int*>(a.status) = kErrTimeout;
+            ok = 0;
+            break;
+          }
+        }
+      }
+      *flag = ok;
+    }
+    epi_bar();
+    if (*reinterpret_cast<volatile int*>(flag) == 0) return;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CW) {
+      float v[CW], v2[CW];
+#pragma unroll
+      for (int c = 0; c < CW; ++c) v[c] = v2[c] = 0.f;
+      add_partials(0, n_seg, c0, v, v2);
+      if (col_scale != nullptr) {
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          v[c] *= col_scale[c0 + c];
+          if (NA == 2) v2[c] *= col_scale[c0 + c];
+        }
+      }
+      tc_emit_chunk<EPI, CW>(a, t, stage_out, row, ethread, v, v2, t.tok0 + c0);
+    }
+    if (ethread == 0) {  // ready for the next launch
+      *claimed = 0;
+      *parked = 0;
+    }
+    return;
   }
 
+  // Cooperative launch (all CTAs resident): the CTA that holds the head of the tile finishes it - the head is
+  // the LAST segment it works on, every other segment is the FIRST one of another CTA, parked long ago.
+  const bool finisher = sg.kb0 == 0;
   if (!finisher) {
 #pragma unroll 1
     for (int c0 = 0; c0 < ACC_COLS; c0 += CW) {
@@ -543,6 +594,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
   pdl_launch_dependents();
+  if (a.dbg != nullptr && threadIdx.x == 0) {
+    atomicMin(a.dbg + 10, static_cast<unsigned long long>(global_ns()));
+    if (blockIdx.x == 0) a.dbg[0] = global_ns();
+  }
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -569,6 +624,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         }
       }
       pdl_wait();
+      if (a.dbg != nullptr) {
+        atomicMin(a.dbg + 11, static_cast<unsigned long long>(global_ns()));
+        if (blockIdx.x == 0) a.dbg[1] = global_ns();
+      }
       TcSegIter it(a, n_tiles, nkb);
       TcSeg sg;
       uint32_t n = 0;  // k-blocks issued so far (ring position)
@@ -591,6 +650,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           }
           tma_load_2d(st + NA * A_BYTES, &tm_x, &full_bar[s], kb * kTcBK, t.tok0);
         }
+      }
+      if (a.dbg != nullptr) {
+        atomicMax(a.dbg + 12, static_cast<unsigned long long>(global_ns()));
+        if (blockIdx.x == 0) a.dbg[2] = global_ns();
       }
     }
   } else if (warp == 1) {
@@ -627,6 +690,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (ok) tc_commit(&tfull_bar[buf]);
         ++j;
       }
+      if (a.dbg != nullptr) atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -656,12 +720,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     while (it.next(sg)) {
       const uint32_t buf = j & 1, use = j >> 1;
       ++j;
+      const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
+      if (EPI == EPI_RESID && BN <= 64 && ethread < 2 * BN) {
+        // decode: pull the residual rows this tile may need (two 128-byte lines per token) into L1 while the
+        // weights stream, so the end-of-kernel epilogue does not pay an L2 round trip for them
+        const int r = t.tok0 + (ethread >> 1);
+        if (r < a.rows && t.feat0 + (ethread & 1) * 64 < a.n_feat[0])
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(a.e.resid + static_cast<size_t>(r) * a.e.ld_out + t.feat0 + (ethread & 1) * 64));
+      }
       if (!mbar_wait(&tfull_bar[buf], use & 1, a.status)) break;
       tc_fence_after();
-      const TcTile t = tc_tile_coords<BN, EPI>(a, sg.tile, n_ft, n_tt);
       const uint32_t acc = lane_base + buf * ACC_COLS;
+      if (a.dbg != nullptr && ethread == 0) atomicMax(a.dbg + 14, static_cast<unsigned long long>(global_ns()));
       tc_epilogue_segment<BN, EPI>(a, sg, t, acc, &tempty_bar[buf], stage_out, flag, row, ethread, lane, nkb, col_scale);
     }
+    if (a.dbg != nullptr && ethread == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));
   }
 
   tc_fence_before();

@@ -364,6 +364,11 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   a.status = L.c ? L.c->status_dev : nullptr;
   a.e = e;
   a.sumsq_in = sumsq_in;
+  if (L.c != nullptr && L.c->trace_unified && kid >= 0 && kid < 12) {
+    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id
+    cudaMemsetAsync(a.dbg + 10, 0xff, 16, L.st);  // the two minima
+    cudaMemsetAsync(a.dbg + 12, 0, 32, L.st);     // the four maxima
+  }
   a.norm_dim = k;
   a.norm_eps = norm_eps;
   if (stream_k && L.c != nullptr && rows <= kTcDecodeMaxBN) {
@@ -452,6 +457,10 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
   const int ctas = batch * (cf.n_q_heads / g);
   int splits = (2 * c->sm_count + ctas - 1) / ctas;
+  {
+    static const int forced = [] { const char* e = getenv("THINFER_ATTN_SPLITS"); return e ? atoi(e) : 0; }();
+    if (forced > 0) splits = forced;
+  }
   const int by_len = (t_len + 127) / 128;  // at least 128 keys per split
   if (splits > by_len) splits = by_len;
   if (splits > c->max_splits) splits = c->max_splits;
