@@ -135,8 +135,18 @@ int thinfer_decode_step_host(thinfer_ctx* ctx, int32_t slot, const void* host_in
                              void* host_out_primary, void* host_out_logits, void* cuda_stream);
 
 /* Bounded buffer of Section 3.4.2: marks `slot` free so that a later prefill
- * may reuse it.  Host state only; work already enqueued on the slot's KV is
- * ordered by the caller's stream. */
+ * may reuse it (until then a prefill into the slot returns THINFER_EBUSY: the
+ * back-pressure).  Pass the stream on which the slot's decode steps ran: an
+ * event recorded there makes a later prefill of the slot - on any stream -
+ * wait on the device until those steps have finished.
+ *
+ * Stage hand-off.  Prefill and decode use separate activation buffers inside
+ * `scratch`, and every prefill records an event that the slot's first decode
+ * step waits for.  A prefill of one slot and the decode steps of another slot
+ * may therefore be enqueued on two different streams and overlap on the GPU
+ * (the Prefill -> Buffer -> Decode schedule on one device).  Calls of the same
+ * stage (two prefills, or decode steps of two slots) still share buffers: keep
+ * each stage on one stream, or order them yourself. */
 int thinfer_release_slot(thinfer_ctx* ctx, int32_t slot, void* cuda_stream);
 
 /* Host queries (no device work).  *batch / *cur_len: what the slot holds (0, 0 when free). */

@@ -73,6 +73,11 @@ struct LayerMaps {
 struct Slot {
   int batch = 0, cur_len = 0;
   bool busy = false;
+  // hand-off between the stages: `ready` is recorded behind the prefill that filled the slot (decode on another
+  // stream waits for it), `freed` behind the release (a later prefill on another stream waits for it)
+  cudaEvent_t ready = nullptr, freed = nullptr;
+  cudaStream_t ready_stream = nullptr, freed_stream = nullptr;
+  bool ready_valid = false, freed_valid = false;
 };
 
 struct ProfEvent {
@@ -96,6 +101,12 @@ struct thinfer_ctx {
   __half* last = nullptr;
   float* logits = nullptr;
   int32_t* ids_out = nullptr;
+  // the decode path has its own (small) activation buffers, so that a prefill of one slot and decode steps of
+  // another may run on different streams at the same time (the two stages of the pipeline, Section 3.4.2)
+  __half *d_h = nullptr, *d_qbuf = nullptr, *d_attn = nullptr, *d_x1 = nullptr, *d_act = nullptr, *d_xa = nullptr,
+         *d_xb = nullptr;
+  float* d_logits = nullptr;
+  uint8_t *d_stage_in = nullptr, *d_stage_out = nullptr;
   float *part_o = nullptr, *part_ml = nullptr;
   float* splitk_ws = nullptr;   // stream-K partial accumulators
   int* splitk_counters = nullptr;
@@ -160,7 +171,7 @@ int validate_config(const thinfer_config* c, std::string* why) {
 struct ScratchPlan {
   size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
       splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, timeline, mega_common, mega_layers,
-      stage_in, stage_out, total;
+      stage_in, stage_out, d_h, d_qbuf, d_attn, d_x1, d_act, d_xa, d_xb, d_logits, d_stage_in, d_stage_out, total;
   int max_splits, max_tiles;
 };
 
@@ -221,6 +232,19 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
                                        : M * c.hidden * 2;
   p.stage_in = take(in_bytes);
   p.stage_out = take(out_bytes);
+  {
+    const size_t Bm = c.max_batch;
+    p.d_h = take(Bm * c.hidden * 2);
+    p.d_qbuf = take(Bm * qd * 2);
+    p.d_attn = take(Bm * qd * 2);
+    p.d_x1 = take(Bm * c.hidden * 2);
+    p.d_act = take(Bm * c.ffn * 2);
+    p.d_xa = take(Bm * c.hidden * 2);
+    p.d_xb = take(Bm * c.hidden * 2);
+    p.d_logits = take(Bm * (c.vocab > 0 ? c.vocab : 1) * 4);
+    p.d_stage_in = take(c.vocab > 0 ? Bm * 4 : Bm * c.hidden * 2);
+    p.d_stage_out = take(c.vocab > 0 ? Bm * (4 + static_cast<size_t>(c.vocab) * 4) : Bm * c.hidden * 2);
+  }
   p.total = off;
   return p;
 }
@@ -525,10 +549,10 @@ void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int 
 // ----------------------------------------------------------------------------
 // the layer sequences
 // ----------------------------------------------------------------------------
-EpiArgs qkv_epi(thinfer_ctx* c, __half* kc, __half* vc, int seq_len, int pos0) {
+EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_len, int pos0) {
   const thinfer_config& cf = c->cfg;
   EpiArgs e{};
-  e.q_out = c->qbuf;
+  e.q_out = qbuf;
   e.k_cache = kc;
   e.v_cache = vc;
   e.rope_cos = c->rope_cos;
@@ -562,7 +586,7 @@ void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __hal
   rmsnorm_rows(L, x_in, static_cast<const __half*>(w.attn_norm), c->h, rows, cf.hidden, cf.rms_eps);
   {
     const int nf[3] = {qd, kvd, kvd};
-    tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, rows, cf.hidden, nf, qkv_epi(c, kc, vc, seq, 0));
+    tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, rows, cf.hidden, nf, qkv_epi(c, c->qbuf, kc, vc, seq, 0));
   }
   attn_prefill(L, c->qbuf, kc, vc, c->attn, batch, cf.n_q_heads, cf.n_kv_heads, seq, cf.max_seq, cf.head_dim,
                c->status_dev);
@@ -610,27 +634,27 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     // its sums by 1/rms.  Only the first norm of a step still needs its own small kernel.
     const bool first_norm_folded = layer > 0;
     const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
-    if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->h, batch, cf.hidden, cf.rms_eps);
+    if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->d_h, batch, cf.hidden, cf.rms_eps);
     {
       const int nf[3] = {qd, kvd, kvd};
-      tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, first_norm_folded ? c->xg : c->h, batch, cf.hidden, nf,
-                              qkv_epi(c, kc, vc, 1, pos), true, first_norm_folded ? c->sumsq0 : nullptr, cf.rms_eps);
+      tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, first_norm_folded ? c->xg : c->d_h, batch, cf.hidden, nf,
+                              qkv_epi(c, c->d_qbuf, kc, vc, 1, pos), true, first_norm_folded ? c->sumsq0 : nullptr, cf.rms_eps);
     }
-    attn_decode(L, c, c->qbuf, kc, vc, c->attn, batch, pos + 1);
+    attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, pos + 1);
     {
       EpiArgs e{};
-      e.out = c->x1;
+      e.out = c->d_x1;
       e.resid = x_in;
       e.ld_out = cf.hidden;
       e.outg = c->x1g;
       e.gain_next = H(w.ffn_norm);
       e.sumsq = c->sumsq1;
       const int nf[3] = {cf.hidden, 0, 0};
-      tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->attn, batch, qd, nf, e, true);
+      tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->d_attn, batch, qd, nf, e, true);
     }
     {
       EpiArgs e{};
-      e.out = c->act;
+      e.out = c->d_act;
       e.ld_out = cf.ffn;
       const int nf[3] = {cf.ffn, cf.ffn, 0};
       tc_linear<EPI_SWIGLU>(L, THINFER_K_GATEUP, m.wg, m.wu, m.wu, c->x1g, batch, cf.hidden, nf, e, true, c->sumsq1,
@@ -639,7 +663,7 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     {
       EpiArgs e{};
       e.out = x_out;
-      e.resid = c->x1;
+      e.resid = c->d_x1;
       e.ld_out = cf.hidden;
       if (next_gain != nullptr) {
         e.outg = c->xg;
@@ -647,39 +671,39 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
         e.sumsq = c->sumsq0;
       }
       const int nf[3] = {cf.hidden, 0, 0};
-      tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->act, batch, cf.ffn, nf, e, true);
+      tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->d_act, batch, cf.ffn, nf, e, true);
     }
     return;
   }
   {
     const int n[3] = {qd, kvd, kvd};
     gemv<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch,
-                             H(w.attn_norm), cf.rms_eps, qkv_epi(c, kc, vc, 1, pos));
+                             H(w.attn_norm), cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos));
   }
-  attn_decode(L, c, c->qbuf, kc, vc, c->attn, batch, pos + 1);
+  attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, pos + 1);
   {
     EpiArgs e{};
-    e.out = c->x1;
+    e.out = c->d_x1;
     e.resid = x_in;
     e.ld_out = cf.hidden;
     const int n[3] = {cf.hidden, 0, 0};
-    gemv<EPI_RESID, false>(L, THINFER_K_OPROJ, H(w.wo), nullptr, nullptr, n, qd, c->attn, qd, batch, nullptr, 0.f, e);
+    gemv<EPI_RESID, false>(L, THINFER_K_OPROJ, H(w.wo), nullptr, nullptr, n, qd, c->d_attn, qd, batch, nullptr, 0.f, e);
   }
   {
     EpiArgs e{};
-    e.out = c->act;
+    e.out = c->d_act;
     e.ld_out = cf.ffn;
     const int n[3] = {cf.ffn, cf.ffn, 0};
-    gemv<EPI_SWIGLU, true>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->x1, cf.hidden, batch,
+    gemv<EPI_SWIGLU, true>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->d_x1, cf.hidden, batch,
                            H(w.ffn_norm), cf.rms_eps, e);
   }
   {
     EpiArgs e{};
     e.out = x_out;
-    e.resid = c->x1;
+    e.resid = c->d_x1;
     e.ld_out = cf.hidden;
     const int n[3] = {cf.hidden, 0, 0};
-    gemv<EPI_RESID, false>(L, THINFER_K_DOWN, H(w.w_down), nullptr, nullptr, n, cf.ffn, c->act, cf.ffn, batch, nullptr,
+    gemv<EPI_RESID, false>(L, THINFER_K_DOWN, H(w.w_down), nullptr, nullptr, n, cf.ffn, c->d_act, cf.ffn, batch, nullptr,
                            0.f, e);
   }
 }
@@ -721,14 +745,14 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
   a.eps = cf.rms_eps;
   a.x_in = x_in;
   a.x_out = x_out;
-  a.xa = c->xa;
-  a.xb = c->xb;
+  a.xa = c->d_xa;
+  a.xb = c->d_xb;
   a.xg = c->xg;
-  a.x1 = c->x1;
+  a.x1 = c->d_x1;
   a.x1g = c->x1g;
-  a.qbuf = c->qbuf;
-  a.attn = c->attn;
-  a.act = c->act;
+  a.qbuf = c->d_qbuf;
+  a.attn = c->d_attn;
+  a.act = c->d_act;
   a.sumsq0 = c->sumsq0;
   a.sumsq1 = c->sumsq1;
   a.kv_base = c->kv;
@@ -769,16 +793,18 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
 }
 
 // final RMSNorm + LM head + greedy argmax on `batch` rows of x [batch][hidden]
-void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, int32_t* ids_out, float* logits_out) {
+void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, int32_t* ids_out, float* logits_out,
+                     bool decode) {
   const thinfer_config& cf = c->cfg;
-  float* lg = logits_out != nullptr ? logits_out : c->logits;
+  float* lg = logits_out != nullptr ? logits_out : (decode ? c->d_logits : c->logits);
+  __half* hbuf = decode ? c->d_h : c->h;
   EpiArgs e{};
   e.out = lg;
   e.ld_out = cf.vocab;
   const int n[3] = {cf.vocab, 0, 0};
   if (batch >= 2) {
-    rmsnorm_rows(L, x, c->final_norm, c->h, batch, cf.hidden, cf.rms_eps);
-    tc_linear<EPI_PLAIN_F32>(L, THINFER_K_HEAD, c->map_head, c->map_head, c->map_head, c->h, batch, cf.hidden, n, e, true);
+    rmsnorm_rows(L, x, c->final_norm, hbuf, batch, cf.hidden, cf.rms_eps);
+    tc_linear<EPI_PLAIN_F32>(L, THINFER_K_HEAD, c->map_head, c->map_head, c->map_head, hbuf, batch, cf.hidden, n, e, true);
   } else {
     gemv<EPI_PLAIN_F32, true>(L, THINFER_K_HEAD, c->lm_head, nullptr, nullptr, n, cf.hidden, x, cf.hidden, batch,
                               c->final_norm, cf.rms_eps, e);
@@ -810,7 +836,7 @@ int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq,
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, gather_last_rows_kernel, dim3((batch + 7) / 8), dim3(256), 0, x, c->last, batch, seq,
          cf.hidden);
-    head_and_argmax(L, c, c->last, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits));
+    head_and_argmax(L, c, c->last, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits), false);
   }
   return L.rc;
 }
@@ -822,12 +848,12 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
   const __half* x = nullptr;
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((batch + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
-         c->embed, c->xa, batch, cf.hidden, cf.vocab);
-    x = c->xa;
+         c->embed, c->d_xa, batch, cf.hidden, cf.vocab);
+    x = c->d_xa;
   } else {
     x = static_cast<const __half*>(input);
   }
-  __half* pong[2] = {c->xb, c->xa};
+  __half* pong[2] = {c->d_xb, c->d_xa};
   if (c->launch_mode == 2 && mega_supported(c, batch)) {
     __half* dst = cf.vocab == 0 ? static_cast<__half*>(out_primary) : pong[(cf.n_layers - 1) & 1];
     layers_decode_unified(L, c, slot, x, dst, batch, pos);
@@ -839,8 +865,32 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
       x = dst;
     }
   }
-  if (cf.vocab > 0) head_and_argmax(L, c, x, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits));
+  if (cf.vocab > 0)
+    head_and_argmax(L, c, x, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits), true);
   return L.rc;
+}
+
+// Stage hand-off on the device (Section 3.4.2): a prefill waits until the slot's previous tenant has been
+// released on whatever stream that happened; the first decode step of a slot waits for the prefill that filled it.
+bool before_prefill(thinfer_ctx* c, Slot& s, cudaStream_t st) {
+  if (s.freed_valid && s.freed_stream != st && cudaStreamWaitEvent(st, s.freed, 0) != cudaSuccess) return false;
+  (void)c;
+  return true;
+}
+bool after_prefill(Slot& s, cudaStream_t st, int batch, int seq_len) {
+  s.busy = true;
+  s.batch = batch;
+  s.cur_len = seq_len;
+  s.ready_stream = st;
+  s.ready_valid = cudaEventRecord(s.ready, st) == cudaSuccess;
+  return s.ready_valid;
+}
+bool before_decode(Slot& s, cudaStream_t st) {
+  if (s.ready_valid && s.ready_stream != st) {
+    if (cudaStreamWaitEvent(st, s.ready, 0) != cudaSuccess) return false;
+    s.ready_stream = st;  // later steps on this stream are ordered by the stream itself
+  }
+  return true;
 }
 
 int check_prefill_args(thinfer_ctx* c, int slot, const void* input, int batch, int seq, void* out_primary,
@@ -935,6 +985,17 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->kv = static_cast<uint8_t*>(kv_workspace);
   c->kv_layer_bytes = kv_layer_bytes_of(*cfg);
   c->slots.assign(cfg->buf_slots, Slot{});
+  for (Slot& sl : c->slots) {
+    if (cudaEventCreateWithFlags(&sl.ready, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&sl.freed, cudaEventDisableTiming) != cudaSuccess) {
+      for (Slot& s2 : c->slots) {
+        if (s2.ready) cudaEventDestroy(s2.ready);
+        if (s2.freed) cudaEventDestroy(s2.freed);
+      }
+      delete c;
+      return THINFER_ECUDA;
+    }
+  }
 
   const ScratchPlan p = plan_scratch(*cfg);
   uint8_t* s = static_cast<uint8_t*>(scratch);
@@ -966,9 +1027,23 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->mega_layers = reinterpret_cast<MegaLayer*>(s + p.mega_layers);
   c->stage_in = s + p.stage_in;
   c->stage_out = s + p.stage_out;
+  c->d_h = reinterpret_cast<__half*>(s + p.d_h);
+  c->d_qbuf = reinterpret_cast<__half*>(s + p.d_qbuf);
+  c->d_attn = reinterpret_cast<__half*>(s + p.d_attn);
+  c->d_x1 = reinterpret_cast<__half*>(s + p.d_x1);
+  c->d_act = reinterpret_cast<__half*>(s + p.d_act);
+  c->d_xa = reinterpret_cast<__half*>(s + p.d_xa);
+  c->d_xb = reinterpret_cast<__half*>(s + p.d_xb);
+  c->d_logits = reinterpret_cast<float*>(s + p.d_logits);
+  c->d_stage_in = s + p.d_stage_in;
+  c->d_stage_out = s + p.d_stage_out;
   c->max_splits = p.max_splits;
 
   auto cleanup = [&](int code) {
+    for (Slot& sl : c->slots) {
+      if (sl.ready) cudaEventDestroy(sl.ready);
+      if (sl.freed) cudaEventDestroy(sl.freed);
+    }
     if (c->status_host) cudaFreeHost(c->status_host);
     delete c;
     return code;
@@ -1017,8 +1092,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     }
     MegaCommon mc;
     const uint64_t rows = cfg->max_batch;
-    bool mok = make_map_2d(&mc.x_qkv, c->xg, D, rows, 16) && make_map_2d(&mc.x_o, c->attn, qd, rows, 16) &&
-               make_map_2d(&mc.x_gu, c->x1g, D, rows, 16) && make_map_2d(&mc.x_down, c->act, F, rows, 16);
+    bool mok = make_map_2d(&mc.x_qkv, c->xg, D, rows, 16) && make_map_2d(&mc.x_o, c->d_attn, qd, rows, 16) &&
+               make_map_2d(&mc.x_gu, c->x1g, D, rows, 16) && make_map_2d(&mc.x_down, c->d_act, F, rows, 16);
     if (!mok) return cleanup(THINFER_ECUDA);
     if (cudaMemcpy(c->mega_layers, ml.data(), sizeof(MegaLayer) * ml.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(c->mega_common, &mc, sizeof(mc), cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -1035,11 +1110,11 @@ int thinfer_prefill(thinfer_ctx* c, int32_t slot, const void* input, int32_t bat
                     void* out_logits, void* cuda_stream) {
   int rc = check_prefill_args(c, slot, input, batch, seq_len, out_primary, out_logits);
   if (rc != THINFER_OK) return rc;
-  rc = run_prefill(c, slot, input, batch, seq_len, out_primary, out_logits, static_cast<cudaStream_t>(cuda_stream));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!before_prefill(c, c->slots[slot], st)) return fail(c, THINFER_ECUDA, "waiting for the slot's release failed");
+  rc = run_prefill(c, slot, input, batch, seq_len, out_primary, out_logits, st);
   if (rc != THINFER_OK) return rc;
-  c->slots[slot].busy = true;
-  c->slots[slot].batch = batch;
-  c->slots[slot].cur_len = seq_len;
+  if (!after_prefill(c->slots[slot], st, batch, seq_len)) return fail(c, THINFER_ECUDA, "recording the hand-off event failed");
   return THINFER_OK;
 }
 
@@ -1048,6 +1123,7 @@ int thinfer_decode_step(thinfer_ctx* c, int32_t slot, const void* input, void* o
   int rc = check_decode_args(c, slot, input, out_primary, out_logits);
   if (rc != THINFER_OK) return rc;
   Slot& s = c->slots[slot];
+  if (!before_decode(s, static_cast<cudaStream_t>(cuda_stream))) return fail(c, THINFER_ECUDA, "waiting for the prefill failed");
   rc = run_decode(c, slot, input, s.batch, s.cur_len, out_primary, out_logits, static_cast<cudaStream_t>(cuda_stream));
   if (rc != THINFER_OK) return rc;
   ++s.cur_len;
@@ -1062,6 +1138,7 @@ int thinfer_prefill_host(thinfer_ctx* c, int32_t slot, const void* host_input, i
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t rows = static_cast<size_t>(batch) * seq_len;
   const size_t in_bytes = cf.vocab > 0 ? rows * 4 : rows * cf.hidden * 2;
+  if (!before_prefill(c, c->slots[slot], st)) return fail(c, THINFER_ECUDA, "waiting for the slot's release failed");
   if (cudaMemcpyAsync(c->stage_in, host_input, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return fail(c, THINFER_ECUDA, "host-to-device copy failed");
   void* d_primary = c->stage_out;
@@ -1078,9 +1155,7 @@ int thinfer_prefill_host(thinfer_ctx* c, int32_t slot, const void* host_input, i
       e = cudaMemcpyAsync(host_out_logits, d_logits, static_cast<size_t>(batch) * cf.vocab * 4, cudaMemcpyDeviceToHost, st);
   }
   if (e != cudaSuccess) return fail(c, THINFER_ECUDA, "device-to-host copy failed");
-  c->slots[slot].busy = true;
-  c->slots[slot].batch = batch;
-  c->slots[slot].cur_len = seq_len;
+  if (!after_prefill(c->slots[slot], st, batch, seq_len)) return fail(c, THINFER_ECUDA, "recording the hand-off event failed");
   return THINFER_OK;
 }
 
@@ -1092,11 +1167,12 @@ int thinfer_decode_step_host(thinfer_ctx* c, int32_t slot, const void* host_inpu
   Slot& s = c->slots[slot];
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t in_bytes = cf.vocab > 0 ? static_cast<size_t>(s.batch) * 4 : static_cast<size_t>(s.batch) * cf.hidden * 2;
-  if (cudaMemcpyAsync(c->stage_in, host_input, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (!before_decode(s, st)) return fail(c, THINFER_ECUDA, "waiting for the prefill failed");
+  if (cudaMemcpyAsync(c->d_stage_in, host_input, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return fail(c, THINFER_ECUDA, "host-to-device copy failed");
-  void* d_primary = c->stage_out;
-  float* d_logits = reinterpret_cast<float*>(c->stage_out + static_cast<size_t>(cf.max_batch) * 4);
-  rc = run_decode(c, slot, c->stage_in, s.batch, s.cur_len, (cf.vocab == 0 || host_out_primary) ? d_primary : nullptr,
+  void* d_primary = c->d_stage_out;
+  float* d_logits = reinterpret_cast<float*>(c->d_stage_out + static_cast<size_t>(cf.max_batch) * 4);
+  rc = run_decode(c, slot, c->d_stage_in, s.batch, s.cur_len, (cf.vocab == 0 || host_out_primary) ? d_primary : nullptr,
                   (cf.vocab > 0 && host_out_logits) ? d_logits : nullptr, st);
   if (rc != THINFER_OK) return rc;
   cudaError_t e = cudaSuccess;
@@ -1112,11 +1188,18 @@ int thinfer_decode_step_host(thinfer_ctx* c, int32_t slot, const void* host_inpu
   return THINFER_OK;
 }
 
-int thinfer_release_slot(thinfer_ctx* c, int32_t slot, void* /*cuda_stream*/) {
+int thinfer_release_slot(thinfer_ctx* c, int32_t slot, void* cuda_stream) {
   if (c == nullptr) return THINFER_EINVAL;
   if (slot < 0 || slot >= c->cfg.buf_slots) return fail(c, THINFER_EINVAL, "slot %d outside [0, %d)", slot, c->cfg.buf_slots);
-  c->slots[slot] = Slot{};
-  return THINFER_OK;
+  Slot& s = c->slots[slot];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  s.busy = false;
+  s.batch = 0;
+  s.cur_len = 0;
+  s.ready_valid = false;
+  s.freed_stream = st;
+  s.freed_valid = cudaEventRecord(s.freed, st) == cudaSuccess;  // a later prefill on another stream waits for this
+  return s.freed_valid ? THINFER_OK : fail(c, THINFER_ECUDA, "recording the release event failed");
 }
 
 int thinfer_slot_state(const thinfer_ctx* c, int32_t slot, int32_t* batch, int32_t* cur_len) {
@@ -1190,6 +1273,10 @@ void thinfer_destroy(thinfer_ctx* c) {
   for (ProfEvent& e : c->prof_events) {
     cudaEventDestroy(e.beg);
     cudaEventDestroy(e.end);
+  }
+  for (Slot& sl : c->slots) {
+    if (sl.ready) cudaEventDestroy(sl.ready);
+    if (sl.freed) cudaEventDestroy(sl.freed);
   }
   if (c->status_host) cudaFreeHost(c->status_host);
   delete c;

@@ -193,8 +193,8 @@ class Context:
                                               _stream_ptr(stream)), self.h)
 
     # -- bookkeeping ----------------------------------------------------------
-    def release_slot(self, slot=0):
-        _check(lib().thinfer_release_slot(self.h, slot, None), self.h)
+    def release_slot(self, slot=0, stream=None):
+        _check(lib().thinfer_release_slot(self.h, slot, _stream_ptr(stream)), self.h)
 
     def slot_state(self, slot=0):
         b, n = C.c_int32(0), C.c_int32(0)

@@ -384,3 +384,37 @@ def test_launch_modes_agree_bit_for_bit(T, batch):
         ctx.close()
     for a, b in zip(*outs):
         np.testing.assert_array_equal(a, b)
+
+
+def test_prefill_and_decode_stages_on_two_streams(T):
+    # the Prefill -> Buffer -> Decode schedule on one device: slot 1 is being prefilled on one stream while slot 0
+    # decodes on another; the hand-off events order each slot's stages; results equal the serial run bit for bit
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 9)
+    x = torch.from_numpy(synth.hidden_states(shape, 9, (2, 3, 40))).cuda()     # two micro-batches of 3 requests
+
+    def run(two_streams):
+        ctx = _ctx(T, shape, [w], 3, 48, buf_slots=2)
+        sp = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
+        sd = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
+        torch.cuda.synchronize()
+        outs = {}
+        outs["p0"] = ctx.prefill(x[0, :, :30].contiguous(), slot=0, stream=sp)
+        outs["p1"] = ctx.prefill(x[1, :, :30].contiguous(), slot=1, stream=sp)      # runs while slot 0 decodes
+        for i in range(6):
+            outs[f"d0_{i}"] = ctx.decode_step(x[0, :, 30 + i].contiguous(), slot=0, stream=sd)
+        ctx.release_slot(0, stream=sd)
+        outs["p0b"] = ctx.prefill(x[1, :, :25].contiguous(), slot=0, stream=sp)     # waits for the release on the device
+        for i in range(4):
+            outs[f"d1_{i}"] = ctx.decode_step(x[1, :, 30 + i].contiguous(), slot=1, stream=sd)
+        outs["d0b"] = ctx.decode_step(x[1, :, 25].contiguous(), slot=0, stream=sd)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        res = {k: v.cpu().numpy() for k, v in outs.items()}
+        ctx.close()
+        return res
+
+    serial, overlapped = run(False), run(True)
+    for k in serial:
+        np.testing.assert_array_equal(serial[k], overlapped[k], err_msg=k)
