@@ -114,6 +114,20 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights,
 int thinfer_prefill(thinfer_ctx* ctx, int32_t slot, const void* input, int32_t batch, int32_t seq_len,
                     void* out_primary, void* out_logits, void* cuda_stream);
 
+/* Prefill of prompts of DIFFERENT lengths (Section 3.4.1: attention is per request, each with its own KV
+ * cache; the paper pads prompts to one length only for its experiment, Section 4.1).  `input` is laid out as
+ * for thinfer_prefill with seq_len = the padded length; seq_lens: host int32 [batch], 1 <= seq_lens[b] <=
+ * seq_len.  Rows past a request's length are padding: they are computed but mean nothing, and with vocab == 0
+ * the hidden-state output of those rows is unspecified; with vocab > 0 the logits / next ids are those of each
+ * request's own last token.  Later decode steps continue every request from its own length: the new token of
+ * request b sits at position seq_lens[b] + (decode steps so far).  The slot is full when the LONGEST request
+ * reaches max_seq.  Launch mode 2 uses the per-unit kernels for such a slot. */
+int thinfer_prefill_ragged(thinfer_ctx* ctx, int32_t slot, const void* input, int32_t batch, int32_t seq_len,
+                           const int32_t* seq_lens, void* out_primary, void* out_logits, void* cuda_stream);
+
+/* Host query: positions each request of the slot holds (lens_out: host int32 [batch of the slot]). */
+int thinfer_slot_lengths(const thinfer_ctx* ctx, int32_t slot, int32_t* lens_out);
+
 /* One decode step for every request of `slot` (Section 3.4.1, selective
  * batching: projections batched over requests, attention per request).  The
  * new token sits at position cur_len (the number of positions the slot holds);

@@ -23,6 +23,7 @@ struct AttnDecArgs {
   float* part_ml;         // [batch][n_q_heads][splits][2]   (max in log2 units, sum)
   int n_q_heads, n_kv_heads;
   int t_len;              // keys to attend: positions 0 .. t_len-1
+  const int* len_arr;     // ragged: request b attends len_arr[b] + t_len keys (nullptr: t_len for everybody)
   int t_max;
   int splits, chunk;      // chunk = keys per split
   float scale_log2;       // log2(e) / sqrt(D)
@@ -145,8 +146,9 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
   const int split = blockIdx.x, b = blockIdx.z;
   const int h0 = blockIdx.y * G;                                   // first query head of this CTA
   const int hk = h0 / (a.n_q_heads / a.n_kv_heads);
+  const int t_len = a.t_len + (a.len_arr != nullptr ? a.len_arr[b] : 0);
   const int t0 = split * a.chunk;
-  const int t1 = min(a.t_len, t0 + a.chunk);
+  const int t1 = min(t_len, t0 + a.chunk);
 
   float q[G][8];
 #pragma unroll

@@ -31,6 +31,7 @@ struct EpiArgs {
   int head_dim, n_q_heads, n_kv_heads;
   int seq_len;          // tokens per request in this call (1 in decode)
   int pos0;             // position of the first token of each request
+  const int* pos_arr;   // ragged decode: request b sits at position pos_arr[b] + pos0 (nullptr: pos0 for everybody)
   int t_max;            // KV positions per request in the cache
   // RESID only, optional (outg != nullptr): the next RMSNorm is folded into this epilogue.  Beside
   // y = resid + acc the kernel writes outg = y * gain_next (the operand the next projection reads)
@@ -46,7 +47,7 @@ struct EpiArgs {
 __device__ __forceinline__ size_t qkv_offset(const EpiArgs& e, int r, int n, int& kind, int& i_in_head, int& pos) {
   const int b = r / e.seq_len;
   const int s = r - b * e.seq_len;
-  pos = e.pos0 + s;
+  pos = e.pos0 + s + (e.pos_arr != nullptr ? e.pos_arr[b] : 0);
   if (n < e.n_q) {
     kind = 0;
     const int h = n / e.head_dim;

@@ -113,13 +113,15 @@ __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __rest
 
 // dst[b][:] = src[b][seq_len-1][:]  (the last prompt position feeds the LM head).
 __global__ void __launch_bounds__(256) gather_last_rows_kernel(const __half* __restrict__ src, __half* __restrict__ dst,
-                                                               int batch, int seq_len, int n) {
+                                                               int batch, int seq_len, int n,
+                                                               const int* __restrict__ lens) {
   pdl_launch_dependents();
   pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= batch) return;
-  const uint4* s = reinterpret_cast<const uint4*>(src + (static_cast<size_t>(row) * seq_len + seq_len - 1) * n);
+  const int last = (lens != nullptr ? lens[row] : seq_len) - 1;  // ragged prompts end at their own length
+  const uint4* s = reinterpret_cast<const uint4*>(src + (static_cast<size_t>(row) * seq_len + last) * n);
   uint4* d = reinterpret_cast<uint4*>(dst + static_cast<size_t>(row) * n);
   for (int c = lane; c < (n >> 3); c += 32) d[c] = __ldg(s + c);
 }

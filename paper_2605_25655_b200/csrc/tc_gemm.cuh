@@ -184,11 +184,15 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
         cs[c] = 1.f;
         sn[c] = 0.f;
         if (rotate && tok_base + c < a.rows) {
-          const size_t o = static_cast<size_t>(e.pos0 + s) * half + (i >> 1);
+          const int pos = e.pos0 + s + (e.pos_arr != nullptr ? e.pos_arr[b] : 0);
+          const size_t o = static_cast<size_t>(pos) * half + (i >> 1);
           cs[c] = __ldg(e.rope_cos + o);
           sn[c] = __ldg(e.rope_sin + o);
         }
-        if (++s == e.seq_len) s = 0;
+        if (++s == e.seq_len) {
+          s = 0;
+          ++b;
+        }
       }
     }
     const float sgn = (i & 1) ? 1.f : -1.f;
@@ -251,7 +255,8 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
       __half* dst;
       if (t.mat == 0) dst = e.q_out + ((static_cast<size_t>(b) * e.n_q_heads + h) * e.seq_len + s) * e.head_dim + i;
       else dst = (t.mat == 1 ? e.k_cache : e.v_cache) +
-                 ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + e.pos0 + s) * e.head_dim + i;
+                 ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + e.pos0 + s +
+                  (e.pos_arr != nullptr ? e.pos_arr[b] : 0)) * e.head_dim + i;
       *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(st16 + c * kTcBM + piece * 8);
     } else {
       const size_t off = static_cast<size_t>(r) * e.ld_out + n0;

@@ -78,6 +78,10 @@ struct Slot {
   cudaEvent_t ready = nullptr, freed = nullptr;
   cudaStream_t ready_stream = nullptr, freed_stream = nullptr;
   bool ready_valid = false, freed_valid = false;
+  // ragged prompts: request b holds lens[b] + steps positions (cur_len is then the longest request's count)
+  bool ragged = false;
+  int steps = 0;
+  std::vector<int> lens;
 };
 
 struct ProfEvent {
@@ -118,6 +122,7 @@ struct thinfer_ctx {
   unsigned int bar_base = 0;
   unsigned long long* timeline = nullptr;
   bool trace_unified = false;
+  int* slot_lens = nullptr;  // [buf_slots][max_batch] prompt lengths of ragged slots (device)
   MegaCommon* mega_common = nullptr;
   MegaLayer* mega_layers = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
@@ -171,7 +176,7 @@ int validate_config(const thinfer_config* c, std::string* why) {
 struct ScratchPlan {
   size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
       splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, timeline, mega_common, mega_layers,
-      stage_in, stage_out, d_h, d_qbuf, d_attn, d_x1, d_act, d_xa, d_xb, d_logits, d_stage_in, d_stage_out, total;
+      stage_in, stage_out, slot_lens, d_h, d_qbuf, d_attn, d_x1, d_act, d_xa, d_xb, d_logits, d_stage_in, d_stage_out, total;
   int max_splits, max_tiles;
 };
 
@@ -234,6 +239,7 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
   p.stage_out = take(out_bytes);
   {
     const size_t Bm = c.max_batch;
+    p.slot_lens = take(static_cast<size_t>(c.buf_slots) * Bm * 4);
     p.d_h = take(Bm * c.hidden * 2);
     p.d_qbuf = take(Bm * qd * 2);
     p.d_attn = take(Bm * qd * 2);
@@ -464,7 +470,7 @@ void attn_decode_d(Launcher& L, const AttnDecArgs& a, int batch, int ratio) {
 }
 
 void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc, const __half* vc, __half* out,
-                 int batch, int t_len) {
+                 int batch, int t_len, const int* len_arr = nullptr, int len_add = 0) {
   const thinfer_config& cf = c->cfg;
   AttnDecArgs a{};
   a.q = q;
@@ -475,7 +481,8 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   a.part_ml = c->part_ml;
   a.n_q_heads = cf.n_q_heads;
   a.n_kv_heads = cf.n_kv_heads;
-  a.t_len = t_len;
+  a.t_len = len_arr != nullptr ? len_add : t_len;  // ragged: per-request count = len_arr[b] + len_add
+  a.len_arr = len_arr;
   a.t_max = cf.max_seq;
   const int ratio = cf.n_q_heads / cf.n_kv_heads;
   int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
@@ -549,7 +556,8 @@ void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int 
 // ----------------------------------------------------------------------------
 // the layer sequences
 // ----------------------------------------------------------------------------
-EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_len, int pos0) {
+EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_len, int pos0,
+                const int* pos_arr = nullptr) {
   const thinfer_config& cf = c->cfg;
   EpiArgs e{};
   e.q_out = qbuf;
@@ -564,6 +572,7 @@ EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_le
   e.n_kv_heads = cf.n_kv_heads;
   e.seq_len = seq_len;
   e.pos0 = pos0;
+  e.pos_arr = pos_arr;
   e.t_max = cf.max_seq;
   return e;
 }
@@ -617,8 +626,10 @@ void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __hal
   }
 }
 
+// pos: position of the new token (uniform slots), or the number of decode steps so far when `lens` (device,
+// per-request prompt lengths of a ragged slot) is given; max_t: keys the longest request attends.
 void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half* x_in, __half* x_out, int batch,
-                  int pos) {
+                  int pos, const int* lens, int max_t) {
   const thinfer_config& cf = c->cfg;
   const thinfer_layer_weights& w = c->layers[layer];
   const int qd = cf.n_q_heads * cf.head_dim, kvd = cf.n_kv_heads * cf.head_dim;
@@ -638,9 +649,9 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     {
       const int nf[3] = {qd, kvd, kvd};
       tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, first_norm_folded ? c->xg : c->d_h, batch, cf.hidden, nf,
-                              qkv_epi(c, c->d_qbuf, kc, vc, 1, pos), true, first_norm_folded ? c->sumsq0 : nullptr, cf.rms_eps);
+                              qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens), true, first_norm_folded ? c->sumsq0 : nullptr, cf.rms_eps);
     }
-    attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, pos + 1);
+    attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, max_t, lens, pos + 1);
     {
       EpiArgs e{};
       e.out = c->d_x1;
@@ -678,9 +689,9 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
   {
     const int n[3] = {qd, kvd, kvd};
     gemv<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch,
-                             H(w.attn_norm), cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos));
+                             H(w.attn_norm), cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
   }
-  attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, pos + 1);
+  attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, max_t, lens, pos + 1);
   {
     EpiArgs e{};
     e.out = c->d_x1;
@@ -815,7 +826,7 @@ void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, in
 }
 
 int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq, void* out_primary, void* out_logits,
-                cudaStream_t st) {
+                cudaStream_t st, const int* lens_dev = nullptr) {
   const thinfer_config& cf = c->cfg;
   Launcher L{c, st};
   const int rows = batch * seq;
@@ -835,7 +846,7 @@ int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq,
   }
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, gather_last_rows_kernel, dim3((batch + 7) / 8), dim3(256), 0, x, c->last, batch, seq,
-         cf.hidden);
+         cf.hidden, lens_dev);
     head_and_argmax(L, c, c->last, batch, static_cast<int32_t*>(out_primary), static_cast<float*>(out_logits), false);
   }
   return L.rc;
@@ -854,14 +865,17 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
     x = static_cast<const __half*>(input);
   }
   __half* pong[2] = {c->d_xb, c->d_xa};
-  if (c->launch_mode == 2 && mega_supported(c, batch)) {
+  const Slot& sl = c->slots[slot];
+  const int* lens = sl.ragged ? c->slot_lens + static_cast<size_t>(slot) * cf.max_batch : nullptr;
+  const int step_pos = sl.ragged ? sl.steps : pos;  // ragged: every request adds its own prompt length on the device
+  if (c->launch_mode == 2 && mega_supported(c, batch) && !sl.ragged) {
     __half* dst = cf.vocab == 0 ? static_cast<__half*>(out_primary) : pong[(cf.n_layers - 1) & 1];
     layers_decode_unified(L, c, slot, x, dst, batch, pos);
     x = dst;
   } else {
     for (int l = 0; l < cf.n_layers; ++l) {
       __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
-      layer_decode(L, c, slot, l, x, dst, batch, pos);
+      layer_decode(L, c, slot, l, x, dst, batch, step_pos, lens, pos + 1);
       x = dst;
     }
   }
@@ -881,6 +895,7 @@ bool after_prefill(Slot& s, cudaStream_t st, int batch, int seq_len) {
   s.busy = true;
   s.batch = batch;
   s.cur_len = seq_len;
+  s.steps = 0;
   s.ready_stream = st;
   s.ready_valid = cudaEventRecord(s.ready, st) == cudaSuccess;
   return s.ready_valid;
@@ -1027,6 +1042,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->mega_layers = reinterpret_cast<MegaLayer*>(s + p.mega_layers);
   c->stage_in = s + p.stage_in;
   c->stage_out = s + p.stage_out;
+  c->slot_lens = reinterpret_cast<int*>(s + p.slot_lens);
   c->d_h = reinterpret_cast<__half*>(s + p.d_h);
   c->d_qbuf = reinterpret_cast<__half*>(s + p.d_qbuf);
   c->d_attn = reinterpret_cast<__half*>(s + p.d_attn);
@@ -1114,7 +1130,40 @@ int thinfer_prefill(thinfer_ctx* c, int32_t slot, const void* input, int32_t bat
   if (!before_prefill(c, c->slots[slot], st)) return fail(c, THINFER_ECUDA, "waiting for the slot's release failed");
   rc = run_prefill(c, slot, input, batch, seq_len, out_primary, out_logits, st);
   if (rc != THINFER_OK) return rc;
+  c->slots[slot].ragged = false;
   if (!after_prefill(c->slots[slot], st, batch, seq_len)) return fail(c, THINFER_ECUDA, "recording the hand-off event failed");
+  return THINFER_OK;
+}
+
+int thinfer_prefill_ragged(thinfer_ctx* c, int32_t slot, const void* input, int32_t batch, int32_t seq_len,
+                           const int32_t* seq_lens, void* out_primary, void* out_logits, void* cuda_stream) {
+  int rc = check_prefill_args(c, slot, input, batch, seq_len, out_primary, out_logits);
+  if (rc != THINFER_OK) return rc;
+  if (seq_lens == nullptr) return fail(c, THINFER_EINVAL, "seq_lens is NULL");
+  int longest = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (seq_lens[b] < 1 || seq_lens[b] > seq_len)
+      return fail(c, THINFER_EINVAL, "seq_lens[%d] = %d outside [1, %d]", b, seq_lens[b], seq_len);
+    if (seq_lens[b] > longest) longest = seq_lens[b];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Slot& s = c->slots[slot];
+  if (!before_prefill(c, s, st)) return fail(c, THINFER_ECUDA, "waiting for the slot's release failed");
+  s.lens.assign(seq_lens, seq_lens + batch);
+  int* lens_dev = c->slot_lens + static_cast<size_t>(slot) * c->cfg.max_batch;
+  if (cudaMemcpyAsync(lens_dev, s.lens.data(), static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return fail(c, THINFER_ECUDA, "copying the prompt lengths failed");
+  rc = run_prefill(c, slot, input, batch, seq_len, out_primary, out_logits, st, lens_dev);
+  if (rc != THINFER_OK) return rc;
+  s.ragged = true;
+  if (!after_prefill(s, st, batch, longest)) return fail(c, THINFER_ECUDA, "recording the hand-off event failed");
+  return THINFER_OK;
+}
+
+int thinfer_slot_lengths(const thinfer_ctx* c, int32_t slot, int32_t* lens_out) {
+  if (c == nullptr || lens_out == nullptr || slot < 0 || slot >= c->cfg.buf_slots) return THINFER_EINVAL;
+  const Slot& s = c->slots[slot];
+  for (int b = 0; b < s.batch; ++b) lens_out[b] = s.ragged ? s.lens[b] + s.steps : s.cur_len;
   return THINFER_OK;
 }
 
@@ -1127,6 +1176,7 @@ int thinfer_decode_step(thinfer_ctx* c, int32_t slot, const void* input, void* o
   rc = run_decode(c, slot, input, s.batch, s.cur_len, out_primary, out_logits, static_cast<cudaStream_t>(cuda_stream));
   if (rc != THINFER_OK) return rc;
   ++s.cur_len;
+  ++s.steps;
   return THINFER_OK;
 }
 
@@ -1155,6 +1205,7 @@ int thinfer_prefill_host(thinfer_ctx* c, int32_t slot, const void* host_input, i
       e = cudaMemcpyAsync(host_out_logits, d_logits, static_cast<size_t>(batch) * cf.vocab * 4, cudaMemcpyDeviceToHost, st);
   }
   if (e != cudaSuccess) return fail(c, THINFER_ECUDA, "device-to-host copy failed");
+  c->slots[slot].ragged = false;
   if (!after_prefill(c->slots[slot], st, batch, seq_len)) return fail(c, THINFER_ECUDA, "recording the hand-off event failed");
   return THINFER_OK;
 }
@@ -1185,6 +1236,7 @@ int thinfer_decode_step_host(thinfer_ctx* c, int32_t slot, const void* host_inpu
   }
   if (e != cudaSuccess) return fail(c, THINFER_ECUDA, "device-to-host copy failed");
   ++s.cur_len;
+  ++s.steps;
   return THINFER_OK;
 }
 
@@ -1196,6 +1248,8 @@ int thinfer_release_slot(thinfer_ctx* c, int32_t slot, void* cuda_stream) {
   s.busy = false;
   s.batch = 0;
   s.cur_len = 0;
+  s.ragged = false;
+  s.steps = 0;
   s.ready_valid = false;
   s.freed_stream = st;
   s.freed_valid = cudaEventRecord(s.freed, st) == cudaSuccess;  // a later prefill on another stream waits for this

@@ -19,7 +19,8 @@ ERR_NAMES = {OK: "THINFER_OK", EINVAL: "THINFER_EINVAL", EUNSUPPORTED: "THINFER_
 K_RMSNORM, K_QKV, K_ATTN, K_ATTN_COMBINE, K_OPROJ, K_GATEUP, K_DOWN, K_HEAD, K_EMBED, K_ARGMAX, K_DECODE_UNIFIED = range(11)
 
 EXPORTS = (
-    "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_decode_step",
+    "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_prefill_ragged", "thinfer_slot_lengths",
+    "thinfer_decode_step",
     "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
     "thinfer_kv_pointer", "thinfer_status", "thinfer_set_launch_mode", "thinfer_profile_select",
     "thinfer_profile_read", "thinfer_trace_unified", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
@@ -66,6 +67,8 @@ def lib():
     L.thinfer_workspace_bytes.argtypes = [C.POINTER(Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.thinfer_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
     L.thinfer_prefill.argtypes = [vp, i32, vp, i32, i32, vp, vp, vp]
+    L.thinfer_prefill_ragged.argtypes = [vp, i32, vp, i32, i32, C.POINTER(i32), vp, vp, vp]
+    L.thinfer_slot_lengths.argtypes = [vp, i32, C.POINTER(i32)]
     L.thinfer_decode_step.argtypes = [vp, i32, vp, vp, vp, vp]
     L.thinfer_prefill_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, vp]
     L.thinfer_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -164,6 +167,29 @@ class Context:
         _check(lib().thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, ids.data_ptr(),
                                      logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
         return (ids, logits) if want_logits else ids
+
+    def prefill_ragged(self, inp, seq_lens, slot=0, stream=None, want_logits=False):
+        """Prompts of different lengths, padded to inp.shape[1]; seq_lens: one length per request."""
+        torch = self.torch
+        batch, seq = int(inp.shape[0]), int(inp.shape[1])
+        lens = (C.c_int32 * batch)(*[int(v) for v in seq_lens])
+        assert inp.is_cuda and inp.is_contiguous()
+        if self.shape.vocab == 0:
+            out = torch.empty_like(inp)
+            _check(lib().thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, out.data_ptr(), None,
+                                                _stream_ptr(stream)), self.h)
+            return out
+        ids = torch.empty(batch, dtype=torch.int32, device=self.device)
+        logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        _check(lib().thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, ids.data_ptr(),
+                                            logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        return (ids, logits) if want_logits else ids
+
+    def slot_lengths(self, slot=0):
+        b, _ = self.slot_state(slot)
+        buf = (C.c_int32 * max(b, 1))()
+        _check(lib().thinfer_slot_lengths(self.h, slot, buf), self.h)
+        return list(buf)[:b]
 
     def decode_step(self, inp, slot=0, stream=None, want_logits=False, out=None):
         torch = self.torch

@@ -418,3 +418,57 @@ def test_prefill_and_decode_stages_on_two_streams(T):
     serial, overlapped = run(False), run(True)
     for k in serial:
         np.testing.assert_array_equal(serial[k], overlapped[k], err_msg=k)
+
+
+@pytest.mark.parametrize("lens,n_decode,mode", [((5, 17, 32), 4, 1), ((1, 64, 33, 7, 20), 3, 2), ((130,), 2, 1)])
+def test_ragged_prompts_layer(T, lens, n_decode, mode):
+    # prompts of different lengths in one batch: every request must equal the oracle run on that request alone
+    torch, thinfer = T
+    shape = synth.TINY
+    cfg = oracle_config(shape)
+    w = synth.layer_weights(shape, 12)
+    batch, pad = len(lens), max(lens)
+    x = synth.hidden_states(shape, 12, (batch, pad + n_decode))
+    ctx = _ctx(T, shape, [w], batch, pad + n_decode)
+    ctx.set_launch_mode(mode)
+    xd = torch.from_numpy(x).cuda()
+    out = ctx.prefill_ragged(xd[:, :pad].contiguous(), lens).cpu().numpy()
+    # decode inputs: request b consumes x[b, lens[b] + i] at step i (its own continuation)
+    dec = []
+    for i in range(n_decode):
+        step_in = np.stack([x[b, lens[b] + i] for b in range(batch)])
+        dec.append(ctx.decode_step(torch.from_numpy(step_in).cuda()).cpu().numpy())
+        assert ctx.slot_lengths(0) == [l + i + 1 for l in lens]
+    assert ctx.status() == 0
+    for b in range(batch):
+        ref, k, v = O.layer_prefill(cfg, w, x[b:b + 1, :lens[b]])
+        assert_rows_close(out[b, :lens[b]], ref[0], f"request {b} prefill ({lens[b]} tokens)")
+        kg = ctx.kv_view(0, 0, 0).cpu().numpy()[b, :, :lens[b]]
+        assert_rows_close(kg, k[0], f"request {b} K cache", max_err=6e-3)
+        for i in range(n_decode):
+            r, k, v = O.layer_decode(cfg, w, x[b:b + 1, lens[b] + i], k, v, lens[b] + i)
+            assert_rows_close(dec[i][b], r[0], f"request {b} decode step {i}")
+    ctx.close()
+
+
+def test_ragged_prompts_stack_logits(T):
+    torch, thinfer = T
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=688, n_layers=2, vocab=1000)
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, 13)
+    lens = (9, 3, 14)
+    ids = synth.token_ids(shape, 13, (3, 16))
+    ctx = _ctx(T, shape, sw["layers"], 3, 20, stack=sw)
+    nxt, logits = ctx.prefill_ragged(torch.from_numpy(ids[:, :14].copy()).cuda(), lens, want_logits=True)
+    step_ids = np.array([ids[b, lens[b]] for b in range(3)], dtype=np.int32)
+    nxt2, logits2 = ctx.decode_step(torch.from_numpy(step_ids).cuda(), want_logits=True)
+    for b in range(3):
+        ref, _, caches, _ = O.stack_prefill(cfg, sw, ids[b:b + 1, :lens[b]])
+        assert_rows_close(logits.cpu().numpy()[b:b + 1], ref, f"request {b}: logits of its own last prompt token")
+        ref2, _, _, _ = O.stack_decode(cfg, sw, ids[b:b + 1, lens[b]], caches, lens[b])
+        assert_rows_close(logits2.cpu().numpy()[b:b + 1], ref2, f"request {b}: first decode step")
+    with pytest.raises(thinfer.ThinferError) as e:
+        ctx.release_slot(0)
+        ctx.prefill_ragged(torch.from_numpy(ids[:, :14].copy()).cuda(), (9, 0, 14))
+    assert e.value.code == thinfer.EINVAL
+    ctx.close()
