@@ -200,7 +200,10 @@ int thinfer_profile_read(thinfer_ctx* ctx, int32_t* launches, float* total_ms);
  * not NULL, the area is copied to it first (synchronous copy; call after synchronising the stream):
  * entry 0 = kernel end, 1 = start, 2 = prep done, 3 = after the first grid barrier, then per layer
  * QKV done, barrier, attention done, barrier, O done, barrier, gate/up done, barrier, down done
- * (, barrier).  max_entries <= 256.  Host pointer; tracing aid, not part of the hot path. */
+ * (, barrier).  While tracing is on, the stream-K projections of the per-unit decode path also store, per
+ * thinfer_kernel_id k, in entries 16k+10 .. 16k+15: earliest CTA start, earliest pass of the dependency wait,
+ * latest load issued, latest MMA issued, latest accumulator ready, latest epilogue end.  max_entries <= 256.
+ * Host pointer; tracing aid, not part of the hot path. */
 int thinfer_trace_unified(thinfer_ctx* ctx, int32_t enable, uint64_t* host_out, int32_t max_entries);
 
 /* Number of kernels this context has launched so far (host counter). */

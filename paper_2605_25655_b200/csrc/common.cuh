@@ -160,13 +160,6 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
-// Fire-and-forget request that brings a tile into L2 only (no shared memory, no completion tracking).
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* m, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(m)),
-               "r"(x), "r"(y)
-               : "memory");
-}
-
 // ------------------------------------------------------------------ tcgen05
 // Tensor memory: 128 lanes x 512 32-bit columns per SM.  Addresses are
 // (lane << 16) | column.  A warp may touch lanes 32*(warp_id % 4) .. +31 only.

@@ -65,7 +65,6 @@ struct MegaArgs {
   unsigned int* grid_bar;  // arrival counter of the grid barriers; holds bar_base at launch
   unsigned int bar_base;
   int* status;
-  unsigned int prefetch_ahead_bytes;  // how far (per SM) the L2 prefetch walker runs ahead of the loads
   unsigned long long* timeline;  // optional trace: CTA 0 stores %globaltimer at every unit boundary
 };
 
@@ -203,89 +202,12 @@ __device__ __forceinline__ bool mega_grid_sync(const MegaArgs& a, const MegaShar
   return *sh.abort == 0;
 }
 
-// ------------------------------------------------------------------ L2 prefetch walker
-// Walks this CTA's weight tiles of ALL projections of ALL layers in the order the producer will load
-// them, and asks the TMA unit to bring them into L2 ahead of time.  The walker stays a fixed number of
-// bytes ahead of the shared-memory loads, across unit boundaries: while epilogues, stream-K fix-ups and
-// grid barriers hold the loads back, HBM keeps delivering the next unit's weights into L2, and the loads
-// that follow the barrier run at L2 speed until the lead is rebuilt.
-constexpr unsigned int kMegaPrefetchAheadBytes = 0;  // off: measured slower at every distance (64 KB .. 1 MB per SM)
-
-template <int BN, int D>
-struct MegaWalker {
-  int layer, phase, kb;
-  bool have_seg, done;
-  MegaGemm m;
-  TcSegIter it;
-  TcSeg sg;
-  __device__ MegaWalker(const MegaArgs& a) : layer(0), phase(0), kb(0), have_seg(false), done(false), it(TcGemmArgs{}, 0, 1) {
-    open(a);
-  }
-  __device__ void open(const MegaArgs& a) {
-    mega_gemm_desc<BN, D>(a, layer, phase, m);
-    it = TcSegIter(m.g, m.n_tiles, m.nkb);
-    have_seg = false;
-  }
-  // Prefetches the next tile; returns its bytes, or 0 when every unit has been walked.
-  __device__ unsigned int step(const MegaArgs& a) {
-    while (!done) {
-      if (!have_seg) {
-        if (it.next(sg)) {
-          have_seg = true;
-          kb = sg.kb0;
-        } else {
-          if (++phase == 4) {
-            phase = 0;
-            if (++layer == a.n_layers) {
-              done = true;
-              return 0;
-            }
-          }
-          open(a);
-          continue;
-        }
-      }
-      // one token tile in decode: the feature tile index is the tile index
-      int ft = sg.tile;
-      const CUtensorMap* w = m.w0;
-      if (phase == 0) {
-        if (ft >= m.g.tiles[0]) {
-          ft -= m.g.tiles[0];
-          w = m.w1;
-          if (ft >= m.g.tiles[1]) {
-            ft -= m.g.tiles[1];
-            w = m.w2;
-          }
-        }
-      }
-      tma_prefetch_l2_2d(w, kb * kTcBK, ft * kTcBM);
-      unsigned int bytes = kMegaABytes;
-      if (phase == 2) {
-        tma_prefetch_l2_2d(m.w1, kb * kTcBK, ft * kTcBM);
-        bytes += kMegaABytes;
-      }
-      if (++kb == sg.kb1) have_seg = false;
-      return bytes;
-    }
-    return 0;
-  }
-};
-
 // ------------------------------------------------------------------ producer of one projection
 template <int BN, int D, int EPI>
-__device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared& sh, int layer, int phase, uint32_t& n,
-                                             MegaWalker<BN, D>& walker, unsigned int& pf_bytes, unsigned int& ld_bytes) {
+__device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared& sh, int layer, int phase, uint32_t& n) {
   constexpr int NA = tc_num_a(EPI);
   constexpr int SLOT = kMegaABytes + BN * 128;
   constexpr uint32_t TX = SLOT;
-  auto keep_ahead = [&]() {
-    ld_bytes += kMegaABytes;
-    while (static_cast<int>(pf_bytes - ld_bytes) < static_cast<int>(a.prefetch_ahead_bytes)) {
-      const unsigned int b = walker.step(a);
-      if (b == 0) break;
-      pf_bytes += b;
-    }
-  };
   MegaGemm m;
   mega_gemm_desc<BN, D>(a, layer, phase, m);
   // A ring slot holds one weight tile and the token tile it is multiplied with; the gate and the up tile
@@ -302,7 +224,6 @@ __device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared
         const uint32_t q = n + pre;
         const int s = q % kMegaSlots;
         if (!mbar_wait(&sh.empty_bar[s], ((q / kMegaSlots) & 1) ^ 1u, a.status)) return false;
-        keep_ahead();
         mbar_expect_tx(&sh.full_bar[s], TX);
         tma_load_2d(sh.ring + s * SLOT, (NA == 2 && (u & 1)) ? m.w1 : tmw, &sh.full_bar[s], (u / NA) * kTcBK, t.feat0);
       }
@@ -324,7 +245,6 @@ __device__ __forceinline__ bool mega_produce(const MegaArgs& a, const MegaShared
       uint8_t* st = sh.ring + s * SLOT;
       if (i >= pre) {
         if (!mbar_wait(&sh.empty_bar[s], ((q / kMegaSlots) & 1) ^ 1u, a.status)) return false;
-        keep_ahead();
         mbar_expect_tx(&sh.full_bar[s], TX);
         tma_load_2d(st, (NA == 2 && (u & 1)) ? m.w1 : tmw, &sh.full_bar[s], (u / NA) * kTcBK, t.feat0);
       }
@@ -634,14 +554,12 @@ __global__ void __launch_bounds__(kMegaThreads, 1) decode_mega_kernel(const Mega
   if (warp == 0) {
     if (lane == 0) {
       uint32_t n = 0;
-      unsigned int pf_bytes = 0, ld_bytes = 0;
-      MegaWalker<BN, D> walker(a);
       bool ok = true;
       for (int l = 0; l < a.n_layers && ok; ++l) {
-        ok = mega_produce<BN, D, EPI_QKV_ROPE>(a, sh, l, 0, n, walker, pf_bytes, ld_bytes);
-        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 1, n, walker, pf_bytes, ld_bytes);
-        ok = ok && mega_produce<BN, D, EPI_SWIGLU>(a, sh, l, 2, n, walker, pf_bytes, ld_bytes);
-        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 3, n, walker, pf_bytes, ld_bytes);
+        ok = mega_produce<BN, D, EPI_QKV_ROPE>(a, sh, l, 0, n);
+        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 1, n);
+        ok = ok && mega_produce<BN, D, EPI_SWIGLU>(a, sh, l, 2, n);
+        ok = ok && mega_produce<BN, D, EPI_RESID>(a, sh, l, 3, n);
       }
     }
   } else if (warp == 1) {

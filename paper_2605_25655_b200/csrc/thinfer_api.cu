@@ -488,10 +488,6 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
   const int ctas = batch * (cf.n_q_heads / g);
   int splits = (2 * c->sm_count + ctas - 1) / ctas;
-  {
-    static const int forced = [] { const char* e = getenv("THINFER_ATTN_SPLITS"); return e ? atoi(e) : 0; }();
-    if (forced > 0) splits = forced;
-  }
   const int by_len = (t_len + 127) / 128;  // at least 128 keys per split
   if (splits > by_len) splits = by_len;
   if (splits > c->max_splits) splits = c->max_splits;
@@ -779,14 +775,6 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
   a.bar_base = c->bar_base;
   a.status = c->status_dev;
   a.timeline = c->trace_unified ? c->timeline : nullptr;
-  {
-    // debug knob: THINFER_UNIFIED_PREFETCH_KB overrides the L2 prefetch distance (0 switches it off)
-    static const long kb = [] {
-      const char* e = getenv("THINFER_UNIFIED_PREFETCH_KB");
-      return e ? atol(e) : static_cast<long>(kMegaPrefetchAheadBytes / 1024);
-    }();
-    a.prefetch_ahead_bytes = static_cast<unsigned int>(kb < 0 ? 0 : kb) * 1024u;
-  }
   const int ratio = cf.n_q_heads / cf.n_kv_heads;
   const int g = (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
   if (cf.head_dim == 128) {
