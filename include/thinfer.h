@@ -220,7 +220,10 @@ void thinfer_destroy(thinfer_ctx* ctx);
 
 /* y[rows, n_out] = x[rows, k] * w[n_out, k]^T  (Section 3.2.1).  FP16 in,
  * FP16 out (out_fp32 == 0) or FP32 out.  path 0: tcgen05 tensor-core tiles
- * (any rows); path 1: the weight-streaming GEMV (rows <= 16).  k % 8 == 0. */
+ * (any rows); path 1: the weight-streaming FMA GEMV (rows <= 16); path 2: the
+ * weight-streaming skinny GEMM on warp-level tensor-core fragments (rows <= 16),
+ * the kernel the decode projections of up to 16 requests use.  k % 8 == 0,
+ * n_out even. */
 int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32_t n_out, int32_t k,
                       int32_t out_fp32, int32_t path, void* cuda_stream);
 

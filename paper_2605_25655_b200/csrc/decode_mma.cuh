@@ -1,0 +1,383 @@
+// Weight-streaming skinny GEMM for decode with up to 16 tokens (the small-M
+// path of Section 3.2.2 with the fusion units of Section 3.3.1).  The work is
+// bandwidth-bound: every weight is read from HBM exactly once, by a 128-bit
+// load that goes straight into the register fragment of a warp-level tensor
+// core instruction (mma.sync m16n8k16, FP16 in, FP32 accumulate), so that 16
+// tokens cost no more issue slots than one.
+//
+// Decomposition.  The output features are cut into one contiguous share per
+// CTA, balanced to within one feature pair over a grid that is a multiple of
+// the SM count: no wave quantisation and no partial sums that cross CTAs.  A
+// share is at most TM tiles of 16 weight rows.  The 8 warps of a CTA take the
+// 64-element blocks of K in turn (block b belongs to warp b mod 8); for its
+// block a warp loads the token fragment once and walks all tiles of the share
+// with it, one FP32 fragment per tile in registers.  After the stream the 8
+// fragments of a tile are added in warp order through shared memory (a fixed
+// order: results do not depend on timing) and the fused epilogue runs.
+//
+// Weights travel global -> shared memory by 16-byte asynchronous copies
+// (cp.async, no registers held) into a ring that is private to each lane: a
+// lane reads back exactly the bytes it requested, so the ring needs no barrier,
+// only cp.async.wait_group.  The ring is filled before the wait on the previous
+// kernel.  The kernel uses no tensor memory, so under programmatic dependent
+// launch CTAs of the next projection can be resident beside the running ones.
+#pragma once
+#include "epilogue.cuh"
+
+namespace thinfer {
+
+constexpr int kSkWarps = 8;
+constexpr int kSkTokMax = 16;
+constexpr int kSkStages = 4;  // ring depth per warp; one stage = 16 rows x 64 elements = 2 KB
+
+struct SkinnyArgs {
+  const __half* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
+  int n[3];            // rows of each matrix (0 for unused); every count is even
+  int k;               // contraction length, multiple of 64
+  int rows;            // tokens, <= 8 * NT
+  const __half* x;     // [rows][ldx]
+  int ldx;
+  // folded RMSNorm of the token operand: sums of squares per (part, token), [sumsq_parts][sumsq_stride]
+  // (stride 16 when a skinny projection produced them, 64 when a tcgen05 projection did)
+  const float* sumsq_in;
+  int sumsq_parts;
+  int sumsq_stride;
+  int norm_dim;
+  float norm_eps;
+  int tiles_max;       // row tiles of the largest CTA share (<= TM)
+  EpiArgs e;           // RESID with outg: e.sumsq receives [gridDim.x][16]
+  unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
+};
+
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// 16 bytes global -> shared, bypassing L1; src_bytes = 0 writes zeros and reads nothing
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* gsrc, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Row r of the concatenated feature space -> address of that weight row.
+__device__ __forceinline__ const __half* sk_row_ptr(const SkinnyArgs& a, int r) {
+  int m = 0;
+  if (r >= a.n[0]) {
+    r -= a.n[0];
+    m = 1;
+    if (r >= a.n[1]) {
+      r -= a.n[1];
+      m = 2;
+    }
+  }
+  return a.w[m] + static_cast<size_t>(r) * a.k;
+}
+
+// The ring doubles as the parking area of the finished fragments (TM * NT * 128 floats per warp).
+__host__ __device__ constexpr int sk_smem_floats(int tm, int parts) {
+  return kSkWarps * kSkStages * 512 + parts * 16 + tm * 16 + 16 * 16 + 16;
+}
+
+// A "unit" is a pair of adjacent features (rows 2u, 2u+1 of the concatenated space), or for SWIGLU one
+// feature (its gate row and its up row).  A tile is 8 units = the 16 rows of one MMA:
+//   plain:  MMA row j <-> feature 2 u0 + j
+//   SWIGLU: MMA row j < 8 <-> gate row u0 + j, MMA row j + 8 <-> up row u0 + j
+// In the m16n8k16 fragment layout lane (g = lane / 4, t = lane % 4) holds rows g and g + 8 of A, token g of
+// B and the outputs (rows g, g + 8) x (tokens 2t, 2t + 1).  Which k index a register slot stands for is
+// irrelevant as long as A and B agree, so every lane simply takes 16 contiguous bytes: of a 64-element
+// block, lane t holds elements 8t..8t+7 and 32+8t..32+8t+7 of its rows and of its token.
+template <int NT, int TM, int EPI>
+__global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyArgs a) {
+  static_assert(kSkStages * 4 >= TM * NT, "the fragments of a warp are parked in its own ring");
+  pdl_launch_dependents();
+  extern __shared__ __align__(16) float sk_smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  if (a.dbg != nullptr && threadIdx.x == 0) {
+    atomicMin(a.dbg + 10, static_cast<unsigned long long>(global_ns()));  // earliest CTA start
+    atomicMax(a.dbg + 12, static_cast<unsigned long long>(global_ns()));  // latest CTA start
+  }
+  const int units = (EPI == EPI_SWIGLU) ? a.n[0] : (a.n[0] + a.n[1] + a.n[2]) >> 1;
+  const int u_beg = static_cast<int>(static_cast<long long>(blockIdx.x) * units / gridDim.x);
+  const int u_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * units / gridDim.x);
+  const int n_tiles = (u_end - u_beg + 7) >> 3;  // <= TM; the walk below always takes TM tiles, empty ones cost no traffic
+  const int nkb = a.k >> 6;                       // k is a multiple of 64 (checked on the host)
+  const int nkw = (nkb - warp + kSkWarps - 1) / kSkWarps;  // blocks warp, warp + 8, ...
+
+  uint4* ring = reinterpret_cast<uint4*>(sk_smem) + warp * (kSkStages * 128);  // [stage][4 chunks][32 lanes]
+  float* part = sk_smem;                                                       // after the stream: [warp][TM][nt][4][32]
+  float* ssq_in = sk_smem + kSkWarps * kSkStages * 512;                        // [parts][16]
+  float* ssq_tile = ssq_in + a.sumsq_parts * 16;                               // [tile][16]
+  float* red = ssq_tile + TM * 16;                                             // [16][16]
+  float* rstd = red + 256;                                                     // [16]
+
+  // Weight rows of this lane for every tile of the share (row g and row g + 8 of the tile), already at
+  // this lane's first element of block `warp`.  A row outside the share keeps a valid address and a
+  // copy size of zero: the copy then writes zeros and reads nothing.
+  const __half* pa[TM];
+  const __half* pb[TM];
+  uint32_t sza[TM], szb[TM];
+  const size_t lane_off = static_cast<size_t>(warp) * 64 + t * 8;
+#pragma unroll
+  for (int tile = 0; tile < TM; ++tile) {
+    const int u0 = u_beg + tile * 8;
+    if (EPI == EPI_SWIGLU) {
+      const bool ok = u0 + g < u_end;
+      pa[tile] = (ok ? a.w[0] + static_cast<size_t>(u0 + g) * a.k : a.w[0]) + lane_off;
+      pb[tile] = (ok ? a.w[1] + static_cast<size_t>(u0 + g) * a.k : a.w[0]) + lane_off;
+      sza[tile] = szb[tile] = ok ? 16u : 0u;
+    } else {
+      const int ra = 2 * u0 + g, rb = ra + 8;
+      const bool oka = ra < 2 * u_end, okb = rb < 2 * u_end;
+      pa[tile] = (oka ? sk_row_ptr(a, ra) : a.w[0]) + lane_off;
+      pb[tile] = (okb ? sk_row_ptr(a, rb) : a.w[0]) + lane_off;
+      sza[tile] = oka ? 16u : 0u;
+      szb[tile] = okb ? 16u : 0u;
+    }
+  }
+  // requests this warp's block number `blk` (k offset blk * 512 elements from block `warp`) of tile `tile`
+  // into a ring stage: chunk 0/1 = row g, elements 8t.. / 32+8t..; chunk 2/3 = row g + 8
+  const uint32_t ring_lane = smem_u32(ring + lane);
+  auto request = [&](int tile, int blk, int stage) {
+    const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
+    const uint32_t dst = ring_lane + stage * 2048;
+    cp_async_16(dst, pa[tile] + off, sza[tile]);
+    cp_async_16(dst + 512, pa[tile] + off + 32, sza[tile]);
+    cp_async_16(dst + 1024, pb[tile] + off, szb[tile]);
+    cp_async_16(dst + 1536, pb[tile] + off + 32, szb[tile]);
+  };
+
+  // Pair number j = blk * TM + tile lives in stage j mod kSkStages and is requested kSkStages pairs ahead
+  // of its use.  The weights do not depend on the previous kernel: the ring is filled before the wait.
+#pragma unroll
+  for (int j = 0; j < kSkStages; ++j) {
+    if (j / TM < nkw) request(j % TM, j / TM, j);
+    cp_async_commit();
+  }
+  pdl_wait();
+  if (a.dbg != nullptr && threadIdx.x == 0) atomicMin(a.dbg + 11, static_cast<unsigned long long>(global_ns()));
+
+  if (a.sumsq_in != nullptr) {
+    // asynchronous copies straight into shared memory: no registers held, consumed after the stream
+    // (they join whichever group is committed next; the final wait covers them)
+    for (int i = threadIdx.x; i < a.sumsq_parts * 16; i += kSkWarps * 32)
+      cp_async_4(ssq_in + i, a.sumsq_in + (i >> 4) * a.sumsq_stride + (i & 15));
+  }
+
+  // token fragments: XB buffers, requested XB - 1 blocks ahead (the fewer tiles a block has, the further)
+  constexpr int XB = TM == 1 ? 4 : (TM <= 3 ? 3 : 2);
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  const __half* xrow[NT];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+    xrow[nt] = (nt * 8 + g < a.rows) ? a.x + static_cast<size_t>(nt * 8 + g) * a.ldx + lane_off : nullptr;
+  uint4 xq[XB][NT][2];
+  auto load_x = [&](int blk, uint4 (&x)[NT][2]) {
+    const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      x[nt][0] = xrow[nt] != nullptr ? ldg_cached(xrow[nt] + off) : zero;
+      x[nt][1] = xrow[nt] != nullptr ? ldg_cached(xrow[nt] + off + 32) : zero;
+    }
+  };
+#pragma unroll
+  for (int b = 0; b < XB - 1; ++b)
+    if (b < nkw) load_x(b, xq[b]);
+
+  float acc[TM][NT][4];
+#pragma unroll
+  for (int tile = 0; tile < TM; ++tile)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[tile][nt][i] = 0.f;
+
+  int stage = 0;
+  for (int i0 = 0; i0 < nkw; i0 += XB) {
+#pragma unroll
+    for (int b = 0; b < XB; ++b) {
+      const int i = i0 + b;
+      if (i < nkw) {
+        if (i + XB - 1 < nkw) load_x(i + XB - 1, xq[(b + XB - 1) % XB]);
+#pragma unroll
+        for (int tile = 0; tile < TM; ++tile) {
+          // one group per pair, kSkStages pairs ahead: all but the newest kSkStages - 1 groups are complete
+          cp_async_wait_group<kSkStages - 1>();
+          const uint4* src = ring + stage * 128 + lane;
+          const uint4 a0 = src[0], a1 = src[32], b0 = src[64], b1 = src[96];
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            mma_16816(acc[tile][nt], a0.x, b0.x, a0.y, b0.y, xq[b][nt][0].x, xq[b][nt][0].y);
+            mma_16816(acc[tile][nt], a0.z, b0.z, a0.w, b0.w, xq[b][nt][0].z, xq[b][nt][0].w);
+            mma_16816(acc[tile][nt], a1.x, b1.x, a1.y, b1.y, xq[b][nt][1].x, xq[b][nt][1].y);
+            mma_16816(acc[tile][nt], a1.z, b1.z, a1.w, b1.w, xq[b][nt][1].z, xq[b][nt][1].w);
+          }
+          // the stage just read is free again (the same lane wrote and read it: program order is enough);
+          // it receives the pair kSkStages ahead
+          const int t2 = (tile + kSkStages) % TM, db = (tile + kSkStages) / TM;  // constants once unrolled
+          if (i + db < nkw) request(t2, i + db, stage);
+          cp_async_commit();
+          if (++stage == kSkStages) stage = 0;
+        }
+      }
+    }
+  }
+  cp_async_wait_all();
+  __syncwarp();
+  if (a.dbg != nullptr && lane == 0) atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // stream end
+  // park the fragments in this warp's own ring
+  {
+    float* dst = part + static_cast<size_t>(warp) * (kSkStages * 512) + lane;
+#pragma unroll
+    for (int tile = 0; tile < TM; ++tile)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[(tile * NT + nt) * 128 + i * 32] = acc[tile][nt][i];
+  }
+  __syncthreads();
+  if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 14, static_cast<unsigned long long>(global_ns()));
+
+  // ---- 1/rms per token from the producer's per-part sums (fixed order)
+  if (a.sumsq_in != nullptr) {
+    const int tok = threadIdx.x & 15, sl = threadIdx.x >> 4;  // 16 slices of parts
+    float s = 0.f;
+    for (int p = sl; p < a.sumsq_parts; p += 16) s += ssq_in[p * 16 + tok];
+    red[sl * 16 + tok] = s;
+    __syncthreads();
+    if (threadIdx.x < 16) {
+      float tot = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) tot += red[j * 16 + threadIdx.x];
+      rstd[threadIdx.x] = rsqrtf(tot / static_cast<float>(a.norm_dim) + a.norm_eps);
+    }
+    __syncthreads();
+  }
+
+  // ---- K slices added in warp order, then the fused epilogue; one (tile, token tile) per warp at a time
+  const EpiArgs& e = a.e;
+  for (int item = warp; item < n_tiles * NT; item += kSkWarps) {
+    const int tile = item / NT, nt = item - tile * NT;
+    float c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      c[i] = 0.f;
+    }
+#pragma unroll
+    for (int w = 0; w < kSkWarps; ++w) {
+      const float* src = part + static_cast<size_t>(w) * (kSkStages * 512) + (tile * NT + nt) * 128 + lane;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[i] += src[i * 32];
+    }
+    const int u0 = u_beg + tile * 8;
+    const int ta = nt * 8 + 2 * t, tb = ta + 1;
+    if (a.sumsq_in != nullptr) {
+      const float sa = rstd[ta], sb = rstd[tb];
+      c[0] *= sa;
+      c[1] *= sb;
+      c[2] *= sa;
+      c[3] *= sb;
+    }
+    if (EPI == EPI_SWIGLU) {
+      const int f = u0 + g;
+      if (f < u_end) {
+        __half* o = reinterpret_cast<__half*>(e.out);
+        if (ta < a.rows) o[static_cast<size_t>(ta) * e.ld_out + f] = __float2half_rn(silu_f(c[0]) * c[2]);
+        if (tb < a.rows) o[static_cast<size_t>(tb) * e.ld_out + f] = __float2half_rn(silu_f(c[1]) * c[3]);
+      }
+    } else if (EPI == EPI_QKV_ROPE) {
+      // rows g and g + 8 have the parity of g; the other half of a rotation pair sits in lane ^ 4
+      const float sgn = (g & 1) ? 1.f : -1.f;
+#pragma unroll
+      for (int hr = 0; hr < 2; ++hr) {
+        const int row = 2 * u0 + g + 8 * hr;
+        const bool row_ok = row < 2 * u_end;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int tok = ta + j;
+          const float val = c[hr * 2 + j];
+          const float partner = __shfl_xor_sync(0xffffffffu, val, 4);
+          float y = val;
+          int kind = 0, i = 0, pos = 0;
+          size_t off = 0;
+          const bool ok = row_ok && tok < a.rows;
+          if (ok) {
+            off = qkv_offset(e, tok, row, kind, i, pos);
+            if (kind != 2) {
+              const size_t o = static_cast<size_t>(pos) * (e.head_dim >> 1) + (i >> 1);
+              y = fmaf(sgn * partner, __ldg(e.rope_sin + o), val * __ldg(e.rope_cos + o));
+            }
+          }
+          const float y_odd = __shfl_xor_sync(0xffffffffu, y, 4);
+          if (ok && !(g & 1)) {
+            __half* dst = (kind == 0) ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
+            *reinterpret_cast<uint32_t*>(dst + off) = pack2(y, y_odd);
+          }
+        }
+      }
+    } else {
+      float sq[2] = {0.f, 0.f};
+#pragma unroll
+      for (int hr = 0; hr < 2; ++hr) {
+        const int row = 2 * u0 + g + 8 * hr;
+        if (row < 2 * u_end) {
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const int tok = ta + j;
+            if (tok >= a.rows) continue;
+            const size_t off = static_cast<size_t>(tok) * e.ld_out + row;
+            const float v = c[hr * 2 + j];
+            if (EPI == EPI_PLAIN_F32) {
+              reinterpret_cast<float*>(e.out)[off] = v;
+            } else if (EPI == EPI_PLAIN_F16) {
+              reinterpret_cast<__half*>(e.out)[off] = __float2half_rn(v);
+            } else {  // EPI_RESID
+              const __half yh = __float2half_rn(__half2float(e.resid[off]) + v);
+              reinterpret_cast<__half*>(e.out)[off] = yh;
+              if (e.outg != nullptr) {  // folded RMSNorm of the next sub-layer (gain here, 1/rms there)
+                const float y = __half2float(yh);
+                e.outg[off] = __float2half_rn(y * __half2float(e.gain_next[row]));
+                sq[j] = fmaf(y, y, sq[j]);
+              }
+            }
+          }
+        }
+      }
+      if (EPI == EPI_RESID && e.outg != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          sq[j] += __shfl_xor_sync(0xffffffffu, sq[j], 4);
+          sq[j] += __shfl_xor_sync(0xffffffffu, sq[j], 8);
+          sq[j] += __shfl_xor_sync(0xffffffffu, sq[j], 16);
+        }
+        if (g == 0) {
+          ssq_tile[tile * 16 + ta] = sq[0];
+          ssq_tile[tile * 16 + tb] = sq[1];
+        }
+      }
+    }
+  }
+  if (EPI == EPI_RESID && e.outg != nullptr) {
+    __syncthreads();
+    if (threadIdx.x < 16) {
+      float s = 0.f;
+      if (NT * 8 > threadIdx.x)
+        for (int tile = 0; tile < n_tiles; ++tile) s += ssq_tile[tile * 16 + threadIdx.x];
+      e.sumsq[blockIdx.x * 16 + threadIdx.x] = s;
+    }
+  }
+  if (a.dbg != nullptr && lane == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));
+}
+
+}  // namespace thinfer

@@ -16,6 +16,7 @@
 #include "decode_attn.cuh"
 #include "decode_gemv.cuh"
 #include "decode_mega.cuh"
+#include "decode_mma.cuh"
 #include "misc_kernels.cuh"
 #include "prefill_attn.cuh"
 #include "tc_gemm.cuh"
@@ -117,6 +118,8 @@ struct thinfer_ctx {
   // unified decode kernel
   __half *xg = nullptr, *x1g = nullptr;
   float *sumsq0 = nullptr, *sumsq1 = nullptr, *attn_partial = nullptr;
+  int sumsq0_parts = 0, sumsq1_parts = 0;  // parts the last skinny down / O projection left in sumsq0 / sumsq1
+  bool skinny_ok = true;    // hidden, ffn and the head widths suit the skinny decode projections
   int* attn_counters = nullptr;
   unsigned int* grid_bar = nullptr;
   unsigned int bar_base = 0;
@@ -182,6 +185,7 @@ struct ScratchPlan {
 
 constexpr int kTcMaxCtas = 160;      // persistent grid bound (a B200 has 148 SMs)
 constexpr int kTcDecodeMaxBN = 64;   // token tile of the stream-K decode path
+constexpr int kSkMaxCtas = 2 * kTcMaxCtas;  // grid bound of the skinny decode projections that produce sums of squares
 
 ScratchPlan plan_scratch(const thinfer_config& c) {
   ScratchPlan p{};
@@ -223,8 +227,10 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     const size_t parts = (static_cast<size_t>(c.hidden) + 127) / 128;
     p.xg = take(static_cast<size_t>(c.max_batch) * c.hidden * 2);
     p.x1g = take(static_cast<size_t>(c.max_batch) * c.hidden * 2);
-    p.sumsq0 = take(parts * 64 * 4);
-    p.sumsq1 = take(parts * 64 * 4);
+    // [128-feature tile][64 tokens] (tcgen05 producers) or [CTA][16 tokens] (skinny producers, <= 2 CTAs per SM)
+    const size_t ssq = std::max<size_t>(parts * 64 * 4, static_cast<size_t>(kSkMaxCtas) * 16 * 4);
+    p.sumsq0 = take(ssq);
+    p.sumsq1 = take(ssq);
     p.attn_partial = take((static_cast<size_t>(c.max_batch) * c.n_q_heads + kTcMaxCtas * 4) * (c.head_dim + 2) * 4);
     p.attn_counters = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * 4);
     p.grid_bar = take(64);
@@ -450,6 +456,79 @@ void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half
 }
 
 // ----------------------------------------------------------------------------
+// skinny tensor-core streaming dispatch (decode, <= 16 tokens)
+// ----------------------------------------------------------------------------
+constexpr int kSkMaxTiles = 5;  // 16-row tiles per CTA share the kernels are instantiated for (1 .. 5)
+
+int skinny_grid(thinfer_ctx* c, int units) {
+  // two CTAs per SM, more when a share would exceed kSkMaxTiles tiles; never less than one full tile per CTA
+  const int sms = c ? c->sm_count : 148;
+  int g = 2 * sms;
+  while ((units + g - 1) / g > 8 * kSkMaxTiles) g += sms;
+  const int by_work = units / 8 > 0 ? units / 8 : 1;
+  return g < by_work ? g : by_work;
+}
+
+template <int NT, int TM, int EPI>
+void launch_skinny_tm(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
+  static int reserved = 0;  // per instantiation; contexts are created from one thread at a time
+  const int smem = sk_smem_floats(TM, a.sumsq_parts) * 4;
+  if (smem > reserved) {
+    if (smem > 200 * 1024 || !opt_in_smem(skinny_mma_kernel<NT, TM, EPI>, smem)) {
+      L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection needs %d bytes of shared memory", smem);
+      return;
+    }
+    reserved = smem;
+  }
+  L.go(kid, skinny_mma_kernel<NT, TM, EPI>, dim3(grid), dim3(kSkWarps * 32), smem, a);
+}
+
+template <int NT, int EPI>
+void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
+  switch (a.tiles_max) {
+    case 1: launch_skinny_tm<NT, 1, EPI>(L, kid, grid, a); break;
+    case 2: launch_skinny_tm<NT, 2, EPI>(L, kid, grid, a); break;
+    case 3: launch_skinny_tm<NT, 3, EPI>(L, kid, grid, a); break;
+    case 4: launch_skinny_tm<NT, 4, EPI>(L, kid, grid, a); break;
+    default: launch_skinny_tm<NT, 5, EPI>(L, kid, grid, a); break;
+  }
+}
+
+// Returns the grid size: a RESID producer leaves one sum-of-squares part per CTA.
+template <int EPI>
+int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
+           const __half* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, int sumsq_stride, float eps,
+           const EpiArgs& e) {
+  if (L.rc != THINFER_OK) return 0;
+  SkinnyArgs a{};
+  a.w[0] = w0;
+  a.w[1] = w1;
+  a.w[2] = w2;
+  for (int i = 0; i < 3; ++i) a.n[i] = n[i];
+  a.k = k;
+  a.rows = rows;
+  a.x = x;
+  a.ldx = ldx;
+  a.sumsq_in = sumsq_in;
+  a.sumsq_parts = sumsq_in != nullptr ? sumsq_parts : 0;
+  a.sumsq_stride = sumsq_stride;
+  a.norm_dim = k;
+  a.norm_eps = eps;
+  a.e = e;
+  if (L.c != nullptr && L.c->trace_unified && kid >= 0 && kid < 12) {
+    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id
+    cudaMemsetAsync(a.dbg + 10, 0xff, 16, L.st);  // the two minima
+    cudaMemsetAsync(a.dbg + 12, 0, 32, L.st);     // the four maxima
+  }
+  const int units = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
+  const int grid = skinny_grid(L.c, units);
+  a.tiles_max = ((units + grid - 1) / grid + 7) / 8;
+  if (rows <= 8) launch_skinny<1, EPI>(L, kid, grid, a);
+  else launch_skinny<2, EPI>(L, kid, grid, a);
+  return grid;
+}
+
+// ----------------------------------------------------------------------------
 // attention dispatch
 // ----------------------------------------------------------------------------
 template <int D>
@@ -632,6 +711,82 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
   __half* kc = kv_ptr(c, slot, layer, 0);
   __half* vc = kv_ptr(c, slot, layer, 1);
   auto H = [](const void* p) { return static_cast<const __half*>(p); };
+  if (batch <= kSkTokMax && c->skinny_ok) {
+    // Up to 16 tokens.  The wide projections (QKV, gate/up: many output features per SM) run as balanced
+    // weight streams into warp-level tensor-core fragments, with no partial sums across CTAs; the two
+    // projections with few output features and a long contraction (O, down) split K across the SMs on the
+    // tcgen05 stream-K path, which is the faster of the two for them.
+    // The RMSNorm in front of a projection is folded into the projection before it (gain there, 1/rms here).
+    const LayerMaps& m = c->maps[layer];
+    const bool first_norm_folded = layer > 0;
+    const int parts = (cf.hidden + kTcBM - 1) / kTcBM;  // the tcgen05 producers leave one sum per 128-feature tile
+    const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
+    if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->d_h, batch, cf.hidden, cf.rms_eps);
+    {
+      const int n[3] = {qd, kvd, kvd};
+      skinny<EPI_QKV_ROPE>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, first_norm_folded ? c->xg : c->d_h,
+                           cf.hidden, batch, first_norm_folded ? c->sumsq0 : nullptr, batch >= 2 ? parts : c->sumsq0_parts,
+                           batch >= 2 ? 64 : 16, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
+    }
+    attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, max_t, lens, pos + 1);
+    if (batch >= 2) {
+      EpiArgs e{};
+      e.out = c->d_x1;
+      e.resid = x_in;
+      e.ld_out = cf.hidden;
+      e.outg = c->x1g;
+      e.gain_next = H(w.ffn_norm);
+      e.sumsq = c->sumsq1;
+      const int nf[3] = {cf.hidden, 0, 0};
+      tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->d_attn, batch, qd, nf, e, true);
+    } else {
+      EpiArgs e{};
+      e.out = c->d_x1;
+      e.resid = x_in;
+      e.ld_out = cf.hidden;
+      e.outg = c->x1g;
+      e.gain_next = H(w.ffn_norm);
+      e.sumsq = c->sumsq1;
+      const int n[3] = {cf.hidden, 0, 0};
+      c->sumsq1_parts = skinny<EPI_RESID>(L, THINFER_K_OPROJ, H(w.wo), nullptr, nullptr, n, qd, c->d_attn, qd, batch,
+                                          nullptr, 0, 16, 0.f, e);
+    }
+    {
+      EpiArgs e{};
+      e.out = c->d_act;
+      e.ld_out = cf.ffn;
+      const int n[3] = {cf.ffn, cf.ffn, 0};
+      skinny<EPI_SWIGLU>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->x1g, cf.hidden, batch,
+                         c->sumsq1, batch >= 2 ? parts : c->sumsq1_parts, batch >= 2 ? 64 : 16, cf.rms_eps, e);
+    }
+    if (batch >= 2) {
+      EpiArgs e{};
+      e.out = x_out;
+      e.resid = c->d_x1;
+      e.ld_out = cf.hidden;
+      if (next_gain != nullptr) {
+        e.outg = c->xg;
+        e.gain_next = next_gain;
+        e.sumsq = c->sumsq0;
+      }
+      const int nf[3] = {cf.hidden, 0, 0};
+      tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->d_act, batch, cf.ffn, nf, e, true);
+    } else {
+      EpiArgs e{};
+      e.out = x_out;
+      e.resid = c->d_x1;
+      e.ld_out = cf.hidden;
+      if (next_gain != nullptr) {
+        e.outg = c->xg;
+        e.gain_next = next_gain;
+        e.sumsq = c->sumsq0;
+      }
+      const int n[3] = {cf.hidden, 0, 0};
+      c->sumsq0_parts = skinny<EPI_RESID>(L, THINFER_K_DOWN, H(w.w_down), nullptr, nullptr, n, cf.ffn, c->d_act, cf.ffn,
+                                          batch, nullptr, 0, 16, 0.f, e);
+    }
+    return;
+  }
   if (batch >= 2) {
     // batched decode: the weight stream feeds the tensor cores (stream-K over all SMs); plain FMA
     // cannot keep up with HBM beyond a couple of tokens per weight
@@ -981,6 +1136,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   thinfer_ctx* c = new thinfer_ctx();
   c->cfg = *cfg;
   c->sm_count = prop.multiProcessorCount;
+  c->skinny_ok = cfg->hidden % 64 == 0 && cfg->ffn % 64 == 0 && (cfg->n_q_heads * cfg->head_dim) % 64 == 0;
   c->layers.assign(weights->layers, weights->layers + cfg->n_layers);
   c->embed = static_cast<const __half*>(weights->embed);
   c->final_norm = static_cast<const __half*>(weights->final_norm);
@@ -1342,6 +1498,14 @@ int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32
     else
       gemv<EPI_PLAIN_F16, false>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k,
                                  static_cast<const __half*>(x), k, rows, nullptr, 0.f, e);
+  } else if (path == 2) {
+    if (rows > kSkTokMax || k % 64 != 0) return THINFER_EUNSUPPORTED;
+    if (out_fp32)
+      skinny<EPI_PLAIN_F32>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
+                            rows, nullptr, 0, 16, 0.f, e);
+    else
+      skinny<EPI_PLAIN_F16>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
+                            rows, nullptr, 0, 16, 0.f, e);
   } else if (path == 0) {
     CUtensorMap mw;
     if (!make_map_2d(&mw, w, k, n_out, 128)) return THINFER_ECUDA;

@@ -49,13 +49,40 @@ def test_linear_streaming_path(T, rows, n_out, k):
         assert_rows_close(y.cpu().numpy(), O.linear(x, w), f"linear gemv {rows}x{n_out}x{k}", max_err=4e-3)
 
 
+# K is a multiple of 64 here.  Covered: fewer features than one 16-row tile per CTA share, K shorter than
+# the 8 warp slices, block counts that do not divide by 8, shares of 1 .. 5 tiles, 9..16 tokens (two token
+# tiles), the 7B projection shapes and a vocabulary-sized output
+@pytest.mark.parametrize("rows,n_out,k", [(1, 256, 256), (2, 130, 64), (3, 1376, 704), (4, 4096, 4096), (7, 256, 11008),
+                                          (16, 512, 1024), (9, 12288, 4096), (16, 4096, 11008), (13, 2, 64),
+                                          (8, 6, 192), (16, 32000, 512), (5, 9472, 320), (11, 18944, 128),
+                                          (16, 22016, 4096)])
+def test_linear_skinny_tensor_core_path(T, rows, n_out, k):
+    torch, thinfer = T
+    rng = np.random.default_rng(rows * 13 + k)
+    x, w = _rand16(rng, (rows, k), 1.0), _rand16(rng, (n_out, k), 0.05)
+    for fp32 in (False, True):
+        y = thinfer.op_linear(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda(), out_fp32=fp32, path=2)
+        torch.cuda.synchronize()
+        assert_rows_close(y.cpu().numpy(), O.linear(x, w), f"linear skinny {rows}x{n_out}x{k}", max_err=4e-3)
+
+
+def test_linear_skinny_rejects_what_it_does_not_cover(T):
+    torch, thinfer = T
+    x = torch.zeros(17, 64, dtype=torch.float16, device="cuda")
+    w = torch.zeros(8, 64, dtype=torch.float16, device="cuda")
+    with pytest.raises(thinfer.ThinferError):
+        thinfer.op_linear(x, w, path=2)            # more than 16 tokens
+    with pytest.raises(thinfer.ThinferError):
+        thinfer.op_linear(x[:4, :40].contiguous(), w[:, :40].contiguous(), path=2)  # K not a multiple of 64
+
+
 def test_linear_identity_weight_is_exact(T):
     torch, thinfer = T
     rng = np.random.default_rng(5)
     x = _rand16(rng, (40, 192), 1.0)
     w = np.eye(192, dtype=np.float16)
-    for path in (0, 1):
-        xs = x[:16] if path == 1 else x
+    for path in (0, 1, 2):
+        xs = x[:16] if path >= 1 else x
         y = thinfer.op_linear(torch.from_numpy(xs).cuda(), torch.from_numpy(w).cuda(), path=path)
         np.testing.assert_array_equal(y.cpu().numpy(), xs)
 
