@@ -28,7 +28,7 @@ namespace thinfer {
 
 constexpr int kSkWarps = 8;
 constexpr int kSkTokMax = 16;
-constexpr int kSkStages = 4;  // ring depth per warp; one stage = 16 rows x 64 elements = 2 KB
+// ring depth per warp is the template parameter ST; one stage = 16 rows x 64 elements = 2 KB
 
 struct SkinnyArgs {
   const __half* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
@@ -44,6 +44,10 @@ struct SkinnyArgs {
   int sumsq_stride;
   int norm_dim;
   float norm_eps;
+  // NORM kernels instead take the raw rows in x and the gain here: RMSNorm as a prologue.  Every CTA reads
+  // all of x anyway, so the sums of squares come from the token fragments it already holds, the gain is
+  // multiplied in (FP16, the rounding of a stored normalised operand) and 1/rms scales the finished sums.
+  const __half* gamma;
   int tiles_max;       // row tiles of the largest CTA share (<= TM)
   EpiArgs e;           // RESID with outg: e.sumsq receives [gridDim.x][16]
   unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
@@ -66,6 +70,16 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait_group() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
+// element-wise FP16 product of two groups of 8 halves
+__device__ __forceinline__ uint4 hmul2x4(const uint4& a, const uint4& b) {
+  uint4 r;
+  const __half2* pa = reinterpret_cast<const __half2*>(&a);
+  const __half2* pb = reinterpret_cast<const __half2*>(&b);
+  __half2* pr = reinterpret_cast<__half2*>(&r);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) pr[i] = __hmul2(pa[i], pb[i]);
+  return r;
+}
 __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
 }
@@ -86,21 +100,21 @@ __device__ __forceinline__ const __half* sk_row_ptr(const SkinnyArgs& a, int r) 
 }
 
 // The ring doubles as the parking area of the finished fragments (TM * NT * 128 floats per warp).
-__host__ __device__ constexpr int sk_smem_floats(int tm, int parts) {
-  return kSkWarps * kSkStages * 512 + parts * 16 + tm * 16 + 16 * 16 + 16;
+__host__ __device__ constexpr int sk_smem_floats(int tm, int stages, int parts) {
+  return kSkWarps * stages * 512 + parts * 16 + tm * 16 + 16 * 16 + 16;
 }
 
-// A "unit" is a pair of adjacent features (rows 2u, 2u+1 of the concatenated space), or for SWIGLU one
-// feature (its gate row and its up row).  A tile is 8 units = the 16 rows of one MMA:
-//   plain:  MMA row j <-> feature 2 u0 + j
-//   SWIGLU: MMA row j < 8 <-> gate row u0 + j, MMA row j + 8 <-> up row u0 + j
+// A "unit" of the partition is a pair of adjacent features (rows 2u, 2u+1 of the concatenated space), or
+// for SWIGLU one feature (its gate row and its up row).  A tile is the 16 rows of one MMA:
+//   plain:  MMA row j <-> row (tile start) + j
+//   SWIGLU: MMA row j < 8 <-> gate row (tile start) + j, MMA row j + 8 <-> up row (tile start) + j
 // In the m16n8k16 fragment layout lane (g = lane / 4, t = lane % 4) holds rows g and g + 8 of A, token g of
 // B and the outputs (rows g, g + 8) x (tokens 2t, 2t + 1).  Which k index a register slot stands for is
 // irrelevant as long as A and B agree, so every lane simply takes 16 contiguous bytes: of a 64-element
 // block, lane t holds elements 8t..8t+7 and 32+8t..32+8t+7 of its rows and of its token.
-template <int NT, int TM, int EPI>
-__global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyArgs a) {
-  static_assert(kSkStages * 4 >= TM * NT, "the fragments of a warp are parked in its own ring");
+template <int NT, int TM, int ST, int EPI, bool NORM = false>
+__global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_kernel(const SkinnyArgs a) {
+  static_assert(ST * 4 >= TM * NT, "the fragments of a warp are parked in its own ring");
   pdl_launch_dependents();
   extern __shared__ __align__(16) float sk_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -111,57 +125,68 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
   const int units = (EPI == EPI_SWIGLU) ? a.n[0] : (a.n[0] + a.n[1] + a.n[2]) >> 1;
   const int u_beg = static_cast<int>(static_cast<long long>(blockIdx.x) * units / gridDim.x);
   const int u_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * units / gridDim.x);
-  const int n_tiles = (u_end - u_beg + 7) >> 3;  // <= TM; the walk below always takes TM tiles, empty ones cost no traffic
-  const int nkb = a.k >> 6;                       // k is a multiple of 64 (checked on the host)
-  const int nkw = (nkb - warp + kSkWarps - 1) / kSkWarps;  // blocks warp, warp + 8, ...
+  // Rows of the share in tile coordinates.  SWIGLU: "row" = feature, a tile holds 8 features (8 gate rows
+  // and 8 up rows).  Otherwise a tile holds 16 rows.  Tiles start at the share, except when several
+  // matrices are concatenated (QKV): there a tile starts at a multiple of 16 rows, so that no tile lies
+  // across two matrices (their row counts are multiples of 16), and the first and the last tile of a share
+  // may be partial.  Rows outside [r_lo, r_hi) cost no traffic.
+  constexpr int TR = (EPI == EPI_SWIGLU) ? 8 : 16;  // share rows per tile
+  const int r_lo = (EPI == EPI_SWIGLU) ? u_beg : 2 * u_beg;
+  const int r_hi = (EPI == EPI_SWIGLU) ? u_end : 2 * u_end;
+  const int row00 = (EPI == EPI_SWIGLU || a.n[1] == 0) ? r_lo : (r_lo & ~15);  // first row of tile 0
+  const int n_tiles = r_hi > r_lo ? (r_hi - row00 + TR - 1) / TR : 0;  // <= TM; the walk always takes TM tiles
+  const int nkb = a.k >> 6;                                  // k is a multiple of 64 (checked on the host)
+  const int nkw = (nkb - warp + kSkWarps - 1) / kSkWarps;    // blocks warp, warp + 8, ...
 
-  uint4* ring = reinterpret_cast<uint4*>(sk_smem) + warp * (kSkStages * 128);  // [stage][4 chunks][32 lanes]
-  float* part = sk_smem;                                                       // after the stream: [warp][TM][nt][4][32]
-  float* ssq_in = sk_smem + kSkWarps * kSkStages * 512;                        // [parts][16]
-  float* ssq_tile = ssq_in + a.sumsq_parts * 16;                               // [tile][16]
-  float* red = ssq_tile + TM * 16;                                             // [16][16]
-  float* rstd = red + 256;                                                     // [16]
+  uint4* ring = reinterpret_cast<uint4*>(sk_smem) + warp * (ST * 128);  // [stage][16 rows][8 chunks]
+  float* part = sk_smem;                                                // after the stream: [warp][TM][nt][4][32]
+  float* ssq_in = sk_smem + kSkWarps * ST * 512;                        // [parts][16]
+  float* ssq_tile = ssq_in + a.sumsq_parts * 16;                        // [tile][16]
+  float* red = ssq_tile + TM * 16;                                      // [16][16]
+  float* rstd = red + 256;                                              // [16]
 
-  // Weight rows of this lane for every tile of the share (row g and row g + 8 of the tile), already at
-  // this lane's first element of block `warp`.  A row outside the share keeps a valid address and a
-  // copy size of zero: the copy then writes zeros and reads nothing.
-  const __half* pa[TM];
-  const __half* pb[TM];
-  uint32_t sza[TM], szb[TM];
-  const size_t lane_off = static_cast<size_t>(warp) * 64 + t * 8;
+  // The warp copies a (tile, block) pair cooperatively, 4 rows x 128 contiguous bytes per instruction: lane
+  // l takes 16-byte chunk l % 8 of tile row l / 8 + 4 j in instruction j.  A stage is row-major
+  // [16][128 B] with chunk c of row r at position c ^ 4 (r & 1): the copies and the fragment reads (row g,
+  // chunks t and 4 + t) are both free of bank conflicts.  A row outside the share keeps a computable
+  // address and a copy size of zero: the copy then writes zeros and reads nothing.
+  const int crow = lane >> 3, cchunk = lane & 7;
+  const uint32_t coop_dst = smem_u32(ring) + crow * 128 + ((cchunk ^ ((crow & 1) << 2)) << 4);
+  const size_t coop_off = static_cast<size_t>(warp) * 64 + cchunk * 8;
+  const int lim_lo = r_lo - row00 - crow, lim_hi = r_hi - row00 - crow;  // tile row TR*tile + 4j (+crow) is in the share
+                                                                         // iff lim_lo <= TR*tile + 4j < lim_hi
+  const __half* tb[TM];  // plain: row crow of the tile, at this lane's chunk of block `warp`
+  if (EPI != EPI_SWIGLU) {
+    const int last = a.n[0] + a.n[1] + a.n[2] - 1;
 #pragma unroll
-  for (int tile = 0; tile < TM; ++tile) {
-    const int u0 = u_beg + tile * 8;
-    if (EPI == EPI_SWIGLU) {
-      const bool ok = u0 + g < u_end;
-      pa[tile] = (ok ? a.w[0] + static_cast<size_t>(u0 + g) * a.k : a.w[0]) + lane_off;
-      pb[tile] = (ok ? a.w[1] + static_cast<size_t>(u0 + g) * a.k : a.w[0]) + lane_off;
-      sza[tile] = szb[tile] = ok ? 16u : 0u;
-    } else {
-      const int ra = 2 * u0 + g, rb = ra + 8;
-      const bool oka = ra < 2 * u_end, okb = rb < 2 * u_end;
-      pa[tile] = (oka ? sk_row_ptr(a, ra) : a.w[0]) + lane_off;
-      pb[tile] = (okb ? sk_row_ptr(a, rb) : a.w[0]) + lane_off;
-      sza[tile] = oka ? 16u : 0u;
-      szb[tile] = okb ? 16u : 0u;
-    }
+    for (int tile = 0; tile < TM; ++tile) tb[tile] = sk_row_ptr(a, min(row00 + tile * 16 + crow, last)) + coop_off;
   }
-  // requests this warp's block number `blk` (k offset blk * 512 elements from block `warp`) of tile `tile`
-  // into a ring stage: chunk 0/1 = row g, elements 8t.. / 32+8t..; chunk 2/3 = row g + 8
-  const uint32_t ring_lane = smem_u32(ring + lane);
   auto request = [&](int tile, int blk, int stage) {
     const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
-    const uint32_t dst = ring_lane + stage * 2048;
-    cp_async_16(dst, pa[tile] + off, sza[tile]);
-    cp_async_16(dst + 512, pa[tile] + off + 32, sza[tile]);
-    cp_async_16(dst + 1024, pb[tile] + off, szb[tile]);
-    cp_async_16(dst + 1536, pb[tile] + off + 32, szb[tile]);
+    const uint32_t dst = coop_dst + stage * 2048;
+    if (EPI == EPI_SWIGLU) {
+      const size_t row0 = static_cast<size_t>(r_lo + tile * 8 + crow) * a.k + coop_off + off;
+      const uint32_t s0 = tile * 8 < lim_hi ? 16u : 0u, s1 = tile * 8 + 4 < lim_hi ? 16u : 0u;
+      const size_t o0 = s0 ? row0 : 0, o1 = s1 ? row0 + static_cast<size_t>(4) * a.k : 0;
+      cp_async_16(dst, a.w[0] + o0, s0);
+      cp_async_16(dst + 512, a.w[0] + o1, s1);
+      cp_async_16(dst + 1024, a.w[1] + o0, s0);
+      cp_async_16(dst + 1536, a.w[1] + o1, s1);
+    } else {
+      const __half* src = tb[tile] + off;
+      const size_t k4 = static_cast<size_t>(4) * a.k;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool ok = tile * 16 + 4 * j >= lim_lo && tile * 16 + 4 * j < lim_hi;
+        cp_async_16(dst + 512 * j, ok ? src + j * k4 : a.w[0], ok ? 16u : 0u);
+      }
+    }
   };
 
-  // Pair number j = blk * TM + tile lives in stage j mod kSkStages and is requested kSkStages pairs ahead
-  // of its use.  The weights do not depend on the previous kernel: the ring is filled before the wait.
+  // Pair number j = blk * TM + tile lives in stage j mod ST and is requested ST pairs ahead of its use.
+  // The weights do not depend on the previous kernel: the ring is filled before the wait.
 #pragma unroll
-  for (int j = 0; j < kSkStages; ++j) {
+  for (int j = 0; j < ST; ++j) {
     if (j / TM < nkw) request(j % TM, j / TM, j);
     cp_async_commit();
   }
@@ -181,7 +206,8 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
   const __half* xrow[NT];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt)
-    xrow[nt] = (nt * 8 + g < a.rows) ? a.x + static_cast<size_t>(nt * 8 + g) * a.ldx + lane_off : nullptr;
+    xrow[nt] = (nt * 8 + g < a.rows) ? a.x + static_cast<size_t>(nt * 8 + g) * a.ldx + static_cast<size_t>(warp) * 64 + t * 8
+                                     : nullptr;
   uint4 xq[XB][NT][2];
   auto load_x = [&](int blk, uint4 (&x)[NT][2]) {
     const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
@@ -203,19 +229,49 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[tile][nt][i] = 0.f;
 
+  float ssx[NT];  // NORM: this lane's share of the sum of squares of token nt * 8 + g
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) ssx[nt] = 0.f;
+  const __half* grow = NORM ? a.gamma + static_cast<size_t>(warp) * 64 + t * 8 : nullptr;
+
   int stage = 0;
+  const int frag0 = g * 8 + (t ^ ((g & 1) << 2));  // row g, chunk t (chunk 4 + t: position ^ 4; row g + 8: + 64)
   for (int i0 = 0; i0 < nkw; i0 += XB) {
 #pragma unroll
     for (int b = 0; b < XB; ++b) {
       const int i = i0 + b;
       if (i < nkw) {
         if (i + XB - 1 < nkw) load_x(i + XB - 1, xq[(b + XB - 1) % XB]);
+        if (NORM) {
+          const size_t off = static_cast<size_t>(i) * (kSkWarps * 64);
+          const uint4 g0 = ldg_cached(grow + off), g1 = ldg_cached(grow + off + 32);
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            float f[8];
+            unpack8(xq[b][nt][0], f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ssx[nt] = fmaf(f[j], f[j], ssx[nt]);
+            unpack8(xq[b][nt][1], f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ssx[nt] = fmaf(f[j], f[j], ssx[nt]);
+            xq[b][nt][0] = hmul2x4(xq[b][nt][0], g0);
+            xq[b][nt][1] = hmul2x4(xq[b][nt][1], g1);
+          }
+        }
 #pragma unroll
         for (int tile = 0; tile < TM; ++tile) {
-          // one group per pair, kSkStages pairs ahead: all but the newest kSkStages - 1 groups are complete
-          cp_async_wait_group<kSkStages - 1>();
-          const uint4* src = ring + stage * 128 + lane;
-          const uint4 a0 = src[0], a1 = src[32], b0 = src[64], b1 = src[96];
+          // one group per pair, ST pairs ahead: all but the newest ST - 1 groups are complete.  Lanes read
+          // what other lanes copied: a warp barrier on both sides of the reads.
+          cp_async_wait_group<ST - 1>();
+          __syncwarp();
+          const uint4* src = ring + stage * 128;
+          const uint4 a0 = src[frag0], a1 = src[frag0 ^ 4], b0 = src[64 + frag0], b1 = src[64 + (frag0 ^ 4)];
+          __syncwarp();
+          // the stage is free again; it receives the pair ST ahead
+          const int t2 = (tile + ST) % TM, db = (tile + ST) / TM;  // constants once unrolled
+          if (i + db < nkw) request(t2, i + db, stage);
+          cp_async_commit();
+          if (++stage == ST) stage = 0;
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             mma_16816(acc[tile][nt], a0.x, b0.x, a0.y, b0.y, xq[b][nt][0].x, xq[b][nt][0].y);
@@ -223,12 +279,6 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
             mma_16816(acc[tile][nt], a1.x, b1.x, a1.y, b1.y, xq[b][nt][1].x, xq[b][nt][1].y);
             mma_16816(acc[tile][nt], a1.z, b1.z, a1.w, b1.w, xq[b][nt][1].z, xq[b][nt][1].w);
           }
-          // the stage just read is free again (the same lane wrote and read it: program order is enough);
-          // it receives the pair kSkStages ahead
-          const int t2 = (tile + kSkStages) % TM, db = (tile + kSkStages) / TM;  // constants once unrolled
-          if (i + db < nkw) request(t2, i + db, stage);
-          cp_async_commit();
-          if (++stage == kSkStages) stage = 0;
         }
       }
     }
@@ -238,7 +288,7 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
   if (a.dbg != nullptr && lane == 0) atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // stream end
   // park the fragments in this warp's own ring
   {
-    float* dst = part + static_cast<size_t>(warp) * (kSkStages * 512) + lane;
+    float* dst = part + static_cast<size_t>(warp) * (ST * 512) + lane;
 #pragma unroll
     for (int tile = 0; tile < TM; ++tile)
 #pragma unroll
@@ -246,8 +296,28 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
 #pragma unroll
         for (int i = 0; i < 4; ++i) dst[(tile * NT + nt) * 128 + i * 32] = acc[tile][nt][i];
   }
+  if (NORM) {
+    // lanes t = 0..3 of a token hold disjoint parts of K; warps hold disjoint blocks
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      ssx[nt] += __shfl_xor_sync(0xffffffffu, ssx[nt], 1);
+      ssx[nt] += __shfl_xor_sync(0xffffffffu, ssx[nt], 2);
+      if (t == 0) red[warp * 16 + nt * 8 + g] = ssx[nt];
+    }
+  }
   __syncthreads();
   if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 14, static_cast<unsigned long long>(global_ns()));
+  if (NORM) {
+    if (threadIdx.x < 16) {
+      float tot = 0.f;
+      if (threadIdx.x < NT * 8) {
+#pragma unroll
+        for (int w = 0; w < kSkWarps; ++w) tot += red[w * 16 + threadIdx.x];
+      }
+      rstd[threadIdx.x] = rsqrtf(tot / static_cast<float>(a.k) + a.norm_eps);
+    }
+    __syncthreads();
+  }
 
   // ---- 1/rms per token from the producer's per-part sums (fixed order)
   if (a.sumsq_in != nullptr) {
@@ -276,13 +346,13 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
     }
 #pragma unroll
     for (int w = 0; w < kSkWarps; ++w) {
-      const float* src = part + static_cast<size_t>(w) * (kSkStages * 512) + (tile * NT + nt) * 128 + lane;
+      const float* src = part + static_cast<size_t>(w) * (ST * 512) + (tile * NT + nt) * 128 + lane;
 #pragma unroll
       for (int i = 0; i < 4; ++i) c[i] += src[i * 32];
     }
-    const int u0 = u_beg + tile * 8;
+    const int row0 = row00 + tile * TR;  // first share row of the tile
     const int ta = nt * 8 + 2 * t, tb = ta + 1;
-    if (a.sumsq_in != nullptr) {
+    if (NORM || a.sumsq_in != nullptr) {
       const float sa = rstd[ta], sb = rstd[tb];
       c[0] *= sa;
       c[1] *= sb;
@@ -290,8 +360,8 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
       c[3] *= sb;
     }
     if (EPI == EPI_SWIGLU) {
-      const int f = u0 + g;
-      if (f < u_end) {
+      const int f = row0 + g;
+      if (f < r_hi) {
         __half* o = reinterpret_cast<__half*>(e.out);
         if (ta < a.rows) o[static_cast<size_t>(ta) * e.ld_out + f] = __float2half_rn(silu_f(c[0]) * c[2]);
         if (tb < a.rows) o[static_cast<size_t>(tb) * e.ld_out + f] = __float2half_rn(silu_f(c[1]) * c[3]);
@@ -301,8 +371,8 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
       const float sgn = (g & 1) ? 1.f : -1.f;
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
-        const int row = 2 * u0 + g + 8 * hr;
-        const bool row_ok = row < 2 * u_end;
+        const int row = row0 + g + 8 * hr;
+        const bool row_ok = row >= r_lo && row < r_hi;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           const int tok = ta + j;
@@ -330,8 +400,8 @@ __global__ void __launch_bounds__(kSkWarps * 32) skinny_mma_kernel(const SkinnyA
       float sq[2] = {0.f, 0.f};
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
-        const int row = 2 * u0 + g + 8 * hr;
-        if (row < 2 * u_end) {
+        const int row = row0 + g + 8 * hr;
+        if (row >= r_lo && row < r_hi) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const int tok = ta + j;

@@ -401,9 +401,7 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   a.e = e;
   a.sumsq_in = sumsq_in;
   if (L.c != nullptr && L.c->trace_unified && kid >= 0 && kid < 12) {
-    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id
-    cudaMemsetAsync(a.dbg + 10, 0xff, 16, L.st);  // the two minima
-    cudaMemsetAsync(a.dbg + 12, 0, 32, L.st);     // the four maxima
+    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id, reset at the start of the step
   }
   a.norm_dim = k;
   a.norm_eps = norm_eps;
@@ -460,45 +458,55 @@ void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half
 // ----------------------------------------------------------------------------
 constexpr int kSkMaxTiles = 5;  // 16-row tiles per CTA share the kernels are instantiated for (1 .. 5)
 
-int skinny_grid(thinfer_ctx* c, int units) {
-  // two CTAs per SM, more when a share would exceed kSkMaxTiles tiles; never less than one full tile per CTA
-  const int sms = c ? c->sm_count : 148;
-  int g = 2 * sms;
-  while ((units + g - 1) / g > 8 * kSkMaxTiles) g += sms;
-  const int by_work = units / 8 > 0 ? units / 8 : 1;
-  return g < by_work ? g : by_work;
+// Largest number of tiles a CTA share touches (mirrors the kernel's tile rule).
+int skinny_tiles_max(int units, int grid, bool swiglu, bool concatenated) {
+  int worst = 0;
+  for (int cta = 0; cta < grid; ++cta) {
+    const int ub = static_cast<int>(static_cast<long long>(cta) * units / grid);
+    const int ue = static_cast<int>(static_cast<long long>(cta + 1) * units / grid);
+    if (ue <= ub) continue;
+    const int lo = swiglu ? ub : 2 * ub, hi = swiglu ? ue : 2 * ue, tr = swiglu ? 8 : 16;
+    const int r0 = (swiglu || !concatenated) ? lo : (lo & ~15);
+    worst = std::max(worst, (hi - r0 + tr - 1) / tr);
+  }
+  return worst;
 }
 
-template <int NT, int TM, int EPI>
+template <int NT, int TM, int ST, int EPI, bool NORM>
 void launch_skinny_tm(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
   static int reserved = 0;  // per instantiation; contexts are created from one thread at a time
-  const int smem = sk_smem_floats(TM, a.sumsq_parts) * 4;
+  const int smem = sk_smem_floats(TM, ST, a.sumsq_parts) * 4;
   if (smem > reserved) {
-    if (smem > 200 * 1024 || !opt_in_smem(skinny_mma_kernel<NT, TM, EPI>, smem)) {
+    if (smem > 220 * 1024 || !opt_in_smem(skinny_mma_kernel<NT, TM, ST, EPI, NORM>, smem)) {
       L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection needs %d bytes of shared memory", smem);
       return;
     }
     reserved = smem;
   }
-  L.go(kid, skinny_mma_kernel<NT, TM, EPI>, dim3(grid), dim3(kSkWarps * 32), smem, a);
+  L.go(kid, skinny_mma_kernel<NT, TM, ST, EPI, NORM>, dim3(grid), dim3(kSkWarps * 32), smem, a);
 }
 
-template <int NT, int EPI>
-void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
+template <int NT, int EPI, bool NORM>
+void launch_skinny(Launcher& L, int kid, int grid, bool deep, const SkinnyArgs& a) {
+  if (deep) {  // one CTA per SM, an 8-stage ring: half of a 4096-long contraction is requested before the wait
+    if (a.tiles_max <= 1) launch_skinny_tm<NT, 1, 8, EPI, NORM>(L, kid, grid, a);
+    else launch_skinny_tm<NT, 2, 8, EPI, NORM>(L, kid, grid, a);
+    return;
+  }
   switch (a.tiles_max) {
-    case 1: launch_skinny_tm<NT, 1, EPI>(L, kid, grid, a); break;
-    case 2: launch_skinny_tm<NT, 2, EPI>(L, kid, grid, a); break;
-    case 3: launch_skinny_tm<NT, 3, EPI>(L, kid, grid, a); break;
-    case 4: launch_skinny_tm<NT, 4, EPI>(L, kid, grid, a); break;
-    default: launch_skinny_tm<NT, 5, EPI>(L, kid, grid, a); break;
+    case 1: launch_skinny_tm<NT, 1, 4, EPI, NORM>(L, kid, grid, a); break;
+    case 2: launch_skinny_tm<NT, 2, 4, EPI, NORM>(L, kid, grid, a); break;
+    case 3: launch_skinny_tm<NT, 3, 4, EPI, NORM>(L, kid, grid, a); break;
+    case 4: launch_skinny_tm<NT, 4, 4, EPI, NORM>(L, kid, grid, a); break;
+    default: launch_skinny_tm<NT, 5, 4, EPI, NORM>(L, kid, grid, a); break;
   }
 }
 
 // Returns the grid size: a RESID producer leaves one sum-of-squares part per CTA.
-template <int EPI>
+template <int EPI, bool NORM = false>
 int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
            const __half* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, int sumsq_stride, float eps,
-           const EpiArgs& e) {
+           const EpiArgs& e, const __half* gamma = nullptr) {
   if (L.rc != THINFER_OK) return 0;
   SkinnyArgs a{};
   a.w[0] = w0;
@@ -512,19 +520,37 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
   a.sumsq_in = sumsq_in;
   a.sumsq_parts = sumsq_in != nullptr ? sumsq_parts : 0;
   a.sumsq_stride = sumsq_stride;
+  a.gamma = gamma;
   a.norm_dim = k;
   a.norm_eps = eps;
   a.e = e;
   if (L.c != nullptr && L.c->trace_unified && kid >= 0 && kid < 12) {
-    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id
-    cudaMemsetAsync(a.dbg + 10, 0xff, 16, L.st);  // the two minima
-    cudaMemsetAsync(a.dbg + 12, 0, 32, L.st);     // the four maxima
+    a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id, reset at the start of the step
   }
   const int units = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
-  const int grid = skinny_grid(L.c, units);
-  a.tiles_max = ((units + grid - 1) / grid + 7) / 8;
-  if (rows <= 8) launch_skinny<1, EPI>(L, kid, grid, a);
-  else launch_skinny<2, EPI>(L, kid, grid, a);
+  const bool swiglu = EPI == EPI_SWIGLU, concatenated = n[1] != 0 && !swiglu;
+  const int sms = L.c ? L.c->sm_count : 148;
+  // Few features per SM and a long contraction (O, down): one CTA per SM with a deep ring.  Otherwise two
+  // (or more) CTAs per SM with a 4-stage ring each.
+  bool deep = false;
+  int grid = sms;
+  if (units >= 8 * sms) {
+    const int t1 = skinny_tiles_max(units, sms, swiglu, concatenated);
+    deep = t1 <= 2 && k >= 2048;
+  }
+  if (!deep) {
+    grid = 2 * sms;
+    while (skinny_tiles_max(units, grid, swiglu, concatenated) > kSkMaxTiles) grid += sms;
+    const int by_work = units / 8 > 0 ? units / 8 : 1;  // never less than one full tile per CTA
+    if (grid > by_work) grid = by_work;
+  }
+  a.tiles_max = skinny_tiles_max(units, grid, swiglu, concatenated);
+  if (a.tiles_max > kSkMaxTiles) {
+    L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection: %d tiles per share", a.tiles_max);
+    return 0;
+  }
+  if (rows <= 8) launch_skinny<1, EPI, NORM>(L, kid, grid, deep, a);
+  else launch_skinny<2, EPI, NORM>(L, kid, grid, deep, a);
   return grid;
 }
 
@@ -721,15 +747,20 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     const bool first_norm_folded = layer > 0;
     const int parts = (cf.hidden + kTcBM - 1) / kTcBM;  // the tcgen05 producers leave one sum per 128-feature tile
     const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
-    if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->d_h, batch, cf.hidden, cf.rms_eps);
+    static const bool od_env = [] { const char* e = getenv("THINFER_OD_TC"); return e != nullptr && atoi(e) != 0; }();
+    const bool od_tc = batch >= 2 && od_env;
     {
       const int n[3] = {qd, kvd, kvd};
-      skinny<EPI_QKV_ROPE>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, first_norm_folded ? c->xg : c->d_h,
-                           cf.hidden, batch, first_norm_folded ? c->sumsq0 : nullptr, batch >= 2 ? parts : c->sumsq0_parts,
-                           batch >= 2 ? 64 : 16, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
+      if (first_norm_folded)
+        skinny<EPI_QKV_ROPE>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, c->xg, cf.hidden, batch, c->sumsq0,
+                             od_tc ? parts : c->sumsq0_parts, od_tc ? 64 : 16, cf.rms_eps,
+                             qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
+      else  // the first norm of a step has no projection in front of it: RMSNorm as a prologue of this one
+        skinny<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch, nullptr,
+                                   0, 16, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens), H(w.attn_norm));
     }
     attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, max_t, lens, pos + 1);
-    if (batch >= 2) {
+    if (od_tc) {
       EpiArgs e{};
       e.out = c->d_x1;
       e.resid = x_in;
@@ -757,9 +788,9 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
       e.ld_out = cf.ffn;
       const int n[3] = {cf.ffn, cf.ffn, 0};
       skinny<EPI_SWIGLU>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->x1g, cf.hidden, batch,
-                         c->sumsq1, batch >= 2 ? parts : c->sumsq1_parts, batch >= 2 ? 64 : 16, cf.rms_eps, e);
+                         c->sumsq1, od_tc ? parts : c->sumsq1_parts, od_tc ? 64 : 16, cf.rms_eps, e);
     }
-    if (batch >= 2) {
+    if (od_tc) {
       EpiArgs e{};
       e.out = x_out;
       e.resid = c->d_x1;
@@ -972,6 +1003,7 @@ int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq,
                 cudaStream_t st, const int* lens_dev = nullptr) {
   const thinfer_config& cf = c->cfg;
   Launcher L{c, st};
+  if (c->trace_unified) L.go(-3, trace_reset_kernel, dim3(1), dim3(256), 0, c->timeline, 12);
   const int rows = batch * seq;
   const __half* x = nullptr;
   if (cf.vocab > 0) {
@@ -999,6 +1031,7 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
                cudaStream_t st) {
   const thinfer_config& cf = c->cfg;
   Launcher L{c, st};
+  if (c->trace_unified) L.go(-3, trace_reset_kernel, dim3(1), dim3(256), 0, c->timeline, 12);
   const __half* x = nullptr;
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((batch + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
