@@ -348,7 +348,7 @@ def run_ours(args):
         "prefill": {"value": pre_tokens / (pre_ms * 1e-3), "unit": "tok/s", "ms": pre_ms / args.steps,
                     "achieved_TFLOPs": pre_tflops, "frac_of_tensor_peak": pre_tflops / tc_peak,
                     "peak_TFLOPs": tc_peak, "peak_kind": peak_kind + " bf16 sustained (same tensor-pipe rate as fp16)"},
-        "roofline": {"kernel": ("gemv_stream_kernel<SWIGLU>" if B == 1 else "tc_gemm_kernel<16..64, SWIGLU> stream-K")
+        "roofline": {"kernel": ("skinny_mma_kernel<SWIGLU>" if B <= 16 else "tc_gemm_kernel<32..64, SWIGLU> stream-K")
                      + " (decode gate/up projection)", "bound": "hbm",
                      "achieved": gu_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gu_gbs / hbm_peak,
                      "traffic": captured_traffic("decode_gateup_b16", B), "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3,

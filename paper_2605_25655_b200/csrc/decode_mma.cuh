@@ -33,6 +33,7 @@ constexpr int kSkTokMax = 16;
 struct SkinnyArgs {
   const __half* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
   int n[3];            // rows of each matrix (0 for unused); every count is even
+  int cta0[4];         // CTAs cta0[m] .. cta0[m+1]-1 share matrix m (SWIGLU: everything is "matrix" 0)
   int k;               // contraction length, multiple of 64
   int rows;            // tokens, <= 8 * NT
   const __half* x;     // [rows][ldx]
@@ -85,20 +86,6 @@ __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 
-// Row r of the concatenated feature space -> address of that weight row.
-__device__ __forceinline__ const __half* sk_row_ptr(const SkinnyArgs& a, int r) {
-  int m = 0;
-  if (r >= a.n[0]) {
-    r -= a.n[0];
-    m = 1;
-    if (r >= a.n[1]) {
-      r -= a.n[1];
-      m = 2;
-    }
-  }
-  return a.w[m] + static_cast<size_t>(r) * a.k;
-}
-
 // The ring doubles as the parking area of the finished fragments (TM * NT * 128 floats per warp).
 __host__ __device__ constexpr int sk_smem_floats(int tm, int stages, int parts) {
   return kSkWarps * stages * 512 + parts * 16 + tm * 16 + 16 * 16 + 16;
@@ -113,7 +100,7 @@ __host__ __device__ constexpr int sk_smem_floats(int tm, int stages, int parts) 
 // irrelevant as long as A and B agree, so every lane simply takes 16 contiguous bytes: of a 64-element
 // block, lane t holds elements 8t..8t+7 and 32+8t..32+8t+7 of its rows and of its token.
 template <int NT, int TM, int ST, int EPI, bool NORM = false>
-__global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_kernel(const SkinnyArgs a) {
+__global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const SkinnyArgs a) {
   static_assert(ST * 4 >= TM * NT, "the fragments of a warp are parked in its own ring");
   pdl_launch_dependents();
   extern __shared__ __align__(16) float sk_smem[];
@@ -122,19 +109,22 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
     atomicMin(a.dbg + 10, static_cast<unsigned long long>(global_ns()));  // earliest CTA start
     atomicMax(a.dbg + 12, static_cast<unsigned long long>(global_ns()));  // latest CTA start
   }
-  const int units = (EPI == EPI_SWIGLU) ? a.n[0] : (a.n[0] + a.n[1] + a.n[2]) >> 1;
-  const int u_beg = static_cast<int>(static_cast<long long>(blockIdx.x) * units / gridDim.x);
-  const int u_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * units / gridDim.x);
-  // Rows of the share in tile coordinates.  SWIGLU: "row" = feature, a tile holds 8 features (8 gate rows
-  // and 8 up rows).  Otherwise a tile holds 16 rows.  Tiles start at the share, except when several
-  // matrices are concatenated (QKV): there a tile starts at a multiple of 16 rows, so that no tile lies
-  // across two matrices (their row counts are multiples of 16), and the first and the last tile of a share
-  // may be partial.  Rows outside [r_lo, r_hi) cost no traffic.
+  // The CTAs are dealt out to the matrices in proportion to their rows, so a share never lies across two
+  // matrices; inside its matrix a CTA takes a contiguous run of units, balanced to within one unit.
+  const int m = (static_cast<int>(blockIdx.x) >= a.cta0[2]) ? 2 : (static_cast<int>(blockIdx.x) >= a.cta0[1] ? 1 : 0);
+  const int m_ctas = a.cta0[m + 1] - a.cta0[m], m_cta = blockIdx.x - a.cta0[m];
+  const int units = (EPI == EPI_SWIGLU) ? a.n[0] : a.n[m] >> 1;
+  const int u_beg = static_cast<int>(static_cast<long long>(m_cta) * units / m_ctas);
+  const int u_end = static_cast<int>(static_cast<long long>(m_cta + 1) * units / m_ctas);
+  // Rows of the share, numbered inside the matrix.  SWIGLU: "row" = feature, a tile holds 8 features (8 gate
+  // rows and 8 up rows); otherwise a tile holds 16 rows.  Tiles start at the share; the last one may be
+  // partial.  Rows outside [r_lo, r_hi) cost no traffic.
   constexpr int TR = (EPI == EPI_SWIGLU) ? 8 : 16;  // share rows per tile
   const int r_lo = (EPI == EPI_SWIGLU) ? u_beg : 2 * u_beg;
   const int r_hi = (EPI == EPI_SWIGLU) ? u_end : 2 * u_end;
-  const int row00 = (EPI == EPI_SWIGLU || a.n[1] == 0) ? r_lo : (r_lo & ~15);  // first row of tile 0
-  const int n_tiles = r_hi > r_lo ? (r_hi - row00 + TR - 1) / TR : 0;  // <= TM; the walk always takes TM tiles
+  const int row00 = r_lo;                                    // first row of tile 0
+  const int r_cat = (m == 0) ? 0 : (m == 1 ? a.n[0] : a.n[0] + a.n[1]);  // row of the concatenated space = r_cat + row
+  const int n_tiles = (r_hi - r_lo + TR - 1) / TR;           // <= TM; the walk always takes TM tiles
   const int nkb = a.k >> 6;                                  // k is a multiple of 64 (checked on the host)
   const int nkw = (nkb - warp + kSkWarps - 1) / kSkWarps;    // blocks warp, warp + 8, ...
 
@@ -153,13 +143,12 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
   const int crow = lane >> 3, cchunk = lane & 7;
   const uint32_t coop_dst = smem_u32(ring) + crow * 128 + ((cchunk ^ ((crow & 1) << 2)) << 4);
   const size_t coop_off = static_cast<size_t>(warp) * 64 + cchunk * 8;
-  const int lim_lo = r_lo - row00 - crow, lim_hi = r_hi - row00 - crow;  // tile row TR*tile + 4j (+crow) is in the share
-                                                                         // iff lim_lo <= TR*tile + 4j < lim_hi
+  const int lim_hi = r_hi - r_lo - crow;  // tile row TR * tile + 4 j (+ crow) is in the share iff TR * tile + 4 j < lim_hi
   const __half* tb[TM];  // plain: row crow of the tile, at this lane's chunk of block `warp`
   if (EPI != EPI_SWIGLU) {
-    const int last = a.n[0] + a.n[1] + a.n[2] - 1;
 #pragma unroll
-    for (int tile = 0; tile < TM; ++tile) tb[tile] = sk_row_ptr(a, min(row00 + tile * 16 + crow, last)) + coop_off;
+    for (int tile = 0; tile < TM; ++tile)
+      tb[tile] = a.w[m] + static_cast<size_t>(min(row00 + tile * 16 + crow, a.n[m] - 1)) * a.k + coop_off;
   }
   auto request = [&](int tile, int blk, int stage) {
     const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
@@ -177,7 +166,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
       const size_t k4 = static_cast<size_t>(4) * a.k;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const bool ok = tile * 16 + 4 * j >= lim_lo && tile * 16 + 4 * j < lim_hi;
+        const bool ok = tile * 16 + 4 * j < lim_hi;
         cp_async_16(dst + 512 * j, ok ? src + j * k4 : a.w[0], ok ? 16u : 0u);
       }
     }
@@ -244,7 +233,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
         if (i + XB - 1 < nkw) load_x(i + XB - 1, xq[(b + XB - 1) % XB]);
         if (NORM) {
           const size_t off = static_cast<size_t>(i) * (kSkWarps * 64);
-          const uint4 g0 = ldg_cached(grow + off), g1 = ldg_cached(grow + off + 32);
+          const uint4 g0 = ldg_cached(grow + off), g1 = ldg_cached(grow + off + 32);  // 8 KB in all: stays in L1
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             float f[8];
@@ -350,7 +339,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
 #pragma unroll
       for (int i = 0; i < 4; ++i) c[i] += src[i * 32];
     }
-    const int row0 = row00 + tile * TR;  // first share row of the tile
+    const int row0 = row00 + tile * TR;  // first share row of the tile (numbered inside the matrix)
     const int ta = nt * 8 + 2 * t, tb = ta + 1;
     if (NORM || a.sumsq_in != nullptr) {
       const float sa = rstd[ta], sb = rstd[tb];
@@ -372,7 +361,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
         const int row = row0 + g + 8 * hr;
-        const bool row_ok = row >= r_lo && row < r_hi;
+        const bool row_ok = row < r_hi;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           const int tok = ta + j;
@@ -383,7 +372,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
           size_t off = 0;
           const bool ok = row_ok && tok < a.rows;
           if (ok) {
-            off = qkv_offset(e, tok, row, kind, i, pos);
+            off = qkv_offset(e, tok, r_cat + row, kind, i, pos);
             if (kind != 2) {
               const size_t o = static_cast<size_t>(pos) * (e.head_dim >> 1) + (i >> 1);
               y = fmaf(sgn * partner, __ldg(e.rope_sin + o), val * __ldg(e.rope_cos + o));
@@ -401,7 +390,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, ST <= 4 ? 2 : 1) skinny_mma_ker
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
         const int row = row0 + g + 8 * hr;
-        if (row >= r_lo && row < r_hi) {
+        if (row < r_hi) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const int tok = ta + j;

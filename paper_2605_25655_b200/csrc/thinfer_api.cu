@@ -458,16 +458,33 @@ void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half
 // ----------------------------------------------------------------------------
 constexpr int kSkMaxTiles = 5;  // 16-row tiles per CTA share the kernels are instantiated for (1 .. 5)
 
-// Largest number of tiles a CTA share touches (mirrors the kernel's tile rule).
-int skinny_tiles_max(int units, int grid, bool swiglu, bool concatenated) {
-  int worst = 0;
-  for (int cta = 0; cta < grid; ++cta) {
-    const int ub = static_cast<int>(static_cast<long long>(cta) * units / grid);
-    const int ue = static_cast<int>(static_cast<long long>(cta + 1) * units / grid);
-    if (ue <= ub) continue;
-    const int lo = swiglu ? ub : 2 * ub, hi = swiglu ? ue : 2 * ue, tr = swiglu ? 8 : 16;
-    const int r0 = (swiglu || !concatenated) ? lo : (lo & ~15);
-    worst = std::max(worst, (hi - r0 + tr - 1) / tr);
+// Deals `grid` CTAs out to the matrices in proportion to their rows (every matrix with rows gets at least
+// one) and returns the largest number of tiles a CTA share has (mirrors the kernel's partition).
+int skinny_partition(const int (&n)[3], bool swiglu, int grid, int (&cta0)[4]) {
+  const int mats = swiglu ? 1 : 3;
+  long long total = 0;
+  int used = 0;
+  for (int m = 0; m < mats; ++m) {
+    total += n[m];
+    used += n[m] > 0;
+  }
+  int given = 0, worst = 0;
+  long long rows_before = 0;
+  cta0[0] = 0;
+  for (int m = 0; m < 3; ++m) {
+    int ctas = 0;
+    if (m < mats && n[m] > 0) {
+      --used;
+      rows_before += n[m];
+      // cumulative rounding keeps the total exact; leave one CTA for every matrix still to come
+      ctas = static_cast<int>((rows_before * grid + total / 2) / total) - given;
+      if (ctas < 1) ctas = 1;
+      if (ctas > grid - given - used) ctas = grid - given - used;
+      const int units = swiglu ? n[m] : n[m] / 2, tr = 8;  // 8 units per tile either way
+      worst = std::max(worst, ((units + ctas - 1) / ctas + tr - 1) / tr);
+    }
+    given += ctas;
+    cta0[m + 1] = given;
   }
   return worst;
 }
@@ -487,12 +504,7 @@ void launch_skinny_tm(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
 }
 
 template <int NT, int EPI, bool NORM>
-void launch_skinny(Launcher& L, int kid, int grid, bool deep, const SkinnyArgs& a) {
-  if (deep) {  // one CTA per SM, an 8-stage ring: half of a 4096-long contraction is requested before the wait
-    if (a.tiles_max <= 1) launch_skinny_tm<NT, 1, 8, EPI, NORM>(L, kid, grid, a);
-    else launch_skinny_tm<NT, 2, 8, EPI, NORM>(L, kid, grid, a);
-    return;
-  }
+void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
   switch (a.tiles_max) {
     case 1: launch_skinny_tm<NT, 1, 4, EPI, NORM>(L, kid, grid, a); break;
     case 2: launch_skinny_tm<NT, 2, 4, EPI, NORM>(L, kid, grid, a); break;
@@ -528,29 +540,25 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
     a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id, reset at the start of the step
   }
   const int units = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
-  const bool swiglu = EPI == EPI_SWIGLU, concatenated = n[1] != 0 && !swiglu;
+  const bool swiglu = EPI == EPI_SWIGLU;
   const int sms = L.c ? L.c->sm_count : 148;
-  // Few features per SM and a long contraction (O, down): one CTA per SM with a deep ring.  Otherwise two
-  // (or more) CTAs per SM with a 4-stage ring each.
-  bool deep = false;
-  int grid = sms;
-  if (units >= 8 * sms) {
-    const int t1 = skinny_tiles_max(units, sms, swiglu, concatenated);
-    deep = t1 <= 2 && k >= 2048;
+  // Two CTAs per SM with a 4-stage ring per warp (a one-CTA variant with an 8-stage ring, tried for the two
+  // projections with few features per SM, was slower); more CTAs when a share would exceed kSkMaxTiles tiles.
+  const int mats = swiglu ? 1 : (n[0] > 0) + (n[1] > 0) + (n[2] > 0);
+  int grid = 2 * sms;
+  const int by_work = std::max(units / 8, mats);  // never less than one full tile per CTA
+  if (grid > by_work) grid = by_work;
+  a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
+  while (a.tiles_max > kSkMaxTiles && grid < 64 * sms) {
+    grid += sms;
+    a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
   }
-  if (!deep) {
-    grid = 2 * sms;
-    while (skinny_tiles_max(units, grid, swiglu, concatenated) > kSkMaxTiles) grid += sms;
-    const int by_work = units / 8 > 0 ? units / 8 : 1;  // never less than one full tile per CTA
-    if (grid > by_work) grid = by_work;
-  }
-  a.tiles_max = skinny_tiles_max(units, grid, swiglu, concatenated);
   if (a.tiles_max > kSkMaxTiles) {
     L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection: %d tiles per share", a.tiles_max);
     return 0;
   }
-  if (rows <= 8) launch_skinny<1, EPI, NORM>(L, kid, grid, deep, a);
-  else launch_skinny<2, EPI, NORM>(L, kid, grid, deep, a);
+  if (rows <= 8) launch_skinny<1, EPI, NORM>(L, kid, grid, a);
+  else launch_skinny<2, EPI, NORM>(L, kid, grid, a);
   return grid;
 }
 
