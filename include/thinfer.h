@@ -186,7 +186,9 @@ int thinfer_set_launch_mode(thinfer_ctx* ctx, int32_t mode);
 /* Per-kernel timing for roofline reports.  When `kernel_id` >= 0 every launch
  * of that kernel (thinfer_kernel_id) is bracketed by CUDA events on its own
  * stream; thinfer_profile_read synchronises those events and returns the count
- * and the summed duration since the last read.  -1 switches it off. */
+ * and the summed duration since the last read.  -1 switches it off.
+ * (THINFER_K_ATTN_COMBINE is kept for numbering only: the split-KV merge runs
+ * inside the decode attention kernel and has no launches of its own.) */
 typedef enum {
   THINFER_K_RMSNORM = 0, THINFER_K_QKV = 1, THINFER_K_ATTN = 2, THINFER_K_ATTN_COMBINE = 3,
   THINFER_K_OPROJ = 4, THINFER_K_GATEUP = 5, THINFER_K_DOWN = 6, THINFER_K_HEAD = 7,

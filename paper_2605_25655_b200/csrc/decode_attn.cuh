@@ -5,7 +5,9 @@
 // head are processed in the same pass.  The KV range is split across CTAs
 // (split-KV); every lane group keeps a running (max, sum, output) triple that
 // is merged by the online-softmax rule first inside the warp, then across the
-// CTA's warps, then across splits by a small combine kernel.
+// CTA's warps, then across splits by whichever CTA of a (request, head group)
+// finishes last (a ticket counter; the partials are added in split order, so the
+// result does not depend on who that is).
 #pragma once
 #include "common.cuh"
 
@@ -21,6 +23,7 @@ struct AttnDecArgs {
   __half* out;            // [batch][n_q_heads * D]
   float* part_o;          // [batch][n_q_heads][splits][D]   un-normalised partial outputs
   float* part_ml;         // [batch][n_q_heads][splits][2]   (max in log2 units, sum)
+  int* tickets;           // [batch][n_q_heads / G] arrival counters, zero between launches (splits > 1)
   int n_q_heads, n_kv_heads;
   int t_len;              // keys to attend: positions 0 .. t_len-1
   const int* len_arr;     // ragged: request b attends len_arr[b] + t_len keys (nullptr: t_len for everybody)
@@ -209,25 +212,36 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
       }
     }
   }
-}
+  if (a.splits == 1) return;
 
-// Merges the split-KV partials: out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
-template <int D>
-__global__ void __launch_bounds__(D) attn_decode_combine_kernel(const AttnDecArgs a) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const size_t bh = blockIdx.x;  // (request, query head)
-  const int i = threadIdx.x;
-  float mx = -INFINITY;
-  for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, a.part_ml[(bh * a.splits + s) * 2]);
-  float L = 0.f, O = 0.f;
-  for (int s = 0; s < a.splits; ++s) {
-    const size_t p = bh * a.splits + s;
-    const float al = exp2f(a.part_ml[p * 2] - mx);
-    L += a.part_ml[p * 2 + 1] * al;
-    O += a.part_o[p * D + i] * al;
+  // split-KV: the CTA that arrives last merges the partials of its G heads,
+  // out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), s in split order
+  __shared__ int is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int* ctr = a.tickets + b * gridDim.y + blockIdx.y;
+    const int ticket = atomicAdd(ctr, 1);
+    is_last = ticket == a.splits - 1;
+    if (is_last) *ctr = 0;  // ready for the next launch
   }
-  a.out[bh * D + i] = __float2half_rn(O / L);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
+    const int g = idx / D, i = idx - g * D;
+    const size_t bh = static_cast<size_t>(b) * a.n_q_heads + h0 + g;
+    float mx = -INFINITY;
+    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, __ldcg(a.part_ml + (bh * a.splits + s) * 2));
+    float L = 0.f, O = 0.f;
+    for (int s = 0; s < a.splits; ++s) {
+      const size_t p = bh * a.splits + s;
+      const float al = exp2f(__ldcg(a.part_ml + p * 2) - mx);
+      L += __ldcg(a.part_ml + p * 2 + 1) * al;
+      O += __ldcg(a.part_o + p * D + i) * al;
+    }
+    a.out[bh * D + i] = __float2half_rn(O / L);
+  }
 }
 
 }  // namespace thinfer

@@ -38,11 +38,10 @@ struct SkinnyArgs {
   int rows;            // tokens, <= 8 * NT
   const __half* x;     // [rows][ldx]
   int ldx;
-  // folded RMSNorm of the token operand: sums of squares per (part, token), [sumsq_parts][sumsq_stride]
-  // (stride 16 when a skinny projection produced them, 64 when a tcgen05 projection did)
+  // folded RMSNorm of the token operand: sums of squares per (part, token), [sumsq_parts][16], as the
+  // RESID epilogue of this kernel leaves them (one part per CTA)
   const float* sumsq_in;
   int sumsq_parts;
-  int sumsq_stride;
   int norm_dim;
   float norm_eps;
   // NORM kernels instead take the raw rows in x and the gain here: RMSNorm as a prologue.  Every CTA reads
@@ -186,7 +185,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
     // asynchronous copies straight into shared memory: no registers held, consumed after the stream
     // (they join whichever group is committed next; the final wait covers them)
     for (int i = threadIdx.x; i < a.sumsq_parts * 16; i += kSkWarps * 32)
-      cp_async_4(ssq_in + i, a.sumsq_in + (i >> 4) * a.sumsq_stride + (i & 15));
+      cp_async_4(ssq_in + i, a.sumsq_in + i);
   }
 
   // token fragments: XB buffers, requested XB - 1 blocks ahead (the fewer tiles a block has, the further)
@@ -386,29 +385,31 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
         }
       }
     } else {
+      // rows g and g + 1 (g even) are neighbours in memory: the even lane takes both, 4 bytes at a time
       float sq[2] = {0.f, 0.f};
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
         const int row = row0 + g + 8 * hr;
-        if (row < r_hi) {
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const int tok = ta + j;
-            if (tok >= a.rows) continue;
-            const size_t off = static_cast<size_t>(tok) * e.ld_out + row;
-            const float v = c[hr * 2 + j];
-            if (EPI == EPI_PLAIN_F32) {
-              reinterpret_cast<float*>(e.out)[off] = v;
-            } else if (EPI == EPI_PLAIN_F16) {
-              reinterpret_cast<__half*>(e.out)[off] = __float2half_rn(v);
-            } else {  // EPI_RESID
-              const __half yh = __float2half_rn(__half2float(e.resid[off]) + v);
-              reinterpret_cast<__half*>(e.out)[off] = yh;
-              if (e.outg != nullptr) {  // folded RMSNorm of the next sub-layer (gain here, 1/rms there)
-                const float y = __half2float(yh);
-                e.outg[off] = __float2half_rn(y * __half2float(e.gain_next[row]));
-                sq[j] = fmaf(y, y, sq[j]);
-              }
+        for (int j = 0; j < 2; ++j) {
+          const int tok = ta + j;
+          const float v0 = c[hr * 2 + j];
+          const float v1 = __shfl_xor_sync(0xffffffffu, v0, 4);
+          if ((g & 1) || row >= r_hi || tok >= a.rows) continue;
+          const size_t off = static_cast<size_t>(tok) * e.ld_out + r_cat + row;
+          if (EPI == EPI_PLAIN_F32) {
+            *reinterpret_cast<float2*>(reinterpret_cast<float*>(e.out) + off) = make_float2(v0, v1);
+          } else if (EPI == EPI_PLAIN_F16) {
+            *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + off) = pack2(v0, v1);
+          } else {  // EPI_RESID
+            const float2 x = __half22float2(*reinterpret_cast<const __half2*>(e.resid + off));
+            const uint32_t yh = pack2(x.x + v0, x.y + v1);
+            *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + off) = yh;
+            if (e.outg != nullptr) {  // folded RMSNorm of the next sub-layer (gain here, 1/rms there)
+              const float2 y = __half22float2(*reinterpret_cast<const __half2*>(&yh));
+              const float2 gn = __half22float2(*reinterpret_cast<const __half2*>(e.gain_next + r_cat + row));
+              *reinterpret_cast<uint32_t*>(e.outg + off) = pack2(y.x * gn.x, y.y * gn.y);
+              sq[j] = fmaf(y.x, y.x, fmaf(y.y, y.y, sq[j]));
             }
           }
         }

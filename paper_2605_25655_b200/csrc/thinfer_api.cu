@@ -517,8 +517,8 @@ void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
 // Returns the grid size: a RESID producer leaves one sum-of-squares part per CTA.
 template <int EPI, bool NORM = false>
 int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
-           const __half* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, int sumsq_stride, float eps,
-           const EpiArgs& e, const __half* gamma = nullptr) {
+           const __half* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, float eps, const EpiArgs& e,
+           const __half* gamma = nullptr) {
   if (L.rc != THINFER_OK) return 0;
   SkinnyArgs a{};
   a.w[0] = w0;
@@ -531,7 +531,6 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
   a.ldx = ldx;
   a.sumsq_in = sumsq_in;
   a.sumsq_parts = sumsq_in != nullptr ? sumsq_parts : 0;
-  a.sumsq_stride = sumsq_stride;
   a.gamma = gamma;
   a.norm_dim = k;
   a.norm_eps = eps;
@@ -578,8 +577,6 @@ void attn_decode_d(Launcher& L, const AttnDecArgs& a, int batch, int ratio) {
     case 2: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 2>, grid, block, 0, a); break;
     default: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 1>, grid, block, 0, a); break;
   }
-  if (a.splits > 1)
-    L.go(THINFER_K_ATTN_COMBINE, attn_decode_combine_kernel<D>, dim3(batch * a.n_q_heads), dim3(D), 0, a);
 }
 
 void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc, const __half* vc, __half* out,
@@ -592,6 +589,7 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   a.out = out;
   a.part_o = c->part_o;
   a.part_ml = c->part_ml;
+  a.tickets = c->attn_counters;
   a.n_q_heads = cf.n_q_heads;
   a.n_kv_heads = cf.n_kv_heads;
   a.t_len = len_arr != nullptr ? len_add : t_len;  // ragged: per-request count = len_arr[b] + len_add
@@ -746,39 +744,24 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
   __half* vc = kv_ptr(c, slot, layer, 1);
   auto H = [](const void* p) { return static_cast<const __half*>(p); };
   if (batch <= kSkTokMax && c->skinny_ok) {
-    // Up to 16 tokens.  The wide projections (QKV, gate/up: many output features per SM) run as balanced
-    // weight streams into warp-level tensor-core fragments, with no partial sums across CTAs; the two
-    // projections with few output features and a long contraction (O, down) split K across the SMs on the
-    // tcgen05 stream-K path, which is the faster of the two for them.
-    // The RMSNorm in front of a projection is folded into the projection before it (gain there, 1/rms here).
-    const LayerMaps& m = c->maps[layer];
+    // Up to 16 tokens: every projection is a balanced weight stream into warp-level tensor-core fragments
+    // (no partial sums across CTAs, no tensor memory, so the CTAs of the next projection move in as this
+    // one's leave and fill their rings before the dependency wait).  The RMSNorm in front of a projection
+    // is folded into the projection before it (gain there, 1/rms here); the first norm of a step has no
+    // projection in front of it and runs as a prologue of the QKV projection.
     const bool first_norm_folded = layer > 0;
-    const int parts = (cf.hidden + kTcBM - 1) / kTcBM;  // the tcgen05 producers leave one sum per 128-feature tile
     const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
-    static const bool od_env = [] { const char* e = getenv("THINFER_OD_TC"); return e != nullptr && atoi(e) != 0; }();
-    const bool od_tc = batch >= 2 && od_env;
     {
       const int n[3] = {qd, kvd, kvd};
       if (first_norm_folded)
         skinny<EPI_QKV_ROPE>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, c->xg, cf.hidden, batch, c->sumsq0,
-                             od_tc ? parts : c->sumsq0_parts, od_tc ? 64 : 16, cf.rms_eps,
-                             qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
-      else  // the first norm of a step has no projection in front of it: RMSNorm as a prologue of this one
+                             c->sumsq0_parts, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens));
+      else
         skinny<EPI_QKV_ROPE, true>(L, THINFER_K_QKV, H(w.wq), H(w.wk), H(w.wv), n, cf.hidden, x_in, cf.hidden, batch, nullptr,
-                                   0, 16, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens), H(w.attn_norm));
+                                   0, cf.rms_eps, qkv_epi(c, c->d_qbuf, kc, vc, 1, pos, lens), H(w.attn_norm));
     }
     attn_decode(L, c, c->d_qbuf, kc, vc, c->d_attn, batch, max_t, lens, pos + 1);
-    if (od_tc) {
-      EpiArgs e{};
-      e.out = c->d_x1;
-      e.resid = x_in;
-      e.ld_out = cf.hidden;
-      e.outg = c->x1g;
-      e.gain_next = H(w.ffn_norm);
-      e.sumsq = c->sumsq1;
-      const int nf[3] = {cf.hidden, 0, 0};
-      tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->d_attn, batch, qd, nf, e, true);
-    } else {
+    {
       EpiArgs e{};
       e.out = c->d_x1;
       e.resid = x_in;
@@ -788,7 +771,7 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
       e.sumsq = c->sumsq1;
       const int n[3] = {cf.hidden, 0, 0};
       c->sumsq1_parts = skinny<EPI_RESID>(L, THINFER_K_OPROJ, H(w.wo), nullptr, nullptr, n, qd, c->d_attn, qd, batch,
-                                          nullptr, 0, 16, 0.f, e);
+                                          nullptr, 0, 0.f, e);
     }
     {
       EpiArgs e{};
@@ -796,21 +779,9 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
       e.ld_out = cf.ffn;
       const int n[3] = {cf.ffn, cf.ffn, 0};
       skinny<EPI_SWIGLU>(L, THINFER_K_GATEUP, H(w.w_gate), H(w.w_up), nullptr, n, cf.hidden, c->x1g, cf.hidden, batch,
-                         c->sumsq1, od_tc ? parts : c->sumsq1_parts, od_tc ? 64 : 16, cf.rms_eps, e);
+                         c->sumsq1, c->sumsq1_parts, cf.rms_eps, e);
     }
-    if (od_tc) {
-      EpiArgs e{};
-      e.out = x_out;
-      e.resid = c->d_x1;
-      e.ld_out = cf.hidden;
-      if (next_gain != nullptr) {
-        e.outg = c->xg;
-        e.gain_next = next_gain;
-        e.sumsq = c->sumsq0;
-      }
-      const int nf[3] = {cf.hidden, 0, 0};
-      tc_linear<EPI_RESID>(L, THINFER_K_DOWN, m.wd, m.wd, m.wd, c->d_act, batch, cf.ffn, nf, e, true);
-    } else {
+    {
       EpiArgs e{};
       e.out = x_out;
       e.resid = c->d_x1;
@@ -822,7 +793,7 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
       }
       const int n[3] = {cf.hidden, 0, 0};
       c->sumsq0_parts = skinny<EPI_RESID>(L, THINFER_K_DOWN, H(w.w_down), nullptr, nullptr, n, cf.ffn, c->d_act, cf.ffn,
-                                          batch, nullptr, 0, 16, 0.f, e);
+                                          batch, nullptr, 0, 0.f, e);
     }
     return;
   }
@@ -1543,10 +1514,10 @@ int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32
     if (rows > kSkTokMax || k % 64 != 0) return THINFER_EUNSUPPORTED;
     if (out_fp32)
       skinny<EPI_PLAIN_F32>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
-                            rows, nullptr, 0, 16, 0.f, e);
+                            rows, nullptr, 0, 0.f, e);
     else
       skinny<EPI_PLAIN_F16>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
-                            rows, nullptr, 0, 16, 0.f, e);
+                            rows, nullptr, 0, 0.f, e);
   } else if (path == 0) {
     CUtensorMap mw;
     if (!make_map_2d(&mw, w, k, n_out, 128)) return THINFER_ECUDA;

@@ -394,21 +394,28 @@ def test_prefill_and_decode_stages_on_two_streams(T):
     w = synth.layer_weights(shape, 9)
     x = torch.from_numpy(synth.hidden_states(shape, 9, (2, 3, 40))).cuda()     # two micro-batches of 3 requests
 
+    # every input is materialised and the device synchronised before the streams start: a temporary made on
+    # torch's current stream would neither be ordered with, nor kept alive for, work on the other streams
+    pin = {"p0": x[0, :, :30].contiguous(), "p1": x[1, :, :30].contiguous(), "p0b": x[1, :, :25].contiguous(),
+           "d0b": x[1, :, 25].contiguous()}
+    d0 = [x[0, :, 30 + i].contiguous() for i in range(6)]
+    d1 = [x[1, :, 30 + i].contiguous() for i in range(4)]
+
     def run(two_streams):
         ctx = _ctx(T, shape, [w], 3, 48, buf_slots=2)
         sp = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
         sd = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
         torch.cuda.synchronize()
         outs = {}
-        outs["p0"] = ctx.prefill(x[0, :, :30].contiguous(), slot=0, stream=sp)
-        outs["p1"] = ctx.prefill(x[1, :, :30].contiguous(), slot=1, stream=sp)      # runs while slot 0 decodes
+        outs["p0"] = ctx.prefill(pin["p0"], slot=0, stream=sp)
+        outs["p1"] = ctx.prefill(pin["p1"], slot=1, stream=sp)      # runs while slot 0 decodes
         for i in range(6):
-            outs[f"d0_{i}"] = ctx.decode_step(x[0, :, 30 + i].contiguous(), slot=0, stream=sd)
+            outs[f"d0_{i}"] = ctx.decode_step(d0[i], slot=0, stream=sd)
         ctx.release_slot(0, stream=sd)
-        outs["p0b"] = ctx.prefill(x[1, :, :25].contiguous(), slot=0, stream=sp)     # waits for the release on the device
+        outs["p0b"] = ctx.prefill(pin["p0b"], slot=0, stream=sp)    # waits for the release on the device
         for i in range(4):
-            outs[f"d1_{i}"] = ctx.decode_step(x[1, :, 30 + i].contiguous(), slot=1, stream=sd)
-        outs["d0b"] = ctx.decode_step(x[1, :, 25].contiguous(), slot=0, stream=sd)
+            outs[f"d1_{i}"] = ctx.decode_step(d1[i], slot=1, stream=sd)
+        outs["d0b"] = ctx.decode_step(pin["d0b"], slot=0, stream=sd)
         torch.cuda.synchronize()
         assert ctx.status() == 0
         res = {k: v.cpu().numpy() for k, v in outs.items()}
