@@ -177,15 +177,27 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
     const bool rotate = t.mat != 2;
     // all table reads of the chunk are issued before any is used: one L2 latency per chunk, not per column
     float cs[CW], sn[CW];
-    {
+    if (e.pos_arr == nullptr) {  // uniform positions (prefill, equal-length decode): no load on the address path
+      int s = tok_base % e.seq_len;
+#pragma unroll
+      for (int c = 0; c < CW; ++c) {
+        cs[c] = 1.f;
+        sn[c] = 0.f;
+        if (rotate && tok_base + c < a.rows) {
+          const size_t o = static_cast<size_t>(e.pos0 + s) * half + (i >> 1);
+          cs[c] = __ldg(e.rope_cos + o);
+          sn[c] = __ldg(e.rope_sin + o);
+        }
+        if (++s == e.seq_len) s = 0;
+      }
+    } else {  // ragged decode: every request has its own position
       int b = tok_base / e.seq_len, s = tok_base - b * e.seq_len;
 #pragma unroll
       for (int c = 0; c < CW; ++c) {
         cs[c] = 1.f;
         sn[c] = 0.f;
         if (rotate && tok_base + c < a.rows) {
-          const int pos = e.pos0 + s + (e.pos_arr != nullptr ? e.pos_arr[b] : 0);
-          const size_t o = static_cast<size_t>(pos) * half + (i >> 1);
+          const size_t o = static_cast<size_t>(e.pos0 + s + e.pos_arr[b]) * half + (i >> 1);
           cs[c] = __ldg(e.rope_cos + o);
           sn[c] = __ldg(e.rope_sin + o);
         }
