@@ -968,7 +968,11 @@ void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, in
   e.out = lg;
   e.ld_out = cf.vocab;
   const int n[3] = {cf.vocab, 0, 0};
-  if (batch >= 2) {
+  if (batch <= kSkTokMax && c->skinny_ok && cf.vocab % 2 == 0) {
+    // final RMSNorm as the prologue of the vocabulary projection, one balanced weight stream
+    skinny<EPI_PLAIN_F32, true>(L, THINFER_K_HEAD, c->lm_head, nullptr, nullptr, n, cf.hidden, x, cf.hidden, batch, nullptr, 0,
+                                cf.rms_eps, e, c->final_norm);
+  } else if (batch >= 2) {
     rmsnorm_rows(L, x, c->final_norm, hbuf, batch, cf.hidden, cf.rms_eps);
     tc_linear<EPI_PLAIN_F32>(L, THINFER_K_HEAD, c->map_head, c->map_head, c->map_head, hbuf, batch, cf.hidden, n, e, true);
   } else {
