@@ -273,7 +273,10 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   }
   cp_async_wait_all();
   __syncwarp();
-  if (a.dbg != nullptr && lane == 0) atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // stream end
+  if (a.dbg != nullptr && lane == 0) {
+    atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // latest stream end of a warp
+    atomicMin(a.dbg + 9, static_cast<unsigned long long>(global_ns()));   // earliest
+  }
   // park the fragments in this warp's own ring
   {
     float* dst = part + static_cast<size_t>(warp) * (ST * 512) + lane;

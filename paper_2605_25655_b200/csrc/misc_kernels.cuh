@@ -188,13 +188,13 @@ __global__ void rope_table_kernel(float* __restrict__ cos_t, float* __restrict__
   sin_t[idx] = static_cast<float>(s);
 }
 
-// Tracing aid: resets the 16 slots of every kernel id before a traced step (slots 10, 11 collect minima,
+// Tracing aid: resets the 16 slots of every kernel id before a traced step (slots 9 .. 11 collect minima,
 // 12 .. 15 maxima), so that no memset sits between the kernels of the step.
 __global__ void trace_reset_kernel(unsigned long long* timeline, int kernels) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= kernels * 16) return;
   const int slot = i & 15;
-  if (slot == 10 || slot == 11) timeline[i] = ~0ull;
+  if (slot >= 9 && slot <= 11) timeline[i] = ~0ull;
   else if (slot >= 12) timeline[i] = 0ull;
 }
 
