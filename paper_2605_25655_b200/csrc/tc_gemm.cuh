@@ -80,7 +80,7 @@ __host__ __device__ constexpr int tc_smem_bytes(int bn, int epi) {
   return tc_stages(bn, epi) * tc_stage_bytes(bn, epi) + tc_stage_out_bytes(bn) + 1024 /*alignment slack*/ + 512 /*barriers, 1/rms*/;
 }
 __host__ __device__ constexpr bool tc_epi_fp32_stage(int epi) {
-  return epi == EPI_RESID || epi == EPI_PLAIN_F32 || epi == EPI_SWIGLU_IL;
+  return epi == EPI_RESID || epi == EPI_PLAIN_F32 || epi == EPI_SWIGLU_IL || epi == EPI_QKV_ROPE;
 }
 // output features per tile: the interleaved gate/up tile produces 64 (its 128 rows are 64 gate + 64 up rows)
 __host__ __device__ constexpr int tc_tile_feats(int epi) { return epi == EPI_SWIGLU_IL ? 64 : kTcBM; }
@@ -170,51 +170,28 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
   __half* st16 = reinterpret_cast<__half*>(stage);
   float* st32 = reinterpret_cast<float*>(stage);
 
+  // RESID: the residual pieces this thread adds in phase B are requested now, so that their latency runs
+  // under phase A and the barrier instead of once per piece (the stores below may alias the loads as far
+  // as the compiler knows, so it would not move them up by itself)
+  constexpr int kPieces = (CW * 16 + 127) / 128;
+  uint4 rx[EPI == EPI_RESID ? kPieces : 1];
+  if (EPI == EPI_RESID && (e.ld_out & 7) == 0) {
+#pragma unroll
+    for (int it = 0; it < kPieces; ++it) {
+      const int idx = ethread + it * 128;
+      const int c = idx >> 4, piece = idx & 15;
+      const int r = tok_base + c, n0 = t.feat0 + piece * 8;
+      rx[it] = make_uint4(0, 0, 0, 0);
+      if (idx < CW * 16 && r < a.rows && a.n_feat[t.mat] - n0 >= 8) {
+        const __half* src = e.resid + static_cast<size_t>(r) * e.ld_out + n0;
+        rx[it] = a.static_finisher ? __ldcg(reinterpret_cast<const uint4*>(src))  // written earlier in the same kernel
+                                   : *reinterpret_cast<const uint4*>(src);        // written by an earlier kernel
+      }
+    }
+  }
+
   // ---------------- phase A
-  if (EPI == EPI_QKV_ROPE) {
-    const int i = (t.feat0 + row) % e.head_dim;  // element inside its head (tiles are 128-aligned, heads 64 or 128)
-    const int half = e.head_dim >> 1;
-    const bool rotate = t.mat != 2;
-    // all table reads of the chunk are issued before any is used: one L2 latency per chunk, not per column
-    float cs[CW], sn[CW];
-    if (e.pos_arr == nullptr) {  // uniform positions (prefill, equal-length decode): no load on the address path
-      int s = tok_base % e.seq_len;
-#pragma unroll
-      for (int c = 0; c < CW; ++c) {
-        cs[c] = 1.f;
-        sn[c] = 0.f;
-        if (rotate && tok_base + c < a.rows) {
-          const size_t o = static_cast<size_t>(e.pos0 + s) * half + (i >> 1);
-          cs[c] = __ldg(e.rope_cos + o);
-          sn[c] = __ldg(e.rope_sin + o);
-        }
-        if (++s == e.seq_len) s = 0;
-      }
-    } else {  // ragged decode: every request has its own position
-      int b = tok_base / e.seq_len, s = tok_base - b * e.seq_len;
-#pragma unroll
-      for (int c = 0; c < CW; ++c) {
-        cs[c] = 1.f;
-        sn[c] = 0.f;
-        if (rotate && tok_base + c < a.rows) {
-          const size_t o = static_cast<size_t>(e.pos0 + s + e.pos_arr[b]) * half + (i >> 1);
-          cs[c] = __ldg(e.rope_cos + o);
-          sn[c] = __ldg(e.rope_sin + o);
-        }
-        if (++s == e.seq_len) {
-          s = 0;
-          ++b;
-        }
-      }
-    }
-    const float sgn = (i & 1) ? 1.f : -1.f;
-#pragma unroll
-    for (int c = 0; c < CW; ++c) {
-      const float val = v[c];
-      const float partner = __shfl_xor_sync(0xffffffffu, val, 1);  // the other element of the (2j, 2j+1) pair
-      st16[c * kTcBM + row] = __float2half_rn(fmaf(sgn * partner, sn[c], val * cs[c]));
-    }
-  } else {
+  {
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
       if (F32) st32[c * kTcBM + row] = v[c];
@@ -253,7 +230,9 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
     return;
   }
 #pragma unroll
-  for (int idx = ethread; idx < CW * 16; idx += 128) {
+  for (int it = 0; it < kPieces; ++it) {
+    const int idx = ethread + it * 128;
+    if (idx >= CW * 16) break;
     const int c = idx >> 4, piece = idx & 15;
     const int r = tok_base + c;
     const int n0 = t.feat0 + piece * 8;  // first feature of the piece inside its matrix
@@ -269,7 +248,31 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
       else dst = (t.mat == 1 ? e.k_cache : e.v_cache) +
                  ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + e.pos0 + s +
                   (e.pos_arr != nullptr ? e.pos_arr[b] : 0)) * e.head_dim + i;
-      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(st16 + c * kTcBM + piece * 8);
+      // the 8 staged FP32 sums are 4 rotation pairs (2j, 2j+1) of one head: their cos / sin are 4 consecutive
+      // table entries, two 16-byte loads per piece (Algorithm 1; V rows are stored as they are)
+      const float* src = st32 + c * kTcBM + piece * 8;
+      float y[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) y[j] = src[j];
+      if (t.mat != 2) {
+        const int pos = e.pos0 + s + (e.pos_arr != nullptr ? e.pos_arr[b] : 0);
+        const size_t o = static_cast<size_t>(pos) * (e.head_dim >> 1) + (i >> 1);
+        const float4 cs = __ldg(reinterpret_cast<const float4*>(e.rope_cos + o));
+        const float4 sn = __ldg(reinterpret_cast<const float4*>(e.rope_sin + o));
+        const float c4[4] = {cs.x, cs.y, cs.z, cs.w}, s4[4] = {sn.x, sn.y, sn.z, sn.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float x0 = y[2 * j], x1 = y[2 * j + 1];
+          y[2 * j] = fmaf(-x1, s4[j], x0 * c4[j]);
+          y[2 * j + 1] = fmaf(x0, s4[j], x1 * c4[j]);
+        }
+      }
+      uint4 o16;
+      o16.x = pack2(y[0], y[1]);
+      o16.y = pack2(y[2], y[3]);
+      o16.z = pack2(y[4], y[5]);
+      o16.w = pack2(y[6], y[7]);
+      *reinterpret_cast<uint4*>(dst) = o16;
     } else {
       const size_t off = static_cast<size_t>(r) * e.ld_out + n0;
       const bool vec = valid == 8 && (e.ld_out & 7) == 0;
@@ -287,9 +290,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
         const float* src = st32 + c * kTcBM + piece * 8;
         if (vec) {
           float x[8];
-          unpack8(a.static_finisher ? __ldcg(reinterpret_cast<const uint4*>(e.resid + off))  // written earlier in the same kernel
-                                   : *reinterpret_cast<const uint4*>(e.resid + off),   // written by an earlier kernel: L1 is fine
-                  x);
+          unpack8(rx[it], x);  // requested before phase A
           uint4 o;
           o.x = pack2(x[0] + src[0], x[1] + src[1]);
           o.y = pack2(x[2] + src[2], x[3] + src[3]);
