@@ -85,6 +85,15 @@ def test_tiny_shapes_ragged(T, batch, seq, n_decode):
     _layer_case(T, synth.TINY, batch=batch, seq=seq, n_decode=n_decode, seed=batch)
 
 
+# the same small layer with every dimension a multiple of 64: decode of up to 16 requests runs on the skinny
+# projections (shares smaller than one 16-row tile, K shorter than the 8 warp slices, 1 .. 16 tokens, GQA)
+@pytest.mark.parametrize("batch,seq,n_decode,hkv", [(1, 32, 8, 4), (2, 1, 6, 4), (3, 130, 3, 2), (5, 77, 2, 1),
+                                                    (8, 33, 3, 4), (9, 20, 3, 2), (16, 40, 2, 4)])
+def test_small_layer_on_skinny_projections(T, batch, seq, n_decode, hkv):
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=hkv, head_dim=64, ffn=704)
+    _layer_case(T, shape, batch=batch, seq=seq, n_decode=n_decode, seed=batch)
+
+
 # ---- launch mode 2: the whole decode step in one cooperative persistent kernel ---------------------
 @pytest.mark.parametrize("batch,seq,n_decode", [(1, 32, 8), (2, 1, 6), (3, 130, 3), (16, 40, 3), (7, 5, 12)])
 def test_unified_decode_kernel_tiny(T, batch, seq, n_decode):
@@ -386,11 +395,12 @@ def test_launch_modes_agree_bit_for_bit(T, batch):
         np.testing.assert_array_equal(a, b)
 
 
-def test_prefill_and_decode_stages_on_two_streams(T):
+@pytest.mark.parametrize("ffn", [688, 704])
+def test_prefill_and_decode_stages_on_two_streams(T, ffn):
     # the Prefill -> Buffer -> Decode schedule on one device: slot 1 is being prefilled on one stream while slot 0
     # decodes on another; the hand-off events order each slot's stages; results equal the serial run bit for bit
     torch, thinfer = T
-    shape = synth.TINY
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64, ffn=ffn)
     w = synth.layer_weights(shape, 9)
     x = torch.from_numpy(synth.hidden_states(shape, 9, (2, 3, 40))).cuda()     # two micro-batches of 3 requests
 
@@ -427,11 +437,14 @@ def test_prefill_and_decode_stages_on_two_streams(T):
         np.testing.assert_array_equal(serial[k], overlapped[k], err_msg=k)
 
 
+# ffn 688 is not a multiple of 64: decode runs on the FMA GEMV (one request) / stream-K tensor-core path;
+# ffn 704 puts the same small layer on the skinny projections (per-request positions in their epilogue)
+@pytest.mark.parametrize("ffn", [688, 704])
 @pytest.mark.parametrize("lens,n_decode,mode", [((5, 17, 32), 4, 1), ((1, 64, 33, 7, 20), 3, 2), ((130,), 2, 1)])
-def test_ragged_prompts_layer(T, lens, n_decode, mode):
+def test_ragged_prompts_layer(T, lens, n_decode, mode, ffn):
     # prompts of different lengths in one batch: every request must equal the oracle run on that request alone
     torch, thinfer = T
-    shape = synth.TINY
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64, ffn=ffn)
     cfg = oracle_config(shape)
     w = synth.layer_weights(shape, 12)
     batch, pad = len(lens), max(lens)
@@ -458,9 +471,10 @@ def test_ragged_prompts_layer(T, lens, n_decode, mode):
     ctx.close()
 
 
-def test_ragged_prompts_stack_logits(T):
+@pytest.mark.parametrize("ffn", [688, 704])
+def test_ragged_prompts_stack_logits(T, ffn):
     torch, thinfer = T
-    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=688, n_layers=2, vocab=1000)
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=ffn, n_layers=2, vocab=1000)
     cfg = oracle_config(shape)
     sw = synth.stack_weights(shape, 13)
     lens = (9, 3, 14)
