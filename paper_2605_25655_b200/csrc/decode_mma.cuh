@@ -127,6 +127,11 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   const int nkb = a.k >> 6;                                  // k is a multiple of 64 (checked on the host)
   const int nkw = (nkb - warp + kSkWarps - 1) / kSkWarps;    // blocks warp, warp + 8, ...
 
+  // Every CTA starts its walk along K at a different block, so that the CTAs do not all read the same
+  // columns of their rows at the same time (the order of the sum is fixed per CTA all the same).
+  const int rot = nkw > 0 ? static_cast<int>(blockIdx.x) % nkw : 0;
+  auto rotated = [&](int blk) { return blk + rot < nkw ? blk + rot : blk + rot - nkw; };
+
   uint4* ring = reinterpret_cast<uint4*>(sk_smem) + warp * (ST * 128);  // [stage][16 rows][8 chunks]
   float* part = sk_smem;                                                // after the stream: [warp][TM][nt][4][32]
   float* ssq_in = sk_smem + kSkWarps * ST * 512;                        // [parts][16]
@@ -150,7 +155,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
       tb[tile] = a.w[m] + static_cast<size_t>(min(row00 + tile * 16 + crow, a.n[m] - 1)) * a.k + coop_off;
   }
   auto request = [&](int tile, int blk, int stage) {
-    const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
+    const size_t off = static_cast<size_t>(rotated(blk)) * (kSkWarps * 64);
     const uint32_t dst = coop_dst + stage * 2048;
     if (EPI == EPI_SWIGLU) {
       const size_t row0 = static_cast<size_t>(r_lo + tile * 8 + crow) * a.k + coop_off + off;
@@ -198,7 +203,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
                                      : nullptr;
   uint4 xq[XB][NT][2];
   auto load_x = [&](int blk, uint4 (&x)[NT][2]) {
-    const size_t off = static_cast<size_t>(blk) * (kSkWarps * 64);
+    const size_t off = static_cast<size_t>(rotated(blk)) * (kSkWarps * 64);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       x[nt][0] = xrow[nt] != nullptr ? ldg_cached(xrow[nt] + off) : zero;
@@ -231,7 +236,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
       if (i < nkw) {
         if (i + XB - 1 < nkw) load_x(i + XB - 1, xq[(b + XB - 1) % XB]);
         if (NORM) {
-          const size_t off = static_cast<size_t>(i) * (kSkWarps * 64);
+          const size_t off = static_cast<size_t>(rotated(i)) * (kSkWarps * 64);
           const uint4 g0 = ldg_cached(grow + off), g1 = ldg_cached(grow + off + 32);  // 8 KB in all: stays in L1
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
