@@ -325,20 +325,34 @@ bool opt_in_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+// The opt-in above is a per-device property of a kernel.  One of these (a function-local static per kernel
+// instantiation) remembers what has been reserved on which device, so that a process that drives several GPUs
+// opts in on each of them and a launch pays one cudaGetDevice instead of a driver call.
+struct SmemOptIn {
+  static constexpr int kMaxDevices = 64;
+  int reserved[kMaxDevices] = {};
+  template <typename K>
+  bool ensure(K kernel, int bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return opt_in_smem(kernel, bytes);
+    if (bytes <= reserved[dev]) return true;
+    if (!opt_in_smem(kernel, bytes)) return false;
+    reserved[dev] = bytes;
+    return true;
+  }
+};
+
 // ----------------------------------------------------------------------------
 // tcgen05 GEMM dispatch
 // ----------------------------------------------------------------------------
 template <int BN, int EPI>
 void launch_tc(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
                const CUtensorMap& x, const TcGemmArgs& a) {
-  static bool ready = false;  // per instantiation; contexts are created from one thread at a time
+  static SmemOptIn opt;
   constexpr int smem = tc_smem_bytes(BN, EPI);
-  if (!ready) {
-    if (!opt_in_smem(tc_gemm_kernel<BN, EPI>, smem)) {
-      L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
-      return;
-    }
-    ready = true;
+  if (!opt.ensure(tc_gemm_kernel<BN, EPI>, smem)) {
+    L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+    return;
   }
   const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
   const int n_tt = (a.rows + BN - 1) / BN;
@@ -491,14 +505,11 @@ int skinny_partition(const int (&n)[3], bool swiglu, int grid, int (&cta0)[4]) {
 
 template <int NT, int TM, int ST, int EPI, bool NORM>
 void launch_skinny_tm(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
-  static int reserved = 0;  // per instantiation; contexts are created from one thread at a time
+  static SmemOptIn opt;
   const int smem = sk_smem_floats(TM, ST, a.sumsq_parts) * 4;
-  if (smem > reserved) {
-    if (smem > 220 * 1024 || !opt_in_smem(skinny_mma_kernel<NT, TM, ST, EPI, NORM>, smem)) {
-      L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection needs %d bytes of shared memory", smem);
-      return;
-    }
-    reserved = smem;
+  if (smem > 220 * 1024 || !opt.ensure(skinny_mma_kernel<NT, TM, ST, EPI, NORM>, smem)) {
+    L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection needs %d bytes of shared memory", smem);
+    return;
   }
   L.go(kid, skinny_mma_kernel<NT, TM, ST, EPI, NORM>, dim3(grid), dim3(kSkWarps * 32), smem, a);
 }
@@ -615,14 +626,11 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
 template <int D>
 void attn_prefill_d(Launcher& L, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                     const AttnPreArgs& a, int batch) {
-  static bool ready = false;
+  static SmemOptIn opt;
   constexpr int smem = attn_pre_smem_bytes(D);
-  if (!ready) {
-    if (!opt_in_smem(attn_prefill_kernel<D>, smem)) {
-      L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
-      return;
-    }
-    ready = true;
+  if (!opt.ensure(attn_prefill_kernel<D>, smem)) {
+    L.rc = fail(L.c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+    return;
   }
   const int n_qt = (a.seq_len + kAttnBQ - 1) / kAttnBQ;
   L.go(THINFER_K_ATTN, attn_prefill_kernel<D>, dim3((n_qt + 1) / 2, a.n_q_heads, batch), dim3(kAttnThreads), smem, mq, mk, mv, a);
@@ -887,14 +895,11 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
 // ----------------------------------------------------------------------------
 template <int D, int G>
 void launch_mega(Launcher& L, thinfer_ctx* c, const MegaArgs& a) {
-  static bool ready = false;
+  static SmemOptIn opt;
   constexpr int smem = mega_smem_bytes<16, D, G>();
-  if (!ready) {
-    if (!opt_in_smem(decode_mega_kernel<16, D, G>, smem)) {
-      L.rc = fail(c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
-      return;
-    }
-    ready = true;
+  if (!opt.ensure(decode_mega_kernel<16, D, G>, smem)) {
+    L.rc = fail(c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+    return;
   }
   L.cooperative = true;
   L.go(THINFER_K_DECODE_UNIFIED, decode_mega_kernel<16, D, G>, dim3(c->sm_count < kTcMaxCtas ? c->sm_count : kTcMaxCtas),
