@@ -53,7 +53,7 @@ def measured_peaks():
 
 
 # --------------------------------------------------------------------------- #
-# algorithmic bytes / flops (stated in the design doc)
+# algorithmic bytes / flops of the workload
 # --------------------------------------------------------------------------- #
 def layer_weight_elems(s):
     qd, kvd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
