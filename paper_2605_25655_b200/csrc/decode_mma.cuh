@@ -1,26 +1,29 @@
 // Weight-streaming skinny GEMM for decode with up to 16 tokens (the small-M
 // path of Section 3.2.2 with the fusion units of Section 3.3.1).  The work is
-// bandwidth-bound: every weight is read from HBM exactly once, by a 128-bit
-// load that goes straight into the register fragment of a warp-level tensor
-// core instruction (mma.sync m16n8k16, FP16 in, FP32 accumulate), so that 16
-// tokens cost no more issue slots than one.
+// bandwidth-bound: every weight is read from HBM exactly once and is consumed by
+// a warp-level tensor-core instruction (mma.sync m16n8k16, FP16 in, FP32
+// accumulate), so that 16 tokens cost no more issue slots than one.
 //
 // Decomposition.  The output features are cut into one contiguous share per
 // CTA, balanced to within one feature pair over a grid that is a multiple of
 // the SM count: no wave quantisation and no partial sums that cross CTAs.  A
 // share is at most TM tiles of 16 weight rows.  The 8 warps of a CTA take the
-// 64-element blocks of K in turn (block b belongs to warp b mod 8); for its
-// block a warp loads the token fragment once and walks all tiles of the share
-// with it, one FP32 fragment per tile in registers.  After the stream the 8
-// fragments of a tile are added in warp order through shared memory (a fixed
-// order: results do not depend on timing) and the fused epilogue runs.
+// 64-element blocks of K in turn (block b belongs to warp b mod 8), every CTA
+// starting at a different block; for its block a warp loads the token fragment
+// once and walks all tiles of the share with it, one FP32 fragment per tile in
+// registers.  After the stream the 8 fragments of a tile are added in warp
+// order through shared memory (a fixed order: results do not depend on timing)
+// and the fused epilogue runs.
 //
 // Weights travel global -> shared memory by 16-byte asynchronous copies
-// (cp.async, no registers held) into a ring that is private to each lane: a
-// lane reads back exactly the bytes it requested, so the ring needs no barrier,
-// only cp.async.wait_group.  The ring is filled before the wait on the previous
-// kernel.  The kernel uses no tensor memory, so under programmatic dependent
-// launch CTAs of the next projection can be resident beside the running ones.
+// (cp.async, no registers held) into a ring of ST stages per warp.  The warp
+// copies a stage cooperatively, 4 rows x 128 contiguous bytes per instruction,
+// into a swizzled layout from which the MMA fragments are read without bank
+// conflicts; cp.async.wait_group plus a warp barrier on both sides of the reads
+// is all the synchronisation the ring needs.  The ring is filled before the
+// wait on the previous kernel.  The kernel uses no tensor memory, so under
+// programmatic dependent launch the CTAs of the next projection move in as the
+// CTAs of this one leave.
 #pragma once
 #include "epilogue.cuh"
 
