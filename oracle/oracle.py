@@ -27,7 +27,9 @@ What each function follows:
 
 Pins (tests/test_oracle_*.py): closed forms, brute-force loops on tiny inputs,
 invariants (RoPE norm / relative position, decode == last prefill row, batch
-independence) and torch CPU float64 library routines.  Hidden-state values at
+independence), torch CPU float64 library routines, and for the layer loop of
+stack_prefill / stack_decode a hand-chained composition of independent torch
+float64 layers with torch's embedding lookup, rms_norm and linear for the head.  Hidden-state values at
 the large configurations have no printed reference in the paper: they are
 pinned only through these functions ("parity unpinned by the paper" for the
 large-shape values themselves).
@@ -52,8 +54,9 @@ class Config:
 
 
 def f64(a):
-    """Exact widening of an FP16/FP32 array to float64."""
-    return np.asarray(a).astype(np.float64)
+    """Exact widening of an FP16/FP32 array to float64 (an array that already is
+    float64 is passed through, not copied)."""
+    return np.asarray(a).astype(np.float64, copy=False)
 
 
 # --------------------------------------------------------------------------- #

@@ -125,6 +125,74 @@ def test_stack_decode_continues_prefill():
     assert caches[0][0].shape == (2, SMALL_STACK.n_kv_heads, 9, SMALL_STACK.head_dim)
 
 
+def test_stack_loop_matches_a_composition_of_independent_torch_layers():
+    # pins the layer loop of the stack: embedding lookup, L independent torch float64 layers chained by hand,
+    # torch rms_norm + linear for the head.  The synthetic weights are scaled up so that every layer changes
+    # the hidden state by a large fraction of its size; a loop that reused layer 0's weights, skipped a layer
+    # or fed a layer the wrong hidden state fails here (and the variants below prove that this check can fail).
+    cfg = _cfg(SMALL_STACK)
+    sw = synth.stack_weights(SMALL_STACK, seed=21)
+    for w in sw["layers"]:
+        for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
+            w[n] = (w[n].astype(np.float32) * 8).astype(np.float16)
+    ids = synth.token_ids(SMALL_STACK, 21, (2, 7))
+    logits, nxt, caches, hid = O.stack_prefill(cfg, sw, ids)
+
+    F = torch.nn.functional
+    x = torch.from_numpy(sw["embed"].astype(np.float64))[torch.from_numpy(ids.astype(np.int64))].numpy()
+    per_layer = []
+    for l, w in enumerate(sw["layers"]):
+        x_prev = x
+        x, k, v = _torch_layer(SMALL_STACK, w, x)
+        per_layer.append(x)
+        np.testing.assert_allclose(hid[l], x, rtol=1e-9, atol=1e-11, err_msg=f"hidden state after layer {l}")
+        np.testing.assert_allclose(caches[l][0], k, rtol=1e-9, atol=1e-11, err_msg=f"K cache of layer {l}")
+        np.testing.assert_allclose(caches[l][1], v, rtol=1e-9, atol=1e-11, err_msg=f"V cache of layer {l}")
+        # the layers are far from the identity and from each other, so the comparisons above can tell them apart
+        assert np.linalg.norm(x - x_prev) > 0.05 * np.linalg.norm(x_prev)
+    hn = F.rms_norm(torch.from_numpy(x[:, -1]), (SMALL_STACK.hidden,),
+                    torch.from_numpy(sw["final_norm"].astype(np.float64)), eps=cfg.rms_eps)
+    ref_logits = F.linear(hn, torch.from_numpy(sw["lm_head"].astype(np.float64))).numpy()
+    np.testing.assert_allclose(logits, ref_logits, rtol=1e-9, atol=1e-11)
+    np.testing.assert_array_equal(nxt, np.argmax(ref_logits, axis=-1))
+
+    # the mistakes this pin is there to catch do change the result: layer 0's weights used everywhere,
+    # and two layers swapped
+    wrong = dict(sw, layers=[sw["layers"][0]] * 3)
+    _, _, _, hid_wrong = O.stack_prefill(cfg, wrong, ids)
+    assert not np.allclose(hid_wrong[1], per_layer[1], rtol=1e-3, atol=1e-6)
+    swapped = dict(sw, layers=[sw["layers"][1], sw["layers"][0], sw["layers"][2]])
+    _, _, _, hid_swapped = O.stack_prefill(cfg, swapped, ids)
+    assert not np.allclose(hid_swapped[2], per_layer[2], rtol=1e-3, atol=1e-6)
+
+    # the decode loop: one more token through stack_decode equals the torch composition over 8 tokens
+    ids8 = np.concatenate([ids, synth.token_ids(SMALL_STACK, 22, (2, 1))], axis=1)
+    lg_dec, _, caches2, hid_dec = O.stack_decode(cfg, sw, ids8[:, 7], caches, 7)
+    x = torch.from_numpy(sw["embed"].astype(np.float64))[torch.from_numpy(ids8.astype(np.int64))].numpy()
+    for l, w in enumerate(sw["layers"]):
+        x, k, v = _torch_layer(SMALL_STACK, w, x)
+        np.testing.assert_allclose(hid_dec[l], x[:, -1], rtol=1e-8, atol=1e-10, err_msg=f"decode hidden, layer {l}")
+        np.testing.assert_allclose(caches2[l][0], k, rtol=1e-8, atol=1e-10)
+    hn = F.rms_norm(torch.from_numpy(x[:, -1]), (SMALL_STACK.hidden,),
+                    torch.from_numpy(sw["final_norm"].astype(np.float64)), eps=cfg.rms_eps)
+    np.testing.assert_allclose(lg_dec, F.linear(hn, torch.from_numpy(sw["lm_head"].astype(np.float64))).numpy(),
+                               rtol=1e-8, atol=1e-10)
+
+
+def test_oracle_accepts_float64_inputs_without_changing_results():
+    # weights that were widened to float64 beforehand (the large-configuration tests do that once per layer)
+    # give bit-identical results to the FP16 arrays they came from
+    cfg = _cfg(SMALL)
+    w = synth.layer_weights(SMALL, seed=4)
+    x = synth.hidden_states(SMALL, 4, (2, 6))
+    a, ka, va = O.layer_prefill(cfg, w, x)
+    w64 = {k: v.astype(np.float64) for k, v in w.items()}
+    b, kb, vb = O.layer_prefill(cfg, w64, x.astype(np.float64))
+    np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(ka, kb)
+    np.testing.assert_array_equal(va, vb)
+
+
 def test_stack_embedding_and_head():
     # zero projections everywhere: hidden == embedding row; logits = head(RMSNorm(embedding row))
     cfg = _cfg(SMALL_STACK)
