@@ -1,21 +1,24 @@
 #!/usr/bin/env python
-"""Benchmark of the hot path: one Llama-7B-shaped decoder layer, FP16, on B200.
+"""Benchmark of the hot path on B200: FP16 Llama-shaped decoder stacks, prefill then greedy decode.
 
-A step = one pass of the whole path over one batch of synthetic input:
-prefill of `batch` prompts of 512 tokens, then 128 decode steps over the FP16
-KV cache.  The headline value is decode tokens/s (batch x 128 / decode time);
-prefill tokens/s and both roofline fractions are reported beside it.
+A step = one pass of the whole path over one batch of synthetic input: prefill of `batch` prompts (which
+emits the first token), then the remaining tokens one decode step at a time over the FP16 KV cache, the ids
+fed back on the device.  The headline value is decode tokens/s; prefill tokens/s, the paper-style end-to-end
+rate (batch x generated / total latency, Section 3.4.1) and the roofline fractions are reported beside it.
 
-  python bench.py --gpus 1 --steps K --warmup W          # this library
-  python bench.py --impl reference ...                    # the CPU oracle, timed on the host cores
+  python bench.py --gpus 1 --steps K --warmup W            # this library, configuration 5 (70B stack)
+  python bench.py --config {c2,c3,c4,c5} ...               # 7B layer / 7B stack / 13B stack / 70B stack
+  python bench.py --impl reference ...                      # the CPU oracle, timed on the host cores
+  python bench.py --tables                                  # operator latencies at the paper's Table 8 / 9 shapes
+  python bench.py --profile {prefill,decode} --config cX    # one layer of that configuration: the case ncu captures
 
-With N > 1 (under torchrun) every rank runs an independent replica of the same
-workload on its own GPU: the path has no exchange step, so there is no
-collective on the data path; times are the maximum over ranks.
+With N > 1 (under torchrun) every rank runs an independent replica of the same workload on its own GPU: the
+path has no exchange step, so there is no collective on the data path; times are the maximum over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -30,16 +33,54 @@ sys.path.insert(0, ROOT)
 
 from paper_2605_25655_b200 import synth  # noqa: E402
 
-PROMPT = 512
-GEN = 128
-SHAPE = synth.LLAMA_7B_LAYER
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_GBS = 8000.0       # the HBM3e figure the target bars are quoted against
+NOMINAL_TFLOPS = 2250.0    # dense FP16 / BF16 tensor peak
 
 
-def captured_traffic(key, batch):
-    """DRAM bytes per launch from the committed ncu capture (batch 16 only; None otherwise)."""
-    path = os.path.join(ROOT, "paper_2605_25655_b200", "ncu_traffic.json")
-    if batch != 16 or not os.path.exists(path):
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    key: str
+    shape: synth.Shape
+    batch: int
+    prompt: int
+    gen: int            # stack: tokens generated per request (1 by the prefill, gen - 1 by decode steps);
+    label: str          # layer-only: decode steps on seeded hidden states
+
+    @property
+    def stack(self):
+        return self.shape.vocab > 0
+
+    @property
+    def decode_steps(self):
+        return self.gen - 1 if self.stack else self.gen
+
+    def name(self, batch=None):
+        b = self.batch if batch is None else batch
+        s = self.shape
+        heads = f"{s.n_q_heads}x{s.head_dim} MHA" if s.n_q_heads == s.n_kv_heads else \
+            f"{s.n_q_heads} query / {s.n_kv_heads} KV heads x {s.head_dim} (GQA)"
+        if self.stack:
+            return (f"{self.label} full stack ({s.n_layers} layers, hidden {s.hidden}, {heads}, FFN {s.ffn}, vocab "
+                    f"{s.vocab}), FP16, batch {b}, prompt {self.prompt}, {self.gen} tokens generated greedily")
+        return (f"{self.label} single decoder layer (hidden {s.hidden}, {heads}, FFN {s.ffn}), FP16, batch {b}, "
+                f"prompt {self.prompt}, {self.gen} decode steps")
+
+
+WORKLOADS = {
+    "c2": Workload("c2", synth.LLAMA_7B_LAYER, 16, 512, 128, "Llama-7B-shaped"),
+    "c3": Workload("c3", synth.LLAMA_7B, 8, 512, 256, "Llama-7B-shaped"),
+    "c4": Workload("c4", synth.LLAMA_13B, 16, 1024, 256, "Llama-13B-shaped"),
+    "c5": Workload("c5", synth.LLAMA_70B, 4, 512, 128, "Llama-2-70B-shaped"),
+}
+DEFAULT_WORKLOAD = "c5"    # the largest configuration that fits one GPU (138 GB of weights)
+
+
+def captured_traffic(key):
+    """DRAM bytes per launch from the committed ncu captures (profiles/ncu_traffic.json); None when the
+    kernel of this workload has no capture."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
         return None
     return json.load(open(path)).get(key, {}).get("traffic_bytes")
 
@@ -61,21 +102,26 @@ def layer_weight_elems(s):
 
 
 def decode_step_bytes(s, batch, t_len):
-    """Weights once + gains, KV read (t_len keys) and append, activations in/out."""
+    """One decode step of the whole model.  Per layer: weights once + gains, KV read (t_len keys) and append;
+    plus activations in/out and, for a stack, the vocabulary projection, the final gain and the embedding rows."""
     kv = batch * 2 * t_len * s.n_kv_heads * s.head_dim * 2
     app = batch * 2 * s.n_kv_heads * s.head_dim * 2
-    act = batch * s.hidden * 2 * 2
-    return 2 * layer_weight_elems(s) + 2 * 2 * s.hidden + kv + app + act
+    per_layer = 2 * layer_weight_elems(s) + 2 * 2 * s.hidden + kv + app
+    total = s.n_layers * per_layer + batch * s.hidden * 2 * 2
+    if s.vocab > 0:
+        total += 2 * s.vocab * s.hidden + 2 * s.hidden + batch * s.vocab * 4
+    return total
 
 
 def gateup_gemv_bytes(s, batch):
     return 2 * (2 * s.ffn * s.hidden) + 2 * s.hidden + batch * s.hidden * 2 + batch * s.ffn * 2
 
 
-def prefill_flops(s, rows, seq):
-    gemm = 2.0 * rows * layer_weight_elems(s)
-    attn = 2.0 * rows * seq * s.head_dim * s.n_q_heads      # causal: QK^T and PV, half of 4*S^2*d
-    return gemm, attn
+def prefill_flops(s, rows, seq, batch):
+    gemm = 2.0 * rows * layer_weight_elems(s) * s.n_layers
+    attn = 2.0 * rows * seq * s.head_dim * s.n_q_heads * s.n_layers   # causal: QK^T and PV, half of 4*S^2*d
+    head = 2.0 * batch * s.vocab * s.hidden
+    return gemm, attn, head
 
 
 def gateup_gemm_flops(s, rows):
@@ -133,23 +179,43 @@ class ClockSampler:
 # --------------------------------------------------------------------------- #
 # oracle legs (host cores)
 # --------------------------------------------------------------------------- #
-def _oracle_sample(batch, n_steps, seed=0):
-    """Times the oracle, as it stands, on `n_steps` decode steps of the workload (KV length PROMPT)."""
+def _oracle_sample(wl, batch, n_steps, seed=0):
+    """Times the oracle, as it stands, on a bounded sample of the decode workload: `n_steps` decode steps of ONE
+    layer at KV length wl.prompt, and (stack configurations) as many calls of the final norm + vocabulary
+    projection.  Returns (seconds per layer step, seconds per head call) lists."""
     from oracle import oracle as O
-    cfg = O.Config(hidden=SHAPE.hidden, n_q_heads=SHAPE.n_q_heads, n_kv_heads=SHAPE.n_kv_heads,
-                   head_dim=SHAPE.head_dim, ffn=SHAPE.ffn)
-    w = synth.layer_weights(SHAPE, seed)
+    s = wl.shape
+    cfg = O.Config(hidden=s.hidden, n_q_heads=s.n_q_heads, n_kv_heads=s.n_kv_heads, head_dim=s.head_dim, ffn=s.ffn)
+    w = synth.layer_weights(s, seed)
     rng = np.random.default_rng(seed)
-    kc = rng.standard_normal((batch, SHAPE.n_kv_heads, PROMPT, SHAPE.head_dim)).astype(np.float16)
-    vc = rng.standard_normal((batch, SHAPE.n_kv_heads, PROMPT, SHAPE.head_dim)).astype(np.float16)
-    x = synth.hidden_states(SHAPE, seed, (batch, n_steps))
-    times = []
+    kc = rng.standard_normal((batch, s.n_kv_heads, wl.prompt, s.head_dim)).astype(np.float16)
+    vc = rng.standard_normal((batch, s.n_kv_heads, wl.prompt, s.head_dim)).astype(np.float16)
+    x = synth.hidden_states(s, seed, (batch, n_steps))
+    sw = None
+    if wl.stack:
+        sw = {"final_norm": synth.stack_tensor(s, seed, "final_norm"), "lm_head": synth.stack_tensor(s, seed, "lm_head")}
+    layer_s, head_s = [], []
     k, v = kc, vc
     for i in range(n_steps):
         t0 = time.perf_counter()
-        _, k, v = O.layer_decode(cfg, w, x[:, i], k, v, PROMPT + i)
-        times.append(time.perf_counter() - t0)
-    return times
+        y, k, v = O.layer_decode(cfg, w, x[:, i], k, v, wl.prompt + i)
+        layer_s.append(time.perf_counter() - t0)
+        if sw is not None:
+            t0 = time.perf_counter()
+            O.argmax_lowest(O.head_logits(cfg, sw, y))
+            head_s.append(time.perf_counter() - t0)
+        else:
+            head_s.append(0.0)
+    return layer_s, head_s
+
+
+def _oracle_sample_text(wl, batch, n):
+    s = wl.shape
+    if wl.stack:
+        return (f"{n} oracle decode steps of ONE layer (+ final norm, vocabulary projection, argmax) at batch {batch}, "
+                f"KV length {wl.prompt}; a model step is taken as {s.n_layers} x the layer time + the head time "
+                f"(one step = {batch} tokens)")
+    return f"{n} oracle decode steps of batch {batch} at KV length {wl.prompt} (one step = {batch} tokens)"
 
 
 def host_threads():
@@ -163,21 +229,23 @@ def host_threads():
     return os.cpu_count()
 
 
-def run_reference(args):
+def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    times = _oracle_sample(args.batch, args.warmup + args.steps)
-    timed = times[args.warmup:]
-    total = sum(timed)
-    value = args.batch * len(timed) / total
-    sample = f"{len(timed)} oracle decode steps of batch {args.batch} at KV length {PROMPT} (one step = {args.batch} tokens)"
+    B = args.batch or wl.batch
+    layer_s, head_s = _oracle_sample(wl, B, args.warmup + args.steps)
+    L = wl.shape.n_layers
+    step_s = [L * a + b for a, b in zip(layer_s, head_s)][args.warmup:]
+    total = sum(step_s)
+    value = B * len(step_s) / total
     line = {
         "impl": "reference", "metric": "decode_tokens_per_s", "value": value, "unit": "tok/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(timed),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(step_s),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args.batch), "batch": args.batch, "prompt": PROMPT, "generate": GEN},
-        "cpu_baseline": {"value": value, "unit": "tok/s", "cores": host_threads(), "kind": "oracle", "sample": sample},
+        "config": {"workload": wl.name(B), "batch": B, "prompt": wl.prompt, "generate": wl.gen},
+        "cpu_baseline": {"value": value, "unit": "tok/s", "cores": host_threads(), "kind": "oracle",
+                         "sample": _oracle_sample_text(wl, B, len(step_s))},
         "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -199,15 +267,96 @@ def whole_job_rate(units_per_rank, world, seconds):
     return world * units_per_rank / seconds
 
 
-def workload_name(batch):
-    return (f"Llama-7B-shaped single decoder layer (hidden 4096, 32x128 MHA, FFN 11008), FP16, batch {batch}, "
-            f"prompt {PROMPT}, {GEN} decode steps")
-
-
 # --------------------------------------------------------------------------- #
 # this library
 # --------------------------------------------------------------------------- #
-def run_ours(args):
+class Runner:
+    """One workload on one device: weights, context, inputs, and the step functions the legs time."""
+
+    def __init__(self, wl, batch, dev, torch, thinfer):
+        self.wl, self.B, self.dev, self.torch, self.thinfer = wl, batch, dev, torch, thinfer
+        s, B = wl.shape, batch
+        self.steps_dec = wl.decode_steps
+        max_seq = wl.prompt + wl.decode_steps
+        if wl.stack:
+            sw = synth.device_stack_weights(s, seed=0, device=dev)
+            self.sw = sw
+            self.ctx = thinfer.Context(s, sw["layers"], {n: sw[n] for n in ("embed", "final_norm", "lm_head")},
+                                       max_batch=B, max_seq=max_seq, device=dev)
+            ids = synth.token_ids(s, 0, (B, wl.prompt))
+            self.h_prompt = torch.from_numpy(ids).pin_memory()
+            self.prompt = self.h_prompt.to(dev)
+            self.id_buf = [torch.zeros(B, dtype=torch.int32, device=dev) for _ in range(2)]
+            self.h_ids = torch.zeros(B, dtype=torch.int32).pin_memory()
+            self.h_ids_out = torch.zeros(B, dtype=torch.int32).pin_memory()
+            self.h2d, self.d2h = B * 4, B * 4
+        else:
+            self.layers = thinfer.to_device_layers([synth.layer_weights(s, seed=0)], device=dev)
+            self.ctx = thinfer.Context(s, self.layers, None, max_batch=B, max_seq=max_seq, device=dev)
+            x_all = torch.from_numpy(synth.hidden_states(s, 0, (B, wl.prompt + wl.gen)))
+            self.h_prompt = x_all[:, :wl.prompt].contiguous().pin_memory()
+            self.prompt = self.h_prompt.to(dev)
+            self.h_prompt_out = torch.empty_like(self.h_prompt).pin_memory()
+            self.h_dec = [x_all[:, wl.prompt + i].contiguous().pin_memory() for i in range(wl.gen)]
+            self.x_dec = [t.to(dev) for t in self.h_dec]
+            self.out_dec = torch.empty(B, s.hidden, dtype=torch.float16, device=dev)
+            self.h_dec_out = torch.empty(B, s.hidden, dtype=torch.float16).pin_memory()
+            self.h2d, self.d2h = B * s.hidden * 2, B * s.hidden * 2
+
+    def prefill(self):
+        if self.wl.stack:
+            return self.ctx.prefill(self.prompt)
+        self.ctx.prefill(self.prompt)
+        return None
+
+    def decode(self, first_ids, n_steps=None):
+        n = self.steps_dec if n_steps is None else n_steps
+        if self.wl.stack:
+            cur = first_ids
+            for i in range(n):
+                cur = self.ctx.decode_step(cur, out=self.id_buf[i & 1])     # ids stay on the device
+            return cur
+        for i in range(n):
+            self.ctx.decode_step(self.x_dec[i], out=self.out_dec)
+        return None
+
+    def one_step(self, events=None):
+        if events:
+            events[0].record()
+        first = self.prefill()
+        if events:
+            events[1].record()
+        self.decode(first)
+        if events:
+            events[2].record()
+        self.ctx.release_slot(0)
+
+    def one_step_host(self):
+        """The same step through the host-buffer entry points: every decode step copies its input from pinned
+        host memory, copies its result back, and the host reads it before it issues the next step."""
+        torch, ctx = self.torch, self.ctx
+        if self.wl.stack:
+            ctx.prefill_host(self.h_prompt, self.h_ids_out)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(self.steps_dec):
+                self.h_ids.copy_(self.h_ids_out)                  # the token just read is the next input
+                ctx.decode_step_host(self.h_ids, self.h_ids_out)
+                torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+        else:
+            ctx.prefill_host(self.h_prompt, self.h_prompt_out)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for i in range(self.steps_dec):
+                ctx.decode_step_host(self.h_dec[i], self.h_dec_out)
+                torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+        ctx.release_slot(0)
+        return dt
+
+
+def run_ours(args, wl):
     import torch
     from paper_2605_25655_b200 import thinfer
 
@@ -222,29 +371,12 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
-    B = args.batch
+    B = args.batch or wl.batch
+    S, s = wl.prompt, wl.shape
     peaks, peak_kind = measured_peaks()
-
-    w_np = synth.layer_weights(SHAPE, seed=0)
-    layers = thinfer.to_device_layers([w_np], device=dev)
-    x_np = synth.hidden_states(SHAPE, 0, (B, PROMPT + GEN))
-    x_all = torch.from_numpy(x_np)
-    x_prompt = x_all[:, :PROMPT].contiguous().to(dev)
-    x_dec = [x_all[:, PROMPT + i].contiguous().to(dev) for i in range(GEN)]
-    ctx = thinfer.Context(SHAPE, layers, None, max_batch=B, max_seq=PROMPT + GEN, buf_slots=1, device=dev)
-    out_dec = torch.empty(B, SHAPE.hidden, dtype=torch.float16, device=dev)
-
-    def one_step(events=None):
-        if events:
-            events[0].record()
-        ctx.prefill(x_prompt)
-        if events:
-            events[1].record()
-        for i in range(GEN):
-            ctx.decode_step(x_dec[i], out=out_dec)
-        if events:
-            events[2].record()
-        ctx.release_slot(0)
+    R = Runner(wl, B, dev, torch, thinfer)
+    ctx = R.ctx
+    n_dec = wl.decode_steps
 
     def sync_all():
         torch.cuda.synchronize()
@@ -253,7 +385,7 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     for _ in range(args.warmup):
-        one_step()
+        R.one_step()
     sync_all()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     sampler = ClockSampler(local)
@@ -263,8 +395,8 @@ def run_ours(args):
     launches0 = ctx.launch_count()
     sync_all()
     wall0 = time.perf_counter()
-    for s in range(args.steps):
-        one_step(evs[s])
+    for i in range(args.steps):
+        R.one_step(evs[i])
     sync_all()
     wall = time.perf_counter() - wall0
     launches = ctx.launch_count() - launches0
@@ -277,28 +409,12 @@ def run_ours(args):
     pre_ms, dec_ms, tot_ms = reduce_max_over_ranks([pre_ms, dec_ms, tot_ms], dist, dev)
 
     # ---- end to end through the host-buffer entry points (pinned memory, copies inside the timed region)
-    h_prompt = x_all[:, :PROMPT].contiguous().pin_memory()
-    h_prompt_out = torch.empty_like(h_prompt).pin_memory()
-    h_dec = [x_all[:, PROMPT + i].contiguous().pin_memory() for i in range(GEN)]
-    h_dec_out = torch.empty(B, SHAPE.hidden, dtype=torch.float16).pin_memory()
-
-    def one_step_host():
-        ctx.prefill_host(h_prompt, h_prompt_out)
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for i in range(GEN):
-            ctx.decode_step_host(h_dec[i], h_dec_out)
-            torch.cuda.synchronize()          # the caller reads each step's result before the next one
-        dt = time.perf_counter() - t0
-        ctx.release_slot(0)
-        return dt
-
-    one_step_host()
-    e2e_s = sum(one_step_host() for _ in range(max(1, min(args.steps, 3))))
-    e2e_steps = max(1, min(args.steps, 3))
+    e2e_steps = max(1, min(args.steps, 2 if wl.stack else 3))
+    R.one_step_host()
+    e2e_s = sum(R.one_step_host() for _ in range(e2e_steps))
     e2e_s = reduce_max_over_ranks([e2e_s], dist, dev)[0]
 
-    # ---- dominant kernels, timed with CUDA events around each of their launches
+    # ---- dominant kernels (gate/up projection), timed with CUDA events around each of their own launches
     def kernel_time(kid, fn):
         ctx.profile_select(kid)
         fn()
@@ -307,65 +423,77 @@ def run_ours(args):
         ctx.profile_select(-1)
         return n, ms
 
-    def decode_only():
-        ctx.prefill(x_prompt)
-        for i in range(GEN):
-            ctx.decode_step(x_dec[i], out=out_dec)
-        ctx.release_slot(0)
-
-    n_gu, ms_gu = kernel_time(thinfer.K_GATEUP, decode_only)     # 1 prefill launch + GEN decode launches
-    ctx.profile_select(thinfer.K_GATEUP)
-    ctx.prefill(x_prompt)
+    first = R.prefill()                                   # untimed: fills the slot for the decode sample
     torch.cuda.synchronize()
-    n_pre, ms_pre_gu = ctx.profile_read()
-    ctx.profile_select(-1)
+    k_steps = min(n_dec, 8)
+    n_dgu, ms_dgu = kernel_time(thinfer.K_GATEUP, lambda: R.decode(first, k_steps))
     ctx.release_slot(0)
-    ms_dec_gu = (ms_gu - ms_pre_gu) / max(1, n_gu - n_pre)
-    ms_pre_gu = ms_pre_gu / max(1, n_pre)
+    n_pgu, ms_pgu = kernel_time(thinfer.K_GATEUP, R.prefill)
+    ctx.release_slot(0)
+    ms_dec_gu = ms_dgu / max(1, n_dgu)
+    ms_pre_gu = ms_pgu / max(1, n_pgu)
 
-    pre_tokens = world * B * PROMPT * args.steps
-    value = whole_job_rate(B * GEN * args.steps, world, dec_ms * 1e-3)
-    dec_bytes = sum(decode_step_bytes(SHAPE, B, PROMPT + i + 1) for i in range(GEN))
+    pre_tokens = world * B * S * args.steps
+    value = whole_job_rate(B * n_dec * args.steps, world, dec_ms * 1e-3)
+    dec_bytes = sum(decode_step_bytes(s, B, S + i + 1) for i in range(n_dec))
     dec_gbs = dec_bytes * args.steps / (dec_ms * 1e-3) / 1e9
-    gemm_fl, attn_fl = prefill_flops(SHAPE, B * PROMPT, PROMPT)
-    pre_tflops = (gemm_fl + attn_fl) * args.steps / (pre_ms * 1e-3) / 1e12
+    gemm_fl, attn_fl, head_fl = prefill_flops(s, B * S, S, B)
+    pre_tflops = (gemm_fl + attn_fl + head_fl) * args.steps / (pre_ms * 1e-3) / 1e12
     hbm_peak = float(peaks["hbm_gbs"])
-    tc_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-    gu_gbs = gateup_gemv_bytes(SHAPE, B) / (ms_dec_gu * 1e-3) / 1e9
-    gu_tflops = gateup_gemm_flops(SHAPE, B * PROMPT) / (ms_pre_gu * 1e-3) / 1e12
+    tc_sustained = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    tc_burst = float(peaks["bf16_tflops"])
+    gu_gbs = gateup_gemv_bytes(s, B) / (ms_dec_gu * 1e-3) / 1e9
+    gu_tflops = gateup_gemm_flops(s, B * S) / (ms_pre_gu * 1e-3) / 1e12
+    weights_gb = synth.model_bytes(s) / 1e9 if wl.stack else 2 * layer_weight_elems(s) / 1e9
+    tc_pre_rows = "tc_gemm_kernel<256, SWIGLU interleaved>" if B * S > 64 else "tc_gemm_kernel<SWIGLU>"
+    dec_kernel = ("skinny_mma_kernel<SWIGLU>" if B <= 16 else "tc_gemm_kernel<32..64, SWIGLU> stream-K")
 
     line = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-        "config": {"workload": workload_name(B), "batch": B, "prompt": PROMPT, "generate": GEN,
-                   "value_is": "batch x generate / decode-phase time; ms_per_step covers prefill + decode",
-                   "l2": "no flush: the 405 MB of layer weights streamed by every decode step and the prefill "
+        "config": {"workload": wl.name(B), "key": wl.key, "batch": B, "prompt": S, "generate": wl.gen,
+                   "decode_steps_per_pass": n_dec,
+                   "value_is": "batch x decode steps / decode-phase time; ms_per_step covers prefill + decode",
+                   "l2": f"no flush: the {weights_gb:.1f} GB of weights streamed by every decode step and the prefill "
                          "activations exceed the 126 MB L2",
                    "multi_gpu": "independent replicas, no collective"},
-        "decode": {"ms_per_token_step": dec_ms / (args.steps * GEN), "achieved_GBs": dec_gbs,
-                   "frac_of_hbm_peak": dec_gbs / hbm_peak, "peak_GBs": hbm_peak, "peak_kind": peak_kind},
+        "decode": {"ms_per_token_step": dec_ms / (args.steps * n_dec), "algorithmic_bytes_per_pass": dec_bytes,
+                   "achieved_GBs": dec_gbs, "frac_of_hbm_peak": dec_gbs / hbm_peak, "peak_GBs": hbm_peak,
+                   "peak_kind": peak_kind, "frac_of_nominal_peak": dec_gbs / NOMINAL_GBS, "nominal_GBs": NOMINAL_GBS},
         "prefill": {"value": pre_tokens / (pre_ms * 1e-3), "unit": "tok/s", "ms": pre_ms / args.steps,
-                    "achieved_TFLOPs": pre_tflops, "frac_of_tensor_peak": pre_tflops / tc_peak,
-                    "peak_TFLOPs": tc_peak, "peak_kind": peak_kind + " bf16 sustained (same tensor-pipe rate as fp16)"},
-        "roofline": {"kernel": ("skinny_mma_kernel<SWIGLU>" if B <= 16 else "tc_gemm_kernel<32..64, SWIGLU> stream-K")
-                     + " (decode gate/up projection)", "bound": "hbm",
+                    "achieved_TFLOPs": pre_tflops, "frac_of_tensor_peak": pre_tflops / tc_sustained,
+                    "peak_TFLOPs": tc_sustained,
+                    "peak_kind": peak_kind + " bf16 sustained (same tensor-pipe rate as fp16)",
+                    "frac_of_nominal_peak": pre_tflops / NOMINAL_TFLOPS, "nominal_TFLOPs": NOMINAL_TFLOPS},
+        "end_to_end_paper_style": {"value": world * B * wl.gen * args.steps / (tot_ms * 1e-3), "unit": "tok/s",
+                                   "is": "batch x generated tokens / (prefill + decode) time, Section 3.4.1"},
+        "roofline": {"kernel": dec_kernel + " (decode gate/up projection)", "bound": "hbm",
                      "achieved": gu_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gu_gbs / hbm_peak,
-                     "traffic": captured_traffic("decode_gateup_b16", B), "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3,
-                     "algorithmic_bytes": gateup_gemv_bytes(SHAPE, B)},
-        "roofline_prefill": {"kernel": "tc_gemm_kernel<256, SWIGLU interleaved> (prefill gate/up projection)", "bound": "tensor",
-                             "achieved": gu_tflops, "peak": tc_peak, "unit": "TFLOP/s", "frac": gu_tflops / tc_peak,
-                             "traffic": captured_traffic("prefill_gateup_b16", B), "peak_kind": peak_kind, "avg_us": ms_pre_gu * 1e3},
-        "e2e": {"value": world * B * GEN * e2e_steps / e2e_s, "unit": "tok/s",
-                "h2d_bytes_per_step": B * SHAPE.hidden * 2, "d2h_bytes_per_step": B * SHAPE.hidden * 2,
-                "note": "per decode step: pinned host input -> device, layer, result -> host, stream synchronised"},
+                     "traffic": captured_traffic(f"decode_gateup_{wl.key}_b{B}"),
+                     "traffic_kind": "captured (committed profile of the same launch, profiles/ncu_traffic.json)",
+                     "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3, "launches_timed": n_dgu,
+                     "algorithmic_bytes": gateup_gemv_bytes(s, B), "frac_of_nominal_peak": gu_gbs / NOMINAL_GBS},
+        "roofline_prefill": {"kernel": tc_pre_rows + " (prefill gate/up projection)", "bound": "tensor",
+                             "achieved": gu_tflops, "peak": tc_burst, "unit": "TFLOP/s", "frac": gu_tflops / tc_burst,
+                             "traffic": captured_traffic(f"prefill_gateup_{wl.key}_b{B}"),
+                             "traffic_kind": "captured (committed profile of the same launch, profiles/ncu_traffic.json)",
+                             "peak_kind": peak_kind + " bf16 burst (the kernel is timed alone)",
+                             "avg_us": ms_pre_gu * 1e3, "launches_timed": n_pgu,
+                             "frac_of_sustained": gu_tflops / tc_sustained,
+                             "frac_of_nominal_peak": gu_tflops / NOMINAL_TFLOPS},
+        "e2e": {"value": world * B * n_dec * e2e_steps / e2e_s, "unit": "tok/s",
+                "h2d_bytes_per_step": R.h2d, "d2h_bytes_per_step": R.d2h,
+                "note": "per decode step: pinned host input -> device, all layers, result -> host, stream synchronised; "
+                        "the host feeds the token it read back in"},
         "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n = 4
-        times = _oracle_sample(B, n)
-        line["cpu_baseline"] = {"value": B * n / sum(times), "unit": "tok/s", "cores": host_threads(), "kind": "oracle",
-                                "sample": f"{n} oracle decode steps of batch {B} at KV length {PROMPT}"}
+        n = 3 if wl.stack else 4
+        layer_s, head_s = _oracle_sample(wl, B, n)
+        step = s.n_layers * sum(layer_s) / n + sum(head_s) / n
+        line["cpu_baseline"] = {"value": B / step, "unit": "tok/s", "cores": host_threads(), "kind": "oracle",
+                                "sample": _oracle_sample_text(wl, B, n)}
     if rank == 0:
         print(json.dumps(line))
     ctx.close()
@@ -374,16 +502,19 @@ def run_ours(args):
     return 0
 
 
-def run_profile_case(args):
-    """A small, self-ending case for ncu: one warm-up pass, then one pass of the chosen phase."""
+def run_profile_case(args, wl):
+    """A small, self-ending case for ncu: ONE layer of the configuration (its shapes, batch and prompt, so every
+    launch equals the one in the full model), one warm-up pass, then one pass of the chosen phase."""
     import torch
     from paper_2605_25655_b200 import thinfer
-    B, n_dec = args.batch, args.profile_decode_steps
-    w = thinfer.to_device_layers([synth.layer_weights(SHAPE, seed=0)])
-    x = torch.from_numpy(synth.hidden_states(SHAPE, 0, (B, PROMPT + n_dec)))
-    xp = x[:, :PROMPT].contiguous().cuda()
-    xd = [x[:, PROMPT + i].contiguous().cuda() for i in range(n_dec)]
-    ctx = thinfer.Context(SHAPE, w, None, max_batch=B, max_seq=PROMPT + n_dec)
+    B, n_dec = args.batch or wl.batch, args.profile_decode_steps
+    s = dataclasses.replace(wl.shape, n_layers=1, vocab=0)
+    w = [synth.device_layer_weights(s, 0, 0)]
+    g = torch.Generator(device="cuda").manual_seed(1)
+    x = torch.randn(B, wl.prompt + n_dec, s.hidden, device="cuda", dtype=torch.float16, generator=g)
+    xp = x[:, :wl.prompt].contiguous()
+    xd = [x[:, wl.prompt + i].contiguous() for i in range(n_dec)]
+    ctx = thinfer.Context(s, w, None, max_batch=B, max_seq=wl.prompt + n_dec)
     for rep in range(2):
         ctx.prefill(xp)
         if args.profile == "decode" or rep == 0:
@@ -392,7 +523,7 @@ def run_profile_case(args):
         ctx.release_slot(0)
         torch.cuda.synchronize()
     assert ctx.status() == 0
-    print(json.dumps({"profile_case": args.profile, "batch": B, "launches": ctx.launch_count()}))
+    print(json.dumps({"profile_case": args.profile, "config": wl.key, "batch": B, "launches": ctx.launch_count()}))
     ctx.close()
     return 0
 
@@ -459,9 +590,11 @@ def run_tables(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS),
+                    help="c2: 7B layer; c3: 7B stack; c4: 13B stack; c5: 70B stack (default)")
+    ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (c2: 1, 4, 16)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", choices=["prefill", "decode"], default=None,
@@ -469,13 +602,14 @@ def main():
     ap.add_argument("--profile-decode-steps", type=int, default=2)
     ap.add_argument("--tables", action="store_true", help="operator micro-benchmarks at the paper's Table 8 / 9 shapes")
     args = ap.parse_args()
+    wl = WORKLOADS[args.config]
     if args.tables:
         return run_tables(args)
     if args.profile:
-        return run_profile_case(args)
+        return run_profile_case(args, wl)
     if args.impl == "reference":
-        return run_reference(args)
-    return run_ours(args)
+        return run_reference(args, wl)
+    return run_ours(args, wl)
 
 
 if __name__ == "__main__":

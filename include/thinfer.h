@@ -91,8 +91,10 @@ typedef struct {
  * table, split-KV partials, staging for the *_host calls.  Host pointers out. */
 int thinfer_workspace_bytes(const thinfer_config* cfg, size_t* kv_bytes, size_t* scratch_bytes);
 
-/* Builds a context.  cfg, weights: host.  kv_workspace, scratch: device, at
- * least the sizes above (else THINFER_ECAPACITY); the context uses them until
+/* Builds a context for one model (Section 4.1: Llama-2 7B / 13B / 70B shapes, FP16 weights shared by all
+ * requests of a batch, Section 3.4.1) with buf_slots KV slots of max_batch x max_seq positions, the
+ * bounded buffer between the prefill and the decode stage (Section 3.4.2).  cfg, weights: host.
+ * kv_workspace, scratch: device, at least the sizes above (else THINFER_ECAPACITY); the context uses them until
  * thinfer_destroy.  Synchronises the device once (table set-up).  *out is set
  * only on success. */
 int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights,
@@ -171,8 +173,35 @@ int thinfer_slot_state(const thinfer_ctx* ctx, int32_t slot, int32_t* batch, int
 int thinfer_kv_pointer(const thinfer_ctx* ctx, int32_t slot, int32_t layer, int32_t which, void** device_ptr);
 
 /* Reads the device status word (0, or a thinfer_err a kernel wrote) without
- * synchronising; meaningful after the caller synchronised the stream. */
+ * synchronising; meaningful after the caller synchronised the stream.  (The paper's pipeline avoids failure
+ * by back-pressure, Section 3.4.2, and describes no error path; this word is how a bounded device-side
+ * wait that ran out is reported.) */
 int thinfer_status(thinfer_ctx* ctx, int32_t* device_status);
+
+/* The status word is sticky: once a kernel has written a code it stays non-zero until it is cleared (a
+ * later failure may replace the code by its own), and a
+ * kernel that gave up may have left arrival counters or the grid barrier of launch mode 2 half-way, so
+ * later steps of the context are not meaningful until it is cleared.  thinfer_clear_status synchronises the
+ * device, puts the counters, the grid barrier and the status word back to their initial state and returns;
+ * the KV slots keep their contents and lengths (release and prefill them again to be safe).  Call it with
+ * no work of the context in flight. */
+int thinfer_clear_status(thinfer_ctx* ctx);
+
+/* Self-test of the bounded device-side wait (no counterpart in the paper).  Enqueues a one-CTA kernel that
+ * waits, for at most limit_ns nanoseconds (1 us .. 100 ms), on a barrier nobody arrives on.  The wait gives
+ * up, the kernel returns normally and THINFER_ETIMEOUT is left in the status word: after synchronising the
+ * stream thinfer_status reports it, thinfer_clear_status clears it, and the context works as before.  This is
+ * the same wait, with a shorter limit, that guards every TMA / tensor-core pipeline of the library. */
+int thinfer_selftest_bounded_wait(thinfer_ctx* ctx, int64_t limit_ns, void* cuda_stream);
+
+/* Inspection hook for tests (Section 3.4.3's per-layer view: the hidden state between layers never leaves
+ * the library otherwise).  After layer layers[i] of every later prefill or decode step - layers[i] = -1
+ * means the input of layer 0, i.e. the embedding rows when vocab > 0 - the hidden state is copied, on the
+ * call's stream, to device_bufs[i]: device FP16 [batch x seq_len, hidden] (prefill) or [batch, hidden]
+ * (decode), caller-owned and large enough.  n = 0 removes all captures.  layers, device_bufs: host arrays
+ * [n], copied.  In launch mode 2 a decode step of up to 16 requests runs all layers in one kernel: only
+ * the last layer's state (and -1) can be captured there, other layers give THINFER_EUNSUPPORTED. */
+int thinfer_capture_hidden(thinfer_ctx* ctx, int32_t n, const int32_t* layers, void* const* device_bufs);
 
 /* Unified launch (Section 3.3.3: one creation + launch for the whole operator
  * graph instead of one per operator).  mode 0: one plain launch per fusion
@@ -212,6 +241,10 @@ int thinfer_trace_unified(thinfer_ctx* ctx, int32_t enable, uint64_t* host_out, 
 int64_t thinfer_launch_count(const thinfer_ctx* ctx);
 
 const char* thinfer_last_error(const thinfer_ctx* ctx);
+
+/* Ends a context (the paper has no counterpart: its pools live for the whole run, Section 3.4.2).  Frees the
+ * host object, its events and the status word; the caller's weights, KV workspace and scratch are untouched
+ * and may be freed afterwards.  No work of the context may be in flight.  NULL is allowed. */
 void thinfer_destroy(thinfer_ctx* ctx);
 
 /* ------------------------------------------------------------------------ *
@@ -259,6 +292,10 @@ int thinfer_op_linear_noalloc(const void* x, const void* w, void* y, int32_t row
 int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, void* out,
                                  int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t seq,
                                  int32_t kv_stride, int32_t head_dim, void* cuda_stream);
+
+/* Greedy pick of the stack's last step (the paper is silent on sampling): ids[r] = the lowest index at
+ * which logits[r, :] is largest.  logits device FP32 [rows, n]; ids device int32 [rows]. */
+int thinfer_op_argmax(const void* logits, void* ids, int32_t rows, int32_t n, void* cuda_stream);
 
 /* y = x * gain / sqrt(mean(x^2) + eps), rows of length n (Section 3.2.4). */
 int thinfer_op_rmsnorm(const void* x, const void* gain, void* y, int32_t rows, int32_t n, float eps,

@@ -116,19 +116,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // phase does not complete within ~2 s: the caller then abandons its role and the
 // kernel drains and returns instead of hanging the device.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_for(uint64_t* bar, uint32_t parity, int* status, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   uint32_t polls = 0;
   while (!mbar_try_wait(bar, parity)) {
     // purely time-based: the warps that wait on one barrier must all take the same decision,
     // because the ones that pass go on to a CTA-level barrier that has no time limit
-    if ((++polls & 0x3ffu) == 0u && global_ns() - t0 > kWaitLimitNs) {
+    if ((++polls & 0x3ffu) == 0u && global_ns() - t0 > limit_ns) {
       if (status != nullptr) *reinterpret_cast<volatile int*>(status) = kErrTimeout;
       return false;
     }
   }
   return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+  return mbar_wait_for(bar, parity, status, kWaitLimitNs);
 }
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

@@ -191,11 +191,28 @@ __global__ void rope_table_kernel(float* __restrict__ cos_t, float* __restrict__
 // Tracing aid: resets the 16 slots of every kernel id before a traced step (slots 9 .. 11 collect minima,
 // 12 .. 15 maxima), so that no memset sits between the kernels of the step.
 __global__ void trace_reset_kernel(unsigned long long* timeline, int kernels) {
+  pdl_launch_dependents();
+  pdl_wait();  // the kernels behind it in the chain only wait for THIS kernel: it must itself be ordered
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= kernels * 16) return;
   const int slot = i & 15;
   if (slot >= 9 && slot <= 11) timeline[i] = ~0ull;
   else if (slot >= 12) timeline[i] = 0ull;
+}
+
+// Self-test of the bounded wait every pipeline of this library relies on: one thread initialises an mbarrier
+// that expects an arrival nobody makes, all threads wait on it with the given limit, the wait gives up,
+// THINFER_ETIMEOUT lands in the status word and the kernel returns normally (nothing traps or hangs).
+__global__ void bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns, unsigned long long* waited_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  const uint64_t t0 = global_ns();
+  const bool ok = mbar_wait_for(&bar, 0, status, limit_ns);
+  if (threadIdx.x == 0 && waited_ns != nullptr) *waited_ns = ok ? 0ull : global_ns() - t0;
 }
 
 }  // namespace thinfer

@@ -113,8 +113,12 @@ struct thinfer_ctx {
   float* d_logits = nullptr;
   uint8_t *d_stage_in = nullptr, *d_stage_out = nullptr;
   float *part_o = nullptr, *part_ml = nullptr;
-  float* splitk_ws = nullptr;   // stream-K partial accumulators
+  float* splitk_ws = nullptr;   // stream-K partial accumulators (decode stage)
   int* splitk_counters = nullptr;
+  float* pf_splitk_ws = nullptr;  // the same for the prefill stage (its vocabulary projection), so that the two
+  int* pf_splitk_counters = nullptr;  // stages may overlap on two streams
+  // inspection: copies of the hidden state behind chosen layers (thinfer_capture_hidden)
+  std::vector<std::pair<int, void*>> captures;
   // unified decode kernel
   __half *xg = nullptr, *x1g = nullptr;
   float *sumsq0 = nullptr, *sumsq1 = nullptr, *attn_partial = nullptr;
@@ -178,9 +182,9 @@ int validate_config(const thinfer_config* c, std::string* why) {
 
 struct ScratchPlan {
   size_t rope_cos, rope_sin, h, qbuf, attn, x1, act, xa, xb, last, logits, ids_out, part_o, part_ml, splitk_ws,
-      splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, timeline, mega_common, mega_layers,
+      splitk_counters, pf_splitk_ws, pf_splitk_counters, xg, x1g, sumsq0, sumsq1, attn_partial, attn_counters, grid_bar, timeline, mega_common, mega_layers,
       stage_in, stage_out, slot_lens, d_h, d_qbuf, d_attn, d_x1, d_act, d_xa, d_xb, d_logits, d_stage_in, d_stage_out, total;
-  int max_splits, max_tiles;
+  int max_splits, max_tiles, pf_tiles;
 };
 
 constexpr int kTcMaxCtas = 160;      // persistent grid bound (a B200 has 148 SMs)
@@ -222,6 +226,11 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     // one slot per (tile, CTA) pair that can occur: tiles + CTAs; a slot holds 128 rows x (2 x 64) FP32 columns
     p.splitk_ws = take((tiles + kTcMaxCtas) * static_cast<size_t>(2 * kTcDecodeMaxBN) * 128 * 4);
     p.splitk_counters = take(tiles * 8);
+    // prefill stage: only its vocabulary projection is ever split along K
+    const size_t head_tiles = c.vocab > 0 ? t128(c.vocab) : 0;
+    p.pf_splitk_ws = take(head_tiles > 0 ? (head_tiles + kTcMaxCtas) * static_cast<size_t>(2 * kTcDecodeMaxBN) * 128 * 4 : 0);
+    p.pf_splitk_counters = take(head_tiles * 8);
+    p.pf_tiles = static_cast<int>(head_tiles);
   }
   {
     const size_t parts = (static_cast<size_t>(c.hidden) + 127) / 128;
@@ -273,6 +282,7 @@ struct Launcher {
   cudaStream_t st;
   int rc = THINFER_OK;
   bool cooperative = false;  // next launch only: all CTAs must be co-resident (grid-wide barriers inside)
+  bool prefill_stage = false;  // stream-K scratch of the prefill stage instead of the decode stage's
 
   template <typename... KArgs, typename... Args>
   void go(int kid, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
@@ -421,8 +431,8 @@ void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   a.norm_eps = norm_eps;
   if (stream_k && L.c != nullptr && rows <= kTcDecodeMaxBN) {
     a.mode = 1;
-    a.partial_ws = L.c->splitk_ws;
-    a.tile_counters = L.c->splitk_counters;
+    a.partial_ws = L.prefill_stage ? L.c->pf_splitk_ws : L.c->splitk_ws;
+    a.tile_counters = L.prefill_stage ? L.c->pf_splitk_counters : L.c->splitk_counters;
   }
   launch_tc_bn<EPI>(L, kid, bn, w0, w1, w2, mx, a);
 }
@@ -959,8 +969,9 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
     else launch_mega<64, 1>(L, c, a);
   }
   // every CTA arrives once per grid barrier: 5 per layer
+  // (a launch that failed enqueued nothing: the device counter did not move either)
   const unsigned int grid = c->sm_count < kTcMaxCtas ? c->sm_count : kTcMaxCtas;
-  c->bar_base += 5u * cf.n_layers * grid;
+  if (L.rc == THINFER_OK) c->bar_base += 5u * cf.n_layers * grid;
 }
 
 // final RMSNorm + LM head + greedy argmax on `batch` rows of x [batch][hidden]
@@ -989,10 +1000,21 @@ void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, in
          cf.vocab);
 }
 
+// inspection hook: a copy of the hidden state behind `layer` (-1: the input of layer 0), enqueued on the stream
+void capture_hidden(Launcher& L, thinfer_ctx* c, int layer, const __half* x, size_t rows) {
+  if (L.rc != THINFER_OK) return;
+  for (const auto& cap : c->captures) {
+    if (cap.first != layer) continue;
+    if (cudaMemcpyAsync(cap.second, x, rows * c->cfg.hidden * 2, cudaMemcpyDeviceToDevice, L.st) != cudaSuccess)
+      L.rc = fail(c, THINFER_ECUDA, "copying a captured hidden state failed");
+  }
+}
+
 int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq, void* out_primary, void* out_logits,
                 cudaStream_t st, const int* lens_dev = nullptr) {
   const thinfer_config& cf = c->cfg;
   Launcher L{c, st};
+  L.prefill_stage = true;
   if (c->trace_unified) L.go(-3, trace_reset_kernel, dim3(1), dim3(256), 0, c->timeline, 12);
   const int rows = batch * seq;
   const __half* x = nullptr;
@@ -1004,10 +1026,12 @@ int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq,
     x = static_cast<const __half*>(input);
   }
   __half* pong[2] = {c->xb, c->xa};
+  if (!c->captures.empty()) capture_hidden(L, c, -1, x, rows);
   for (int l = 0; l < cf.n_layers; ++l) {
     __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
     layer_prefill(L, c, slot, l, x, dst, batch, seq);
     x = dst;
+    if (!c->captures.empty()) capture_hidden(L, c, l, x, rows);
   }
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, gather_last_rows_kernel, dim3((batch + 7) / 8), dim3(256), 0, x, c->last, batch, seq,
@@ -1034,15 +1058,22 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
   const Slot& sl = c->slots[slot];
   const int* lens = sl.ragged ? c->slot_lens + static_cast<size_t>(slot) * cf.max_batch : nullptr;
   const int step_pos = sl.ragged ? sl.steps : pos;  // ragged: every request adds its own prompt length on the device
+  if (!c->captures.empty()) capture_hidden(L, c, -1, x, batch);
   if (c->launch_mode == 2 && mega_supported(c, batch) && !sl.ragged) {
+    for (const auto& cap : c->captures)
+      if (cap.first >= 0 && cap.first != cf.n_layers - 1)
+        return fail(c, THINFER_EUNSUPPORTED, "launch mode 2 runs all layers in one kernel: only the last layer's "
+                                             "hidden state can be captured");
     __half* dst = cf.vocab == 0 ? static_cast<__half*>(out_primary) : pong[(cf.n_layers - 1) & 1];
     layers_decode_unified(L, c, slot, x, dst, batch, pos);
     x = dst;
+    if (!c->captures.empty()) capture_hidden(L, c, cf.n_layers - 1, x, batch);
   } else {
     for (int l = 0; l < cf.n_layers; ++l) {
       __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
       layer_decode(L, c, slot, l, x, dst, batch, step_pos, lens, pos + 1);
       x = dst;
+      if (!c->captures.empty()) capture_hidden(L, c, l, x, batch);
     }
   }
   if (cf.vocab > 0)
@@ -1197,6 +1228,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->part_ml = reinterpret_cast<float*>(s + p.part_ml);
   c->splitk_ws = reinterpret_cast<float*>(s + p.splitk_ws);
   c->splitk_counters = reinterpret_cast<int*>(s + p.splitk_counters);
+  c->pf_splitk_ws = reinterpret_cast<float*>(s + p.pf_splitk_ws);
+  c->pf_splitk_counters = reinterpret_cast<int*>(s + p.pf_splitk_counters);
   c->xg = reinterpret_cast<__half*>(s + p.xg);
   c->x1g = reinterpret_cast<__half*>(s + p.x1g);
   c->sumsq0 = reinterpret_cast<float*>(s + p.sumsq0);
@@ -1260,7 +1293,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   const int n_tab = cfg->max_seq * (cfg->head_dim / 2);
   rope_table_kernel<<<(n_tab + 255) / 256, 256>>>(c->rope_cos, c->rope_sin, cfg->max_seq, cfg->head_dim / 2,
                                                   static_cast<double>(cfg->rope_base));
-  if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 8, 0) != cudaSuccess)
+  if (cudaMemsetAsync(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 8, 0) != cudaSuccess ||
+      (p.pf_tiles > 0 && cudaMemsetAsync(c->pf_splitk_counters, 0, static_cast<size_t>(p.pf_tiles) * 8, 0) != cudaSuccess))
     return cleanup(THINFER_ECUDA);
   {
     // parameter blocks of the unified decode kernel: weight tensor maps per layer, token-operand maps
@@ -1444,6 +1478,42 @@ int thinfer_status(thinfer_ctx* c, int32_t* device_status) {
   return THINFER_OK;
 }
 
+int thinfer_clear_status(thinfer_ctx* c) {
+  if (c == nullptr) return THINFER_EINVAL;
+  // the caller has synchronised: nothing of this context is running.  A kernel that gave up may have left
+  // arrival counters and the grid barrier half-way: put all of them back to their initial state.
+  const ScratchPlan p = plan_scratch(c->cfg);
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(c, THINFER_ECUDA, "device synchronisation failed");
+  if (cudaMemset(c->splitk_counters, 0, static_cast<size_t>(p.max_tiles) * 8) != cudaSuccess ||
+      (p.pf_tiles > 0 && cudaMemset(c->pf_splitk_counters, 0, static_cast<size_t>(p.pf_tiles) * 8) != cudaSuccess) ||
+      cudaMemset(c->attn_counters, 0, static_cast<size_t>(c->cfg.max_batch) * c->cfg.n_q_heads * 4) != cudaSuccess ||
+      cudaMemset(c->grid_bar, 0, 64) != cudaSuccess)
+    return fail(c, THINFER_ECUDA, "resetting the device counters failed");
+  c->bar_base = 0;
+  *reinterpret_cast<volatile int*>(c->status_host) = 0;
+  return THINFER_OK;
+}
+
+int thinfer_selftest_bounded_wait(thinfer_ctx* c, int64_t limit_ns, void* cuda_stream) {
+  if (c == nullptr) return THINFER_EINVAL;
+  if (limit_ns < 1000 || limit_ns > 100000000) return fail(c, THINFER_EINVAL, "limit_ns outside [1 us, 100 ms]");
+  Launcher L{c, static_cast<cudaStream_t>(cuda_stream)};
+  L.go(-4, bounded_wait_selftest_kernel, dim3(1), dim3(64), 0, c->status_dev, static_cast<unsigned long long>(limit_ns),
+       c->timeline + 255);
+  return L.rc;
+}
+
+int thinfer_capture_hidden(thinfer_ctx* c, int32_t n, const int32_t* layers, void* const* device_bufs) {
+  if (c == nullptr || n < 0) return THINFER_EINVAL;
+  if (n > 0 && (layers == nullptr || device_bufs == nullptr)) return fail(c, THINFER_EINVAL, "layers or device_bufs is NULL");
+  for (int i = 0; i < n; ++i)
+    if (layers[i] < -1 || layers[i] >= c->cfg.n_layers || device_bufs[i] == nullptr)
+      return fail(c, THINFER_EINVAL, "capture %d: layer %d outside [-1, %d) or NULL buffer", i, layers[i], c->cfg.n_layers);
+  c->captures.clear();
+  for (int i = 0; i < n; ++i) c->captures.emplace_back(layers[i], device_bufs[i]);
+  return THINFER_OK;
+}
+
 int thinfer_set_launch_mode(thinfer_ctx* c, int32_t mode) {
   if (c == nullptr) return THINFER_EINVAL;
   if (mode < 0 || mode > 2) return fail(c, THINFER_EUNSUPPORTED, "launch mode %d is not available in this build", mode);
@@ -1614,6 +1684,13 @@ int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, vo
   Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
   attn_prefill(L, static_cast<const __half*>(q), static_cast<const __half*>(k), static_cast<const __half*>(v),
                static_cast<__half*>(out), batch, n_q_heads, n_kv_heads, seq, kv_stride, head_dim, nullptr);
+  return L.rc;
+}
+
+int thinfer_op_argmax(const void* logits, void* ids, int32_t rows, int32_t n, void* cuda_stream) {
+  if (logits == nullptr || ids == nullptr || rows <= 0 || n <= 0) return THINFER_EINVAL;
+  Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
+  L.go(-2, argmax_rows_kernel, dim3(rows), dim3(1024), 0, static_cast<const float*>(logits), static_cast<int32_t*>(ids), n);
   return L.rc;
 }
 

@@ -12,6 +12,13 @@ weights and the prompt data set the paper used are replaced by:
 
 Every tensor has its own stream, keyed by (seed, layer, tensor id), so any one
 of them can be regenerated without the others.
+
+Two generators with the same recipe: numpy on the host for the small cases, and
+torch's counter-based CUDA generator for the full-depth configurations, whose
+weights (up to 138 GB) are drawn on the device tensor by tensor and never exist
+on the host as a whole; a consumer on the host copies the one layer it needs.
+The two generators give different values for the same key; a case uses one of
+them throughout.
 """
 from __future__ import annotations
 
@@ -109,3 +116,45 @@ def hidden_states(shape: Shape, seed: int, dims, stream: int = 0) -> np.ndarray:
 def token_ids(shape: Shape, seed: int, dims, stream: int = 0) -> np.ndarray:
     rng = _rng(seed, stream, _IDS_ID)
     return rng.integers(0, shape.vocab, size=tuple(dims), dtype=np.int32)
+
+
+# --------------------------------------------------------------------------- #
+# the same recipe drawn on the device (full-depth configurations)
+# --------------------------------------------------------------------------- #
+def _device_normal16(shape_, mean, std, key, device):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(key))
+    t = torch.empty(shape_, dtype=torch.float16, device=device)
+    t.normal_(mean, std, generator=g)
+    return t
+
+
+def _key(seed, layer, tensor_id):
+    return (int(seed) * 1_000_003 + int(layer)) * 1_009 + int(tensor_id) + 12_345
+
+
+def device_layer_weights(shape: Shape, seed: int, layer: int, device="cuda:0") -> dict:
+    """The nine tensors of one layer as CUDA FP16 tensors drawn on the device."""
+    out = {}
+    for tid, name in enumerate(LAYER_TENSORS):
+        mean = 1.0 if name.endswith("_norm") else 0.0
+        out[name] = _device_normal16(layer_tensor_shape(shape, name), mean, 0.02, _key(seed, layer, tid), device)
+    return out
+
+
+def device_stack_weights(shape: Shape, seed: int = 0, device="cuda:0") -> dict:
+    """Whole model on the device: {"layers": [dict per layer], "embed", "final_norm", "lm_head"}."""
+    out = {"layers": [device_layer_weights(shape, seed, l, device) for l in range(shape.n_layers)]}
+    for i, name in enumerate(_STACK_TENSORS):
+        dims = (shape.hidden,) if name == "final_norm" else (shape.vocab, shape.hidden)
+        out[name] = _device_normal16(dims, 1.0 if name == "final_norm" else 0.0, 0.02,
+                                     _key(seed, 1 << 20, 50 + i), device)
+    return out
+
+
+def model_bytes(shape: Shape) -> int:
+    """FP16 bytes of all weights of a stack configuration."""
+    per_layer = sum(int(np.prod(layer_tensor_shape(shape, n))) for n in LAYER_TENSORS)
+    stack = (2 * shape.vocab * shape.hidden + shape.hidden) if shape.vocab > 0 else 0
+    return 2 * (per_layer * shape.n_layers + stack)

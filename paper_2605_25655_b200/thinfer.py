@@ -22,9 +22,10 @@ EXPORTS = (
     "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_prefill_ragged", "thinfer_slot_lengths",
     "thinfer_decode_step",
     "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
-    "thinfer_kv_pointer", "thinfer_status", "thinfer_set_launch_mode", "thinfer_profile_select",
+    "thinfer_kv_pointer", "thinfer_status", "thinfer_clear_status", "thinfer_capture_hidden", "thinfer_set_launch_mode", "thinfer_profile_select",
     "thinfer_profile_read", "thinfer_trace_unified", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
     "thinfer_op_linear", "thinfer_op_linear_noalloc", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
+    "thinfer_op_argmax", "thinfer_selftest_bounded_wait",
 )
 
 
@@ -76,6 +77,8 @@ def lib():
     L.thinfer_slot_state.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32)]
     L.thinfer_kv_pointer.argtypes = [vp, i32, i32, i32, C.POINTER(vp)]
     L.thinfer_status.argtypes = [vp, C.POINTER(i32)]
+    L.thinfer_clear_status.argtypes = [vp]
+    L.thinfer_capture_hidden.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(vp)]
     L.thinfer_set_launch_mode.argtypes = [vp, i32]
     L.thinfer_profile_select.argtypes = [vp, i32]
     L.thinfer_profile_read.argtypes = [vp, C.POINTER(i32), C.POINTER(C.c_float)]
@@ -90,6 +93,8 @@ def lib():
     L.thinfer_op_linear_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     L.thinfer_op_attention_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
     L.thinfer_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, C.c_float, vp]
+    L.thinfer_op_argmax.argtypes = [vp, vp, i32, i32, vp]
+    L.thinfer_selftest_bounded_wait.argtypes = [vp, i64, vp]
     _lib = L
     return L
 
@@ -241,6 +246,22 @@ class Context:
         _check(lib().thinfer_status(self.h, C.byref(v)), self.h)
         return v.value
 
+    def clear_status(self):
+        _check(lib().thinfer_clear_status(self.h), self.h)
+
+    def selftest_bounded_wait(self, limit_ns=1_000_000, stream=None):
+        _check(lib().thinfer_selftest_bounded_wait(self.h, int(limit_ns), _stream_ptr(stream)), self.h)
+
+    def capture_hidden(self, captures):
+        """captures: dict layer index (-1 = input of layer 0) -> CUDA FP16 tensor that receives the hidden
+        state behind that layer on every later prefill / decode step; {} or None removes all captures."""
+        captures = captures or {}
+        n = len(captures)
+        layers = (C.c_int32 * max(n, 1))(*[int(l) for l in captures])
+        bufs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in captures.values()])
+        self._captures = captures                      # keeps the tensors alive
+        _check(lib().thinfer_capture_hidden(self.h, n, layers, bufs), self.h)
+
     def set_launch_mode(self, mode):
         _check(lib().thinfer_set_launch_mode(self.h, mode), self.h)
 
@@ -318,6 +339,14 @@ def op_rmsnorm(x, gain, eps, stream=None):
     y = torch.empty_like(x)
     _check(lib().thinfer_op_rmsnorm(x.data_ptr(), gain.data_ptr(), y.data_ptr(), rows, n, eps, _stream_ptr(stream)))
     return y
+
+
+def op_argmax(logits, stream=None):
+    import torch
+    rows, n = logits.shape
+    ids = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    _check(lib().thinfer_op_argmax(logits.data_ptr(), ids.data_ptr(), rows, n, _stream_ptr(stream)))
+    return ids
 
 
 def to_device_layers(np_layers, device="cuda:0"):

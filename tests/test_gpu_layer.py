@@ -493,3 +493,171 @@ def test_ragged_prompts_stack_logits(T, ffn):
         ctx.prefill_ragged(torch.from_numpy(ids[:, :14].copy()).cuda(), (9, 0, 14))
     assert e.value.code == thinfer.EINVAL
     ctx.close()
+
+
+# ---- free-running greedy generation (Section 3.4.2: the prefill emits the first token, decode the rest) ----------
+def _greedy_case(T, shape, seed, batch, prompt, n_new):
+    """Generates n_new tokens per request with the ids fed back ON THE DEVICE (no host synchronisation inside the
+    loop) and follows the oracle's own greedy run.  A request counts as agreeing until the first step at which
+    the two picks differ; that may only happen where the oracle's top-2 gap is below 4x the logit error (both
+    picks are then correct answers).  Returns (steps compared, steps agreeing, requests that ever diverged)."""
+    torch, thinfer = T
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, seed)
+    ids0 = synth.token_ids(shape, seed, (batch, prompt))
+    ctx = _ctx(T, shape, sw["layers"], batch, prompt + n_new, stack=sw)
+    cur, lg = ctx.prefill(torch.from_numpy(ids0).cuda(), want_logits=True)
+    gpu_ids, gpu_logits = [cur], [lg]
+    for _ in range(n_new - 1):
+        cur, lg = ctx.decode_step(cur, want_logits=True)       # the previous step's device tensor is the input
+        gpu_ids.append(cur)
+        gpu_logits.append(lg)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    assert ctx.slot_state(0) == (batch, prompt + n_new - 1)
+    gpu_ids = [t.cpu().numpy() for t in gpu_ids]
+    gpu_logits = [t.cpu().numpy() for t in gpu_logits]
+    ctx.close()
+
+    ref_logits, ref_next, caches, _ = O.stack_prefill(cfg, sw, ids0)
+    alive = np.ones(batch, dtype=bool)
+    compared = agreed = 0
+    for step in range(n_new):
+        # the GPU's pick is always the lowest-index argmax of its own logits
+        np.testing.assert_array_equal(gpu_ids[step], np.argmax(gpu_logits[step], axis=-1))
+        for b in np.nonzero(alive)[0]:
+            compared += 1
+            err = np.max(np.abs(gpu_logits[step][b] - ref_logits[b]))
+            top2 = np.sort(ref_logits[b])[-2:]
+            if gpu_ids[step][b] == ref_next[b]:
+                agreed += 1
+                assert err <= 2e-2 * np.sqrt(np.mean(ref_logits[b] ** 2)), f"step {step} request {b}: logits off"
+            else:
+                assert top2[1] - top2[0] <= 4 * err, (f"step {step} request {b}: picks differ although the oracle's "
+                                                      f"top-2 gap {top2[1] - top2[0]:.3e} > 4 x logit error {err:.3e}")
+                alive[b] = False
+        if step + 1 < n_new:
+            ref_logits, ref_next, caches, _ = O.stack_decode(cfg, sw, ref_next.astype(np.int32), caches, prompt + step)
+    return compared, agreed, int((~alive).sum())
+
+
+def test_greedy_generation_small_stack_ids_fed_back_on_device(T):
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=704, n_layers=3, vocab=1000)
+    compared, agreed, diverged = _greedy_case(T, shape, seed=41, batch=4, prompt=12, n_new=24)
+    print(f"greedy, small stack: {agreed}/{compared} request-steps agree with the oracle's greedy run, "
+          f"{diverged}/4 requests met a near-tie")
+    assert agreed >= compared // 2
+
+
+def test_greedy_generation_llama7b_dims_two_layers(T):
+    shape = dataclasses.replace(synth.LLAMA_7B, n_layers=2)
+    compared, agreed, diverged = _greedy_case(T, shape, seed=42, batch=2, prompt=16, n_new=8)
+    print(f"greedy, 2-layer 7B shapes, 32000-way head: {agreed}/{compared} request-steps agree, "
+          f"{diverged}/2 requests met a near-tie")
+    assert agreed >= compared // 2
+
+
+def test_exact_tie_in_the_vocabulary_projection_goes_to_the_lowest_index(T):
+    # rows 8 and 9 of the head are identical and dominate: their logits are bit-identical, the pick must be 8
+    torch, thinfer = T
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=704, n_layers=1, vocab=1000)
+    sw = synth.stack_weights(shape, 43)
+    ids = synth.token_ids(shape, 43, (3, 6))
+    for batch in (3, 1):
+        head = sw["lm_head"].copy()
+        ctx0 = _ctx(T, shape, sw["layers"], batch, 8, stack=sw)
+        cap = torch.zeros(batch * 5, shape.hidden, dtype=torch.float16, device="cuda")
+        ctx0.capture_hidden({0: cap})
+        ctx0.prefill(torch.from_numpy(ids[:batch, :5].copy()).cuda())
+        last = cap.view(batch, 5, -1)[:, -1].float().cpu().numpy()          # final hidden state of the last position
+        ctx0.close()
+        # a head row aligned with request 0's normalised state wins by a wide margin; duplicate it
+        direction = (last[0] * sw["final_norm"].astype(np.float32))
+        direction = (direction / np.linalg.norm(direction)).astype(np.float16)
+        head[8] = direction
+        head[9] = direction
+        sw2 = dict(sw, lm_head=head)
+        ctx = _ctx(T, shape, sw["layers"], batch, 8, stack=sw2)
+        nxt, logits = ctx.prefill(torch.from_numpy(ids[:batch, :5].copy()).cuda(), want_logits=True)
+        lg = logits.cpu().numpy()
+        assert lg[0, 8] == lg[0, 9] and lg[0, 8] == lg[0].max()
+        assert int(nxt.cpu()[0]) == 8
+        ctx.close()
+
+
+def test_bounded_wait_runs_out_and_the_context_recovers(T):
+    # a wait that nothing satisfies gives up after its limit: the kernel returns, the status word reports
+    # THINFER_ETIMEOUT, and after thinfer_clear_status the context computes as before
+    torch, thinfer = T
+    shape = synth.TINY
+    w = synth.layer_weights(shape, 0)
+    x = torch.from_numpy(synth.hidden_states(shape, 0, (2, 12))).cuda()
+    ctx = _ctx(T, shape, [w], 2, 16)
+    before = ctx.prefill(x[:, :11].contiguous()).cpu().numpy()
+    step_before = ctx.decode_step(x[:, 11].contiguous()).cpu().numpy()
+    ctx.release_slot(0)
+    assert ctx.status() == 0
+    ctx.selftest_bounded_wait(limit_ns=2_000_000)                    # 2 ms
+    torch.cuda.synchronize()
+    assert ctx.status() == thinfer.ETIMEOUT
+    ctx.clear_status()
+    assert ctx.status() == 0
+    for mode in (1, 2):
+        ctx.set_launch_mode(mode)
+        after = ctx.prefill(x[:, :11].contiguous()).cpu().numpy()
+        step_after = ctx.decode_step(x[:, 11].contiguous()).cpu().numpy()
+        ctx.release_slot(0)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        np.testing.assert_array_equal(after, before)
+        if mode == 1:
+            np.testing.assert_array_equal(step_after, step_before)
+    with pytest.raises(thinfer.ThinferError):
+        ctx.selftest_bounded_wait(limit_ns=10**10)                    # limits above 100 ms are refused
+    ctx.close()
+
+
+def test_two_stream_stages_with_vocabulary_and_batches_above_16(T):
+    # both stages use the stream-K tensor-core path here (32 requests): the prefill stage's vocabulary projection
+    # and the decode stage's projections have separate partial-sum areas, so slot 1 may be prefilled while slot 0
+    # decodes.  Results: equal to the serial run bit for bit, and to the oracle within tolerance.
+    torch, thinfer = T
+    shape = synth.Shape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn=704, n_layers=2, vocab=1000)
+    cfg = oracle_config(shape)
+    sw = synth.stack_weights(shape, 44)
+    B = 32
+    ids = synth.token_ids(shape, 44, (2, B, 14))
+    dev = torch.from_numpy(ids).cuda()
+    p = [dev[s, :, :10].contiguous() for s in range(2)]
+    d = [[dev[s, :, 10 + i].contiguous() for i in range(4)] for s in range(2)]
+
+    def run(two_streams):
+        ctx = _ctx(T, shape, sw["layers"], B, 16, stack=sw, buf_slots=2)
+        sp = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
+        sd = torch.cuda.Stream() if two_streams else torch.cuda.current_stream()
+        torch.cuda.synchronize()
+        out = {}
+        out["p0"] = ctx.prefill(p[0], slot=0, stream=sp, want_logits=True)[1]
+        for rep in range(3):                                          # keep the prefill stream busy meanwhile
+            out[f"p1_{rep}"] = ctx.prefill(p[1], slot=1, stream=sp, want_logits=True)[1]
+            if rep < 2:
+                ctx.release_slot(1, stream=sp)
+        for i in range(4):
+            out[f"d0_{i}"] = ctx.decode_step(d[0][i], slot=0, stream=sd, want_logits=True)[1]
+        for i in range(4):
+            out[f"d1_{i}"] = ctx.decode_step(d[1][i], slot=1, stream=sd, want_logits=True)[1]
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        res = {k: v.cpu().numpy() for k, v in out.items()}
+        ctx.close()
+        return res
+
+    serial, overlapped = run(False), run(True)
+    for k in serial:
+        np.testing.assert_array_equal(serial[k], overlapped[k], err_msg=k)
+    for s in range(2):
+        ref, _, caches, _ = O.stack_prefill(cfg, sw, ids[s, :, :10])
+        assert_rows_close(overlapped["p0" if s == 0 else "p1_2"], ref, f"slot {s}: prefill logits")
+        for i in range(4):
+            ref, _, caches, _ = O.stack_decode(cfg, sw, ids[s, :, 10 + i], caches, 10 + i)
+            assert_rows_close(overlapped[f"d{s}_{i}"], ref, f"slot {s}: decode logits step {i}")

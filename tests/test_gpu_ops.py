@@ -131,3 +131,23 @@ def test_attention_first_row_returns_v0_and_uniform_keys_give_running_mean(T):
     np.testing.assert_allclose(got[0], v[0, :, 0, :].astype(np.float64), rtol=2e-3, atol=2e-3)
     mean = np.cumsum(v[0].astype(np.float64), axis=1) / np.arange(1, s + 1)[None, :, None]
     np.testing.assert_allclose(got, mean.transpose(1, 0, 2), rtol=0, atol=4e-3)
+
+
+def test_argmax_exact_ties_go_to_the_lowest_index(T):
+    torch, thinfer = T
+    n = 32000
+    rng = np.random.default_rng(5)
+    lg = rng.standard_normal((6, n)).astype(np.float32)
+    lg[0, [31999, 17, 20000]] = 9.0                 # three equal maxima far apart (different threads and warps)
+    lg[1, [1024, 1025]] = 7.5                       # neighbours across a thread-stride boundary
+    lg[2, :] = 1.25                                 # everything ties: index 0
+    lg[3, [5, 31998]] = np.inf                      # infinite maxima tie as well
+    lg[4, :] = -np.inf
+    lg[4, [123, 30000]] = -3.0                      # the rest is -inf
+    lg[5, 31999] = 50.0                             # unique maximum in the last column
+    ids = thinfer.op_argmax(torch.from_numpy(lg).cuda()).cpu().numpy()
+    np.testing.assert_array_equal(ids, [17, 1024, 0, 5, 123, 31999])
+    np.testing.assert_array_equal(ids, O.argmax_lowest(lg))
+    # odd row length, fewer columns than threads
+    small = np.array([[0.0, 2.0, 2.0, -1.0, 2.0]], dtype=np.float32)
+    assert int(thinfer.op_argmax(torch.from_numpy(small).cuda()).cpu()[0]) == 1

@@ -27,10 +27,11 @@ def test_times_are_the_slowest_ranks_and_throughput_is_the_whole_job():
 
 def test_reference_arm_under_two_ranks_prints_once():
     res = _torchrun([os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
-                     "--warmup", "0", "--batch", "1"], 29542)
+                     "--warmup", "0", "--batch", "1", "--config", "c3"], 29542)
     assert res.returncode == 0, res.stderr[-2000:]
     lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
     assert len(lines) == 1
     out = json.loads(lines[0])
     assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["cpu_baseline"]["kind"] == "oracle"
     assert out["e2e"]["h2d_bytes_per_step"] == 0 and out["value"] > 0
+    assert "32 layers" in out["config"]["workload"] and "32 x the layer time" in out["cpu_baseline"]["sample"]
