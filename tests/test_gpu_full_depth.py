@@ -6,9 +6,11 @@ never exists on the host); the oracle sees one layer at a time, widened to float
 into reusable pinned host buffers.
 
 Per configuration:
-  (i)   full depth, reduced token budget (2 requests, 64-token prompt, 4 decode steps, teacher forced), end to
-        end - the oracle runs on its own states, nothing is chained: final hidden state cosine >= 0.999 per
-        token and logits within the row-RMS tolerance, for the per-unit decode path and for the unified kernel;
+  (i)   full depth, reduced token budget (2 requests, 64-token prompt, 4 decode steps, teacher forced):
+        EVERY layer chained (the oracle layer is fed the GPU's own FP16 input of that layer, prefill and each
+        decode step, K/V cache contents included) within 2e-2 x row RMS; and end to end - the oracle's own
+        stack loop on its own states - final hidden state and logits cosine >= 0.999 per token, for the
+        per-unit decode path and for the unified kernel;
   (ii)  the configuration's real batch and prompt length: per-layer chained checks of layers {0, L/2, L-1}
         on the first and the last request (the oracle layer is fed the GPU's own FP16 input of that layer,
         captured with thinfer_capture_hidden), for the prefill and for the first decode step, K/V cache
@@ -98,45 +100,98 @@ def _context(T, m, max_batch, max_seq):
 
 def test_full_depth_end_to_end_on_a_reduced_token_budget(T, model):
     torch, thinfer = T
-    shape, L = model["shape"], model["shape"].n_layers
+    shape, L, D = model["shape"], model["shape"].n_layers, model["shape"].hidden
     cfg = oracle_config(shape)
     B, S, n_dec = 2, 64, 4
     ids = synth.token_ids(shape, 31, (B, S + n_dec))
-    # One pass of the oracle's own stack loop over all S + n_dec tokens.  Row t of a prefill equals the
-    # incremental decode of token t (pinned on the CPU), so its rows are the reference for every decode step.
-    sw_host = dict(model["stack64"], layers=model["host"])
+    idd = torch.from_numpy(ids).cuda()
+
+    # ---- the GPU runs first.  Mode 1 keeps the hidden state behind EVERY layer (prefill and each decode step).
+    gpu = {}
+    for mode in (1, 2):
+        ctx = _context(T, model, B, S + n_dec + 4)
+        ctx.set_launch_mode(mode)
+        pre = torch.zeros(L + 1, B * S, D, dtype=torch.float16, device="cuda")
+        dec = torch.zeros(n_dec, L + 1, B, D, dtype=torch.float16, device="cuda")
+        every = list(range(-1, L)) if mode == 1 else [L - 1]
+        ctx.capture_hidden({l: pre[l + 1] for l in every})
+        nxt, logits = ctx.prefill(idd[:, :S].contiguous(), want_logits=True)
+        steps = [(nxt.cpu().numpy(), logits.cpu().numpy())]
+        for i in range(n_dec):
+            ctx.capture_hidden({l: dec[i, l + 1] for l in every})
+            nxt, logits = ctx.decode_step(idd[:, S + i].contiguous(), want_logits=True)
+            steps.append((nxt.cpu().numpy(), logits.cpu().numpy()))
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        gpu[mode] = dict(pre=pre.view(L + 1, B, S, D), dec=dec, steps=steps)
+        if mode == 1:
+            kv = [(ctx.kv_view(0, l, 0)[:B, :, :S + n_dec].cpu().numpy(), ctx.kv_view(0, l, 1)[:B, :, :S + n_dec].cpu().numpy())
+                  for l in range(L)]
+        ctx.close()
+
+    # ---- chained check of every layer, done while that layer's weights are on the host: the oracle layer is fed
+    # the GPU's own FP16 input of the layer (prefill rows, then each decode step continuing from the GPU's cache)
+    worst = {"prefill": 0.0, "decode": 0.0}
+
+    def chained(l, w):
+        g = gpu[1]
+        ref, kc, vc = O.layer_prefill(cfg, w, g["pre"][l].cpu().numpy())
+        e, _ = assert_rows_close(g["pre"][l + 1].cpu().numpy(), ref, f"layer {l}: prefill output (chained)")
+        worst["prefill"] = max(worst["prefill"], e)
+        kg, vg = kv[l]
+        assert_rows_close(kg[:, :, :S], kc, f"layer {l}: K cache", max_err=6e-3)
+        assert_rows_close(vg[:, :, :S], vc, f"layer {l}: V cache", max_err=6e-3)
+        for i in range(n_dec):
+            t = S + i
+            r, k2, v2 = O.layer_decode(cfg, w, g["dec"][i, l].cpu().numpy(), kg[:, :, :t].astype(np.float64),
+                                       vg[:, :, :t].astype(np.float64), t)
+            e, _ = assert_rows_close(g["dec"][i, l + 1].cpu().numpy(), r, f"layer {l}: decode step t={t} (chained)")
+            worst["decode"] = max(worst["decode"], e)
+            assert_rows_close(kg[:, :, t], k2[:, :, t], f"layer {l}: K append t={t}", max_err=6e-3)
+            assert_rows_close(vg[:, :, t], v2[:, :, t], f"layer {l}: V append t={t}", max_err=6e-3)
+
+    class LayersWithChainedCheck:
+        """Hands the oracle's stack loop one layer at a time and checks that layer on the way."""
+        def __iter__(self):
+            for l in range(L):
+                w = model["host"].fetch(l)
+                chained(l, w)
+                yield w
+
+    # ---- end to end: ONE pass of the oracle's own stack loop over all S + n_dec tokens, on its own states.  Row t
+    # of a prefill equals the incremental decode of token t (pinned on the CPU), so its rows are the reference for
+    # every decode step.
+    sw_host = dict(model["stack64"], layers=LayersWithChainedCheck())
     _, _, _, hid = O.stack_prefill(cfg, sw_host, ids)
     final = hid[-1]                                                    # [B, S + n_dec, D], float64
     ref_logits = {t: O.head_logits(cfg, sw_host, final[:, t]) for t in range(S - 1, S + n_dec)}
     del hid
+    # how far FP16 storage alone moves the result (the oracle's diagnostic switch; context, never the criterion)
+    _, _, _, hid16 = O.stack_prefill(cfg, dict(model["stack64"], layers=model["host"]), ids, emulate_fp16=True)
+    emu_h, emu_cos = row_stats(hid16[-1], final)
+    emu_l, _ = row_stats(O.head_logits(cfg, sw_host, hid16[-1][:, S - 1]), ref_logits[S - 1])
+    del hid16
 
-    idd = torch.from_numpy(ids).cuda()
-    report = []
+    print(f"\n{model['name']} x{L}: chained per-layer max|err|/rms over all {L} layers: prefill {worst['prefill']:.2e}, "
+          f"decode {worst['decode']:.2e}; FP16-storage emulation of the oracle vs the oracle, end to end: hidden "
+          f"{emu_h:.2e} (cos {emu_cos:.6f}), logits {emu_l:.2e}")
     for mode in (1, 2):
-        ctx = _context(T, model, B, S + n_dec + 4)
-        ctx.set_launch_mode(mode)
-        cap = torch.zeros(B * S, shape.hidden, dtype=torch.float16, device="cuda")
-        ctx.capture_hidden({L - 1: cap})
-        nxt, logits = ctx.prefill(idd[:, :S].contiguous(), want_logits=True)
-        got_final = cap.view(B, S, shape.hidden).cpu().numpy()
-        err_h, cos_h = row_stats(got_final, final[:, :S])
-        assert cos_h >= 0.999, f"mode {mode}: final hidden state after {L} layers, cosine {cos_h:.6f}"
-        err_l, cos_l = assert_rows_close(logits.cpu().numpy(), ref_logits[S - 1], f"mode {mode}: prefill logits after {L} layers")
-        _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits[S - 1])
-        report.append((mode, "prefill", err_h, cos_h, err_l, cos_l))
-        for t in range(S, S + n_dec):
-            nxt, logits = ctx.decode_step(idd[:, t].contiguous(), want_logits=True)
-            got = cap[:B].cpu().numpy()
-            err_h, cos_h = row_stats(got, final[:, t])
-            assert cos_h >= 0.999, f"mode {mode}: final hidden state of decode step t={t}, cosine {cos_h:.6f}"
-            err_l, cos_l = assert_rows_close(logits.cpu().numpy(), ref_logits[t], f"mode {mode}: decode logits t={t}")
-            _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits[t])
-            report.append((mode, f"decode t={t}", err_h, cos_h, err_l, cos_l))
-        assert ctx.status() == 0
-        ctx.close()
-    for r in report:
-        print(f"{model['name']} x{L} mode {r[0]} {r[1]}: hidden max|err|/rms {r[2]:.2e} cos {r[3]:.6f}; "
-              f"logits max|err|/rms {r[4]:.2e} cos {r[5]:.6f}")
+        g = gpu[mode]
+        for i, (nxt, logits) in enumerate(g["steps"]):
+            t = S - 1 + i
+            got = g["pre"][L][:, :S].cpu().numpy() if i == 0 else g["dec"][i - 1, L].cpu().numpy()
+            want = final[:, :S] if i == 0 else final[:, t]
+            err_h, cos_h = row_stats(got, want)
+            err_l, cos_l = row_stats(logits, ref_logits[t])
+            print(f"  mode {mode} {'prefill' if i == 0 else f'decode t={t}'}: final hidden max|err|/rms {err_h:.2e} "
+                  f"cos {cos_h:.6f}; logits max|err|/rms {err_l:.2e} cos {cos_l:.6f}")
+            assert np.all(np.isfinite(logits))
+            # end-to-end criterion: cosine >= 0.999 per token (the 2e-2 x RMS bound is the per-layer, chained one);
+            # the maximum error may exceed 2e-2 after tens of layers, but not by more than FP16 storage explains
+            assert cos_h >= 0.999, f"mode {mode} step {i}: final hidden state after {L} layers, cosine {cos_h:.6f}"
+            assert cos_l >= 0.999, f"mode {mode} step {i}: logits after {L} layers, cosine {cos_l:.6f}"
+            assert err_l <= max(2e-2, 4 * emu_l), f"mode {mode} step {i}: logits max|err|/rms {err_l:.2e} vs FP16-storage {emu_l:.2e}"
+            _check_greedy(nxt, logits, ref_logits[t])
 
 
 def test_chained_per_layer_checks_at_the_real_batch_and_prompt(T, model):
