@@ -11,6 +11,7 @@ rate (batch x generated / total latency, Section 3.4.1) and the roofline fractio
   python bench.py --impl reference ...                      # the CPU oracle, timed on the host cores
   python bench.py --tables                                  # operator latencies at the paper's Table 8 / 9 shapes
   python bench.py --profile {prefill,decode} --config cX    # one layer of that configuration: the case ncu captures
+  python bench.py --profile stack --config cX               # two layers + head: the case of the ncu launch list
 
 With N > 1 (under torchrun) every rank runs an independent replica of the same workload on its own GPU: the
 path has no exchange step, so there is no collective on the data path; times are the maximum over ranks.
@@ -502,6 +503,33 @@ def run_ours(args, wl):
     return 0
 
 
+def run_profile_stack(args, wl):
+    """The launch list's case: a TWO-layer stack of the configuration with its vocabulary head, real batch and
+    prompt - every kernel of the benchmark's step appears with the arguments it has in the full model (layer 0
+    with the norm prologue, layer 1 with the folded norm, embedding, head, argmax).  One warm-up pass, then one
+    pass of prefill + `--profile-decode-steps` decode steps.  The full model repeats the per-layer launches of
+    layer 1 (n_layers - 1) times: the summary under profiles/ scales the shares accordingly."""
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    B, n_dec = args.batch or wl.batch, args.profile_decode_steps
+    s = dataclasses.replace(wl.shape, n_layers=2)
+    sw = synth.device_stack_weights(s, 0)
+    ctx = thinfer.Context(s, sw["layers"], {n: sw[n] for n in ("embed", "final_norm", "lm_head")}, max_batch=B,
+                          max_seq=wl.prompt + n_dec)
+    ids = torch.from_numpy(synth.token_ids(s, 0, (B, wl.prompt))).cuda()
+    for rep in range(2):
+        cur = ctx.prefill(ids)
+        for _ in range(n_dec):
+            cur = ctx.decode_step(cur)
+        ctx.release_slot(0)
+        torch.cuda.synchronize()
+    assert ctx.status() == 0
+    print(json.dumps({"profile_case": "stack", "config": wl.key, "batch": B, "layers": 2, "decode_steps": n_dec,
+                      "launches": ctx.launch_count()}))
+    ctx.close()
+    return 0
+
+
 def run_profile_case(args, wl):
     """A small, self-ending case for ncu: ONE layer of the configuration (its shapes, batch and prompt, so every
     launch equals the one in the full model), one warm-up pass, then one pass of the chosen phase."""
@@ -597,14 +625,17 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (c2: 1, 4, 16)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile", choices=["prefill", "decode"], default=None,
-                    help="run one small pass of a phase and exit (the case ncu captures)")
+    ap.add_argument("--profile", choices=["prefill", "decode", "stack"], default=None,
+                    help="run one small pass and exit (the cases ncu captures): one layer of the configuration, "
+                         "prefill or decode phase; or a two-layer stack with the head (the launch list)")
     ap.add_argument("--profile-decode-steps", type=int, default=2)
     ap.add_argument("--tables", action="store_true", help="operator micro-benchmarks at the paper's Table 8 / 9 shapes")
     args = ap.parse_args()
     wl = WORKLOADS[args.config]
     if args.tables:
         return run_tables(args)
+    if args.profile == "stack":
+        return run_profile_stack(args, wl)
     if args.profile:
         return run_profile_case(args, wl)
     if args.impl == "reference":

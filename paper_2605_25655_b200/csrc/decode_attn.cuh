@@ -15,6 +15,7 @@ namespace thinfer {
 
 constexpr int kAttnDecWarps = 4;
 constexpr int kAttnDecUnroll = 4;
+constexpr int kAttnMaxSplits = 32;
 
 struct AttnDecArgs {
   const __half* q;        // [batch][n_q_heads][D], already rotated
@@ -30,6 +31,7 @@ struct AttnDecArgs {
   int t_max;
   int splits, chunk;      // chunk = keys per split
   float scale_log2;       // log2(e) / sqrt(D)
+  unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
 };
 
 // Streams keys t_first, t_first + t_step, ... (< t_end) in groups of UN*KPL and folds them into the
@@ -137,7 +139,12 @@ __device__ __forceinline__ void attn_merge_lane_groups(float (&m)[G], float (&l)
 template <int D, int G>
 __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const AttnDecArgs a) {
   pdl_launch_dependents();
+  if (a.dbg != nullptr && threadIdx.x == 0) {
+    atomicMin(a.dbg + 10, static_cast<unsigned long long>(global_ns()));  // earliest CTA start
+    atomicMax(a.dbg + 12, static_cast<unsigned long long>(global_ns()));  // latest CTA start
+  }
   pdl_wait();
+  if (a.dbg != nullptr && threadIdx.x == 0) atomicMin(a.dbg + 11, static_cast<unsigned long long>(global_ns()));
   constexpr int LPK = D / 8;     // lanes that cover one key row
   constexpr int KPL = 32 / LPK;  // keys per warp-wide load
   constexpr int UN = kAttnDecUnroll;
@@ -173,6 +180,10 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
   }
 
   attn_stream_keys<D, G>(kb, vb, q, t0 + warp * (UN * KPL), t1, kAttnDecWarps * UN * KPL, sub, m, l, o);
+  if (a.dbg != nullptr && lane == 0) {
+    atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // latest stream end of a warp
+    atomicMin(a.dbg + 9, static_cast<unsigned long long>(global_ns()));   // earliest
+  }
   attn_merge_lane_groups<D, G>(m, l, o);
   if (sub == 0) {
 #pragma unroll
@@ -212,6 +223,7 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
       }
     }
   }
+  if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 14, static_cast<unsigned long long>(global_ns()));
   if (a.splits == 1) return;
 
   // split-KV: the CTA that arrives last merges the partials of its G heads,
@@ -228,20 +240,52 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
-    const int g = idx / D, i = idx - g * D;
-    const size_t bh = static_cast<size_t>(b) * a.n_q_heads + h0 + g;
-    float mx = -INFINITY;
-    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, __ldcg(a.part_ml + (bh * a.splits + s) * 2));
-    float L = 0.f, O = 0.f;
-    for (int s = 0; s < a.splits; ++s) {
-      const size_t p = bh * a.splits + s;
-      const float al = exp2f(__ldcg(a.part_ml + p * 2) - mx);
-      L += __ldcg(a.part_ml + p * 2 + 1) * al;
-      O += __ldcg(a.part_o + p * D + i) * al;
-    }
-    a.out[bh * D + i] = __float2half_rn(O / L);
+  // The partials come from L2.  First the (max, sum) pairs of all splits of the G heads in one parallel round
+  // trip, from them the weight 2^(m_s - M) / L of every split; then every thread adds its output elements over
+  // the splits, in split order, with several independent 16-byte loads in flight.
+  __shared__ float sm_pm[G][kAttnMaxSplits], sm_pl[G][kAttnMaxSplits];
+  const size_t bh0 = static_cast<size_t>(b) * a.n_q_heads + h0;
+  for (int idx = threadIdx.x; idx < G * a.splits; idx += kAttnDecWarps * 32) {
+    const int g = idx / a.splits, s = idx - g * a.splits;
+    const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + ((bh0 + g) * a.splits + s) * 2));
+    sm_pm[g][s] = ml.x;
+    sm_pl[g][s] = ml.y;
   }
+  __syncthreads();
+  if (threadIdx.x < G) {
+    const int g = threadIdx.x;
+    float mx = -INFINITY;
+    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, sm_pm[g][s]);
+    float L = 0.f;
+    for (int s = 0; s < a.splits; ++s) {
+      const float al = exp2f(sm_pm[g][s] - mx);
+      L += sm_pl[g][s] * al;
+      sm_pm[g][s] = al;
+    }
+    sm_pl[g][0] = 1.f / L;
+  }
+  __syncthreads();
+  constexpr int V4 = G * D / 4;  // 16-byte pieces of the G output rows
+  for (int idx = threadIdx.x; idx < V4; idx += kAttnDecWarps * 32) {
+    const int g = idx / (D / 4), i4 = idx - g * (D / 4);
+    const float4* src = reinterpret_cast<const float4*>(a.part_o + (bh0 + g) * a.splits * D) + i4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int s = 0; s < a.splits; ++s) {
+      const float4 v = __ldcg(src + static_cast<size_t>(s) * (D / 4));
+      const float al = sm_pm[g][s];
+      acc.x = fmaf(v.x, al, acc.x);
+      acc.y = fmaf(v.y, al, acc.y);
+      acc.z = fmaf(v.z, al, acc.z);
+      acc.w = fmaf(v.w, al, acc.w);
+    }
+    const float inv = sm_pl[g][0];
+    uint2 o;
+    o.x = pack2(acc.x * inv, acc.y * inv);
+    o.y = pack2(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(a.out + (bh0 + g) * D + i4 * 4) = o;
+  }
+  if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));
 }
 
 }  // namespace thinfer

@@ -134,6 +134,7 @@ struct thinfer_ctx {
   MegaLayer* mega_layers = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
+  int attn_ctas_per_sm = 2, attn_min_chunk = 128;  // split-KV policy of decode attention (tuning aids)
   // status word (pinned, mapped)
   int* status_host = nullptr;
   int* status_dev = nullptr;
@@ -621,14 +622,15 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   const int ratio = cf.n_q_heads / cf.n_kv_heads;
   int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
   const int ctas = batch * (cf.n_q_heads / g);
-  int splits = (2 * c->sm_count + ctas - 1) / ctas;
-  const int by_len = (t_len + 127) / 128;  // at least 128 keys per split (64 measured the same)
+  int splits = (c->attn_ctas_per_sm * c->sm_count + ctas - 1) / ctas;
+  const int by_len = (t_len + c->attn_min_chunk - 1) / c->attn_min_chunk;  // keys per split: not fewer than this
   if (splits > by_len) splits = by_len;
   if (splits > c->max_splits) splits = c->max_splits;
   if (splits < 1) splits = 1;
   a.chunk = (t_len + splits - 1) / splits;
   a.splits = (t_len + a.chunk - 1) / a.chunk;
   a.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(cf.head_dim));
+  if (c->trace_unified) a.dbg = c->timeline + 16 * THINFER_K_ATTN;
   if (cf.head_dim == 128) attn_decode_d<128>(L, a, batch, ratio);
   else attn_decode_d<64>(L, a, batch, ratio);
 }
@@ -1254,6 +1256,17 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->d_stage_in = s + p.d_stage_in;
   c->d_stage_out = s + p.d_stage_out;
   c->max_splits = p.max_splits;
+  {
+    // tuning aids for experiments; the defaults are what the library is measured with
+    auto env_int = [](const char* name, int lo, int hi, int dflt) {
+      const char* v = std::getenv(name);
+      if (v == nullptr || *v == 0) return dflt;
+      const long x = std::strtol(v, nullptr, 10);
+      return x < lo || x > hi ? dflt : static_cast<int>(x);
+    };
+    c->attn_ctas_per_sm = env_int("THINFER_ATTN_CTAS_PER_SM", 1, 32, c->attn_ctas_per_sm);
+    c->attn_min_chunk = env_int("THINFER_ATTN_MIN_CHUNK", 8, 4096, c->attn_min_chunk);
+  }
 
   auto cleanup = [&](int code) {
     for (Slot& sl : c->slots) {
