@@ -2,12 +2,13 @@
 // (request, head), the M = 1 case of the staged attention of Section 3.3.2.
 // Per request (selective batching, Section 3.4.1) and bandwidth-bound: K and V
 // rows are streamed once with 128-bit loads; the query heads that share a KV
-// head are processed in the same pass.  The KV range is split across CTAs
-// (split-KV); every lane group keeps a running (max, sum, output) triple that
-// is merged by the online-softmax rule first inside the warp, then across the
-// CTA's warps, then across splits by whichever CTA of a (request, head group)
-// finishes last (a ticket counter; the partials are added in split order, so the
-// result does not depend on who that is).
+// head are processed in the same pass.  The KV ranges are split across CTAs
+// (split-KV, in equal runs over a grid that fills the device once); every lane
+// group keeps a running (max, sum, output) triple that is merged by the
+// online-softmax rule first inside the warp, then across the CTA's warps, then
+// across the segments of a (request, head group) by whichever of its CTAs
+// finishes last (a ticket counter; the partials are added in segment order, so
+// the result does not depend on who that is).
 #pragma once
 #include "common.cuh"
 
@@ -22,14 +23,15 @@ struct AttnDecArgs {
   const __half* k_cache;  // [max_batch][n_kv_heads][t_max][D]
   const __half* v_cache;
   __half* out;            // [batch][n_q_heads * D]
-  float* part_o;          // [batch][n_q_heads][splits][D]   un-normalised partial outputs
-  float* part_ml;         // [batch][n_q_heads][splits][2]   (max in log2 units, sum)
-  int* tickets;           // [batch][n_q_heads / G] arrival counters, zero between launches (splits > 1)
+  float* part_o;          // [batch][n_q_heads][kAttnMaxSplits][D]   un-normalised partial outputs of the segments
+  float* part_ml;         // [batch][n_q_heads][kAttnMaxSplits][2]   (max in log2 units, sum)
+  int* tickets;           // [batch][n_q_heads / G] arrival counters, zero between launches
   int n_q_heads, n_kv_heads;
   int t_len;              // keys to attend: positions 0 .. t_len-1
   const int* len_arr;     // ragged: request b attends len_arr[b] + t_len keys (nullptr: t_len for everybody)
   int t_max;
-  int splits, chunk;      // chunk = keys per split
+  int n_pairs;            // batch * n_q_heads / G
+  int units_per_pair;     // ceil(longest key count / keys per CTA-wide iteration)
   float scale_log2;       // log2(e) / sqrt(D)
   unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
 };
@@ -136,6 +138,115 @@ __device__ __forceinline__ void attn_merge_lane_groups(float (&m)[G], float (&l)
   }
 }
 
+// Shared-memory state of one CTA for merging: per warp the running (max, sum, output) of its keys, and the
+// weights of a pair's segments during the final merge.
+template <int D, int G>
+struct AttnMergeSmem {
+  float m[kAttnDecWarps][G], l[kAttnDecWarps][G];
+  float o[kAttnDecWarps][G][D];
+  float pm[G][kAttnMaxSplits], pl[G][kAttnMaxSplits];
+  int is_last;
+};
+
+// Second half of a segment, after every warp has left its state in `sm` and the CTA has synchronised: merges the
+// warps; a pair with one segment is finished here, otherwise the segment's partial goes to global memory and the
+// CTA of the pair that arrives last merges all of them, in segment order.
+template <int D, int G>
+__device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMergeSmem<D, G>& sm, int b, int h0, int pair,
+                                                    int seg, int n_seg) {
+  const size_t bh0 = static_cast<size_t>(b) * a.n_q_heads + h0;
+  for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
+    const int g = idx / D, i = idx - g * D;
+    float mx = sm.m[0][g];
+#pragma unroll
+    for (int w = 1; w < kAttnDecWarps; ++w) mx = fmaxf(mx, sm.m[w][g]);
+    const float ms = (mx == -INFINITY) ? 0.f : mx;
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnDecWarps; ++w) {
+      const float al = exp2f(sm.m[w][g] - ms);
+      L += sm.l[w][g] * al;
+      O += sm.o[w][g][i] * al;
+    }
+    if (n_seg == 1) {
+      a.out[(bh0 + g) * D + i] = __float2half_rn(O / L);
+    } else {
+      const size_t p = (bh0 + g) * kAttnMaxSplits + seg;
+      a.part_o[p * D + i] = O;
+      if (i == 0) {
+        a.part_ml[p * 2] = mx;
+        a.part_ml[p * 2 + 1] = L;
+      }
+    }
+  }
+  if (n_seg > 1) {
+    // the CTA that arrives last merges the segments of its G heads,
+    // out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), s in segment order
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int* ctr = a.tickets + pair;
+      const int ticket = atomicAdd(ctr, 1);
+      sm.is_last = ticket == n_seg - 1;
+      if (sm.is_last) *ctr = 0;  // ready for the next launch
+    }
+    __syncthreads();
+    if (sm.is_last) {
+      __threadfence();
+      // The partials come from L2.  First the (max, sum) pairs of all segments of the G heads in one parallel
+      // round trip, from them the weight 2^(m_s - M) of every segment and 1 / L; then every thread adds its
+      // output elements over the segments, in segment order, with several 16-byte loads in flight.
+      for (int idx = threadIdx.x; idx < G * n_seg; idx += kAttnDecWarps * 32) {
+        const int g = idx / n_seg, sg = idx - g * n_seg;
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + ((bh0 + g) * kAttnMaxSplits + sg) * 2));
+        sm.pm[g][sg] = ml.x;
+        sm.pl[g][sg] = ml.y;
+      }
+      __syncthreads();
+      if (threadIdx.x < G) {
+        const int g = threadIdx.x;
+        float mx = -INFINITY;
+        for (int sg = 0; sg < n_seg; ++sg) mx = fmaxf(mx, sm.pm[g][sg]);
+        float L = 0.f;
+        for (int sg = 0; sg < n_seg; ++sg) {
+          const float al = exp2f(sm.pm[g][sg] - mx);  // an empty segment has max -inf: weight 0
+          L += sm.pl[g][sg] * al;
+          sm.pm[g][sg] = al;
+        }
+        sm.pl[g][0] = 1.f / L;
+      }
+      __syncthreads();
+      constexpr int V4 = G * D / 4;  // 16-byte pieces of the G output rows
+      for (int idx = threadIdx.x; idx < V4; idx += kAttnDecWarps * 32) {
+        const int g = idx / (D / 4), i4 = idx - g * (D / 4);
+        const float4* src = reinterpret_cast<const float4*>(a.part_o + (bh0 + g) * kAttnMaxSplits * D) + i4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int sg = 0; sg < n_seg; ++sg) {
+          const float4 v = __ldcg(src + static_cast<size_t>(sg) * (D / 4));
+          const float al = sm.pm[g][sg];
+          acc.x = fmaf(v.x, al, acc.x);
+          acc.y = fmaf(v.y, al, acc.y);
+          acc.z = fmaf(v.z, al, acc.z);
+          acc.w = fmaf(v.w, al, acc.w);
+        }
+        const float inv = sm.pl[g][0];
+        uint2 ov;
+        ov.x = pack2(acc.x * inv, acc.y * inv);
+        ov.y = pack2(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(a.out + (bh0 + g) * D + i4 * 4) = ov;
+      }
+    }
+  }
+}
+
+// Balanced split-KV schedule.  A "pair" is one request and one group of G query heads that share a KV head;
+// its keys are cut into units of one CTA-wide iteration (kAttnDecWarps x UN x KPL keys).  The units of all pairs,
+// laid end to end, are dealt out in equal contiguous runs to a grid that fills the resident CTA slots of the
+// device exactly once: every CTA streams the same number of keys (+- one unit) whatever the batch, head count
+// and sequence length are, so there is neither a partly filled last wave nor an idle SM.  A run may end inside
+// a pair and continue into the next one: a CTA then works on up to a few (pair, key range) segments in turn.
+// The segments of a pair are merged by whichever of its CTAs finishes last (ticket counter), in segment order.
 template <int D, int G>
 __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const AttnDecArgs a) {
   pdl_launch_dependents();
@@ -148,142 +259,71 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
   constexpr int LPK = D / 8;     // lanes that cover one key row
   constexpr int KPL = 32 / LPK;  // keys per warp-wide load
   constexpr int UN = kAttnDecUnroll;
-  __shared__ float sm_m[kAttnDecWarps][G], sm_l[kAttnDecWarps][G];
-  __shared__ float sm_o[kAttnDecWarps][G][D];
+  constexpr int UNIT = kAttnDecWarps * UN * KPL;  // keys of one CTA-wide iteration
+  __shared__ AttnMergeSmem<D, G> sm;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane / LPK, dl = lane % LPK;
-  const int split = blockIdx.x, b = blockIdx.z;
-  const int h0 = blockIdx.y * G;                                   // first query head of this CTA
-  const int hk = h0 / (a.n_q_heads / a.n_kv_heads);
-  const int t_len = a.t_len + (a.len_arr != nullptr ? a.len_arr[b] : 0);
-  const int t0 = split * a.chunk;
-  const int t1 = min(t_len, t0 + a.chunk);
+  const int groups = a.n_q_heads / G;                // pairs per request
+  const long long n_units = static_cast<long long>(a.n_pairs) * a.units_per_pair;
+  const long long grid = gridDim.x;
+  const long long u_beg = static_cast<long long>(blockIdx.x) * n_units / grid;
+  const long long u_end = (static_cast<long long>(blockIdx.x) + 1) * n_units / grid;
+  // the CTA that holds unit x: the largest i with floor(i * n_units / grid) <= x
+  auto cta_of = [&](long long x) { return static_cast<int>(((x + 1) * grid - 1) / n_units); };
 
-  float q[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    unpack8(ldg_cached(a.q + (static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + dl * 8), q[g]);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) q[g][i] *= a.scale_log2;
-  }
-  const __half* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
-  const __half* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+  for (long long u = u_beg; u < u_end;) {
+    const int pair = static_cast<int>(u / a.units_per_pair);
+    const long long pair_u0 = static_cast<long long>(pair) * a.units_per_pair;
+    const long long seg_end = min(u_end, pair_u0 + a.units_per_pair);
+    const int b = pair / groups, h0 = (pair - b * groups) * G;
+    const int hk = h0 / (a.n_q_heads / a.n_kv_heads);
+    const int t_len = a.t_len + (a.len_arr != nullptr ? a.len_arr[b] : 0);
+    const int t0 = static_cast<int>(u - pair_u0) * UNIT;
+    const int t1 = min(t_len, static_cast<int>(seg_end - pair_u0) * UNIT);
+    const int first_cta = cta_of(pair_u0), n_seg = cta_of(pair_u0 + a.units_per_pair - 1) - first_cta + 1;
+    const int seg = static_cast<int>(blockIdx.x) - first_cta;
+    u = seg_end;
 
-  float m[G], l[G], o[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    m[g] = -INFINITY;
-    l[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
-  }
-
-  attn_stream_keys<D, G>(kb, vb, q, t0 + warp * (UN * KPL), t1, kAttnDecWarps * UN * KPL, sub, m, l, o);
-  if (a.dbg != nullptr && lane == 0) {
-    atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // latest stream end of a warp
-    atomicMin(a.dbg + 9, static_cast<unsigned long long>(global_ns()));   // earliest
-  }
-  attn_merge_lane_groups<D, G>(m, l, o);
-  if (sub == 0) {
+    float q[G][8];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      if (dl == 0) {
-        sm_m[warp][g] = m[g];
-        sm_l[warp][g] = l[g];
-      }
+      unpack8(ldg_cached(a.q + (static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + dl * 8), q[g]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) sm_o[warp][g][dl * 8 + i] = o[g][i];
+      for (int i = 0; i < 8; ++i) q[g][i] *= a.scale_log2;
     }
-  }
-  __syncthreads();
+    const __half* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+    const __half* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
 
-  for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
-    const int g = idx / D, i = idx - g * D;
-    float mx = sm_m[0][g];
+    float m[G], l[G], o[G][8];
 #pragma unroll
-    for (int w = 1; w < kAttnDecWarps; ++w) mx = fmaxf(mx, sm_m[w][g]);
-    const float ms = (mx == -INFINITY) ? 0.f : mx;
-    float L = 0.f, O = 0.f;
+    for (int g = 0; g < G; ++g) {
+      m[g] = -INFINITY;
+      l[g] = 0.f;
 #pragma unroll
-    for (int w = 0; w < kAttnDecWarps; ++w) {
-      const float al = exp2f(sm_m[w][g] - ms);
-      L += sm_l[w][g] * al;
-      O += sm_o[w][g][i] * al;
+      for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
     }
-    const int h = h0 + g;
-    if (a.splits == 1) {
-      a.out[(static_cast<size_t>(b) * a.n_q_heads + h) * D + i] = __float2half_rn(O / L);
-    } else {
-      const size_t p = (static_cast<size_t>(b) * a.n_q_heads + h) * a.splits + split;
-      a.part_o[p * D + i] = O;
-      if (i == 0) {
-        a.part_ml[p * 2] = mx;
-        a.part_ml[p * 2 + 1] = L;
+
+    attn_stream_keys<D, G>(kb, vb, q, t0 + warp * (UN * KPL), t1, UNIT, sub, m, l, o);
+    if (a.dbg != nullptr && lane == 0) {
+      atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // latest stream end of a warp
+      atomicMin(a.dbg + 9, static_cast<unsigned long long>(global_ns()));   // earliest
+    }
+    attn_merge_lane_groups<D, G>(m, l, o);
+    if (sub == 0) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        if (dl == 0) {
+          sm.m[warp][g] = m[g];
+          sm.l[warp][g] = l[g];
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sm.o[warp][g][dl * 8 + i] = o[g][i];
       }
     }
-  }
-  if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 14, static_cast<unsigned long long>(global_ns()));
-  if (a.splits == 1) return;
-
-  // split-KV: the CTA that arrives last merges the partials of its G heads,
-  // out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), s in split order
-  __shared__ int is_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int* ctr = a.tickets + b * gridDim.y + blockIdx.y;
-    const int ticket = atomicAdd(ctr, 1);
-    is_last = ticket == a.splits - 1;
-    if (is_last) *ctr = 0;  // ready for the next launch
-  }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  // The partials come from L2.  First the (max, sum) pairs of all splits of the G heads in one parallel round
-  // trip, from them the weight 2^(m_s - M) / L of every split; then every thread adds its output elements over
-  // the splits, in split order, with several independent 16-byte loads in flight.
-  __shared__ float sm_pm[G][kAttnMaxSplits], sm_pl[G][kAttnMaxSplits];
-  const size_t bh0 = static_cast<size_t>(b) * a.n_q_heads + h0;
-  for (int idx = threadIdx.x; idx < G * a.splits; idx += kAttnDecWarps * 32) {
-    const int g = idx / a.splits, s = idx - g * a.splits;
-    const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + ((bh0 + g) * a.splits + s) * 2));
-    sm_pm[g][s] = ml.x;
-    sm_pl[g][s] = ml.y;
-  }
-  __syncthreads();
-  if (threadIdx.x < G) {
-    const int g = threadIdx.x;
-    float mx = -INFINITY;
-    for (int s = 0; s < a.splits; ++s) mx = fmaxf(mx, sm_pm[g][s]);
-    float L = 0.f;
-    for (int s = 0; s < a.splits; ++s) {
-      const float al = exp2f(sm_pm[g][s] - mx);
-      L += sm_pl[g][s] * al;
-      sm_pm[g][s] = al;
-    }
-    sm_pl[g][0] = 1.f / L;
-  }
-  __syncthreads();
-  constexpr int V4 = G * D / 4;  // 16-byte pieces of the G output rows
-  for (int idx = threadIdx.x; idx < V4; idx += kAttnDecWarps * 32) {
-    const int g = idx / (D / 4), i4 = idx - g * (D / 4);
-    const float4* src = reinterpret_cast<const float4*>(a.part_o + (bh0 + g) * a.splits * D) + i4;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int s = 0; s < a.splits; ++s) {
-      const float4 v = __ldcg(src + static_cast<size_t>(s) * (D / 4));
-      const float al = sm_pm[g][s];
-      acc.x = fmaf(v.x, al, acc.x);
-      acc.y = fmaf(v.y, al, acc.y);
-      acc.z = fmaf(v.z, al, acc.z);
-      acc.w = fmaf(v.w, al, acc.w);
-    }
-    const float inv = sm_pl[g][0];
-    uint2 o;
-    o.x = pack2(acc.x * inv, acc.y * inv);
-    o.y = pack2(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2*>(a.out + (bh0 + g) * D + i4 * 4) = o;
+    __syncthreads();
+    attn_finish_segment<D, G>(a, sm, b, h0, pair, seg, n_seg);
+    __syncthreads();  // the shared arrays are reused by the next segment
   }
   if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));
 }

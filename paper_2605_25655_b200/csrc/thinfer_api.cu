@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "decode_attn.cuh"
+#include "decode_attn_gqa.cuh"
 #include "decode_gemv.cuh"
 #include "decode_mega.cuh"
 #include "decode_mma.cuh"
@@ -134,7 +135,7 @@ struct thinfer_ctx {
   MegaLayer* mega_layers = nullptr;
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
-  int attn_ctas_per_sm = 2, attn_min_chunk = 128;  // split-KV policy of decode attention (tuning aids)
+  int attn_waves = 1, attn_min_units = 2;  // split-KV schedule of decode attention (tuning aids)
   // status word (pinned, mapped)
   int* status_host = nullptr;
   int* status_dev = nullptr;
@@ -202,7 +203,7 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
   };
   const size_t M = static_cast<size_t>(c.max_batch) * c.max_seq;
   const size_t qd = static_cast<size_t>(c.n_q_heads) * c.head_dim;
-  p.max_splits = 32;
+  p.max_splits = kAttnMaxSplits;
   p.rope_cos = take(static_cast<size_t>(c.max_seq) * (c.head_dim / 2) * 4);
   p.rope_sin = take(static_cast<size_t>(c.max_seq) * (c.head_dim / 2) * 4);
   p.h = take(M * c.hidden * 2);
@@ -588,23 +589,67 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
 // ----------------------------------------------------------------------------
 // attention dispatch
 // ----------------------------------------------------------------------------
-template <int D>
-void attn_decode_d(Launcher& L, const AttnDecArgs& a, int batch, int ratio) {
-  int g = 1;
-  if (ratio % 8 == 0) g = 8;
-  else if (ratio % 4 == 0) g = 4;
-  else if (ratio % 2 == 0) g = 2;
-  const dim3 grid(a.splits, a.n_q_heads / g, batch), block(kAttnDecWarps * 32);
-  switch (g) {
-    case 8: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 8>, grid, block, 0, a); break;
-    case 4: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 4>, grid, block, 0, a); break;
-    case 2: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 2>, grid, block, 0, a); break;
-    default: L.go(THINFER_K_ATTN, attn_decode_kernel<D, 1>, grid, block, 0, a); break;
+// One decode-attention launch on the balanced split-KV schedule.  `unit`: keys of one CTA-wide iteration of the
+// kernel; `smem`: its dynamic shared memory.  The number of CTAs that fit on the device at once is asked of the
+// runtime once per kernel and device.
+template <void (*kernel)(const AttnDecArgs)>
+void launch_attn_decode(Launcher& L, thinfer_ctx* c, int unit, int smem, int pairs_per_request, AttnDecArgs a,
+                        int batch, int t_len) {
+  static SmemOptIn opt;
+  static int per_sm[SmemOptIn::kMaxDevices] = {};
+  if (smem > 0 && !opt.ensure(kernel, smem)) {
+    L.rc = fail(c, THINFER_ECUDA, "cannot reserve %d bytes of shared memory", smem);
+    return;
+  }
+  int dev = 0, ctas_per_sm = 2;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < SmemOptIn::kMaxDevices) {
+    if (per_sm[dev] == 0) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kAttnDecWarps * 32, smem) != cudaSuccess || n < 1) n = 2;
+      per_sm[dev] = n;
+    }
+    ctas_per_sm = per_sm[dev];
+  }
+  a.n_pairs = batch * pairs_per_request;
+  a.units_per_pair = (t_len + unit - 1) / unit;
+  const long long n_units = static_cast<long long>(a.n_pairs) * a.units_per_pair;
+  // One CTA per resident slot (times attn_waves, a tuning aid), every CTA the same number of units; not more
+  // CTAs than pairs of units, and few enough that no pair is cut into more than kAttnMaxSplits segments.
+  const long long slots = static_cast<long long>(ctas_per_sm) * c->sm_count * c->attn_waves;
+  long long grid = slots;
+  grid = std::min(grid, std::max<long long>(1, n_units / c->attn_min_units));
+  grid = std::min(grid, static_cast<long long>(kAttnMaxSplits - 2) * a.n_pairs);
+  // Every segment costs a query load, a merge and a ticket.  When a whole number of equal segments per pair
+  // fills at least 80 % of the slots, that grid (every CTA exactly one segment) beats the exactly balanced one.
+  const long long per_pair = grid / a.n_pairs;
+  if (per_pair >= 1 && per_pair * a.n_pairs * 10 >= slots * 8) grid = per_pair * a.n_pairs;
+  L.go(THINFER_K_ATTN, kernel, dim3(static_cast<unsigned>(grid)), dim3(kAttnDecWarps * 32), smem, a);
+}
+
+template <int D, int G>
+void attn_decode_dg(Launcher& L, thinfer_ctx* c, const AttnDecArgs& a, int batch, int t_len) {
+  if constexpr (G >= 4) {
+    // grouped-query models: the G heads of a pair are the rows of a tensor-core tile
+    launch_attn_decode<attn_decode_gqa_kernel<D, G>>(L, c, kGqaUnit, gqa_ring_bytes<D>(), a.n_q_heads / G, a, batch, t_len);
+  } else {
+    constexpr int kUnit = kAttnDecWarps * kAttnDecUnroll * (32 / (D / 8));
+    launch_attn_decode<attn_decode_kernel<D, G>>(L, c, kUnit, 0, a.n_q_heads / G, a, batch, t_len);
   }
 }
 
+template <int D>
+void attn_decode_d(Launcher& L, thinfer_ctx* c, const AttnDecArgs& a, int batch, int t_len, int ratio) {
+  if (ratio % 8 == 0) attn_decode_dg<D, 8>(L, c, a, batch, t_len);
+  else if (ratio % 4 == 0) attn_decode_dg<D, 4>(L, c, a, batch, t_len);
+  else if (ratio % 2 == 0) attn_decode_dg<D, 2>(L, c, a, batch, t_len);
+  else attn_decode_dg<D, 1>(L, c, a, batch, t_len);
+}
+
+// t_len: keys the longest request attends (the unit count of the schedule); with `len_arr` (ragged slots) request b
+// attends len_arr[b] + len_add keys
 void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc, const __half* vc, __half* out,
                  int batch, int t_len, const int* len_arr = nullptr, int len_add = 0) {
+  if (L.rc != THINFER_OK) return;
   const thinfer_config& cf = c->cfg;
   AttnDecArgs a{};
   a.q = q;
@@ -619,20 +664,11 @@ void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc,
   a.t_len = len_arr != nullptr ? len_add : t_len;  // ragged: per-request count = len_arr[b] + len_add
   a.len_arr = len_arr;
   a.t_max = cf.max_seq;
-  const int ratio = cf.n_q_heads / cf.n_kv_heads;
-  int g = (ratio % 8 == 0) ? 8 : (ratio % 4 == 0) ? 4 : (ratio % 2 == 0) ? 2 : 1;
-  const int ctas = batch * (cf.n_q_heads / g);
-  int splits = (c->attn_ctas_per_sm * c->sm_count + ctas - 1) / ctas;
-  const int by_len = (t_len + c->attn_min_chunk - 1) / c->attn_min_chunk;  // keys per split: not fewer than this
-  if (splits > by_len) splits = by_len;
-  if (splits > c->max_splits) splits = c->max_splits;
-  if (splits < 1) splits = 1;
-  a.chunk = (t_len + splits - 1) / splits;
-  a.splits = (t_len + a.chunk - 1) / a.chunk;
   a.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(cf.head_dim));
   if (c->trace_unified) a.dbg = c->timeline + 16 * THINFER_K_ATTN;
-  if (cf.head_dim == 128) attn_decode_d<128>(L, a, batch, ratio);
-  else attn_decode_d<64>(L, a, batch, ratio);
+  const int ratio = cf.n_q_heads / cf.n_kv_heads;
+  if (cf.head_dim == 128) attn_decode_d<128>(L, c, a, batch, t_len, ratio);
+  else attn_decode_d<64>(L, c, a, batch, t_len, ratio);
 }
 
 template <int D>
@@ -1264,8 +1300,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
       const long x = std::strtol(v, nullptr, 10);
       return x < lo || x > hi ? dflt : static_cast<int>(x);
     };
-    c->attn_ctas_per_sm = env_int("THINFER_ATTN_CTAS_PER_SM", 1, 32, c->attn_ctas_per_sm);
-    c->attn_min_chunk = env_int("THINFER_ATTN_MIN_CHUNK", 8, 4096, c->attn_min_chunk);
+    c->attn_waves = env_int("THINFER_ATTN_WAVES", 1, 8, c->attn_waves);
+    c->attn_min_units = env_int("THINFER_ATTN_MIN_UNITS", 1, 64, c->attn_min_units);
   }
 
   auto cleanup = [&](int code) {
