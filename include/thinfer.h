@@ -233,7 +233,9 @@ int thinfer_profile_read(thinfer_ctx* ctx, int32_t* launches, float* total_ms);
  * QKV done, barrier, attention done, barrier, O done, barrier, gate/up done, barrier, down done
  * (, barrier).  While tracing is on, the stream-K projections of the per-unit decode path also store, per
  * thinfer_kernel_id k, in entries 16k+10 .. 16k+15: earliest CTA start, earliest pass of the dependency wait,
- * latest load issued, latest MMA issued, latest accumulator ready, latest epilogue end.  max_entries <= 256.
+ * latest load issued, latest MMA issued, latest accumulator ready, latest epilogue end.  max_entries <= 4352: entries
+ * from 256 on hold, for the kernel id named by the environment variable THINFER_TRACE_CTA_KID at thinfer_create, four
+ * values per CTA of its last launch (SM id, time past the dependency wait, last warp's stream end, end).
  * Host pointer; tracing aid, not part of the hot path. */
 int thinfer_trace_unified(thinfer_ctx* ctx, int32_t enable, uint64_t* host_out, int32_t max_entries);
 

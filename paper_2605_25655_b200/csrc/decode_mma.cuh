@@ -54,6 +54,7 @@ struct SkinnyArgs {
   int tiles_max;       // row tiles of the largest CTA share (<= TM)
   EpiArgs e;           // RESID with outg: e.sumsq receives [gridDim.x][16]
   unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
+  unsigned long long* cta_log;  // tracing aid: per CTA {SM id, past the dependency wait, last warp's stream end, end} or nullptr
 };
 
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -188,6 +189,13 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   }
   pdl_wait();
   if (a.dbg != nullptr && threadIdx.x == 0) atomicMin(a.dbg + 11, static_cast<unsigned long long>(global_ns()));
+  if (a.cta_log != nullptr && threadIdx.x == 0) {
+    unsigned int smid;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+    a.cta_log[blockIdx.x * 4] = smid;
+    a.cta_log[blockIdx.x * 4 + 1] = global_ns();
+    a.cta_log[blockIdx.x * 4 + 2] = 0;
+  }
 
   if (a.sumsq_in != nullptr) {
     // asynchronous copies straight into shared memory: no registers held, consumed after the stream
@@ -285,6 +293,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
     atomicMax(a.dbg + 13, static_cast<unsigned long long>(global_ns()));  // latest stream end of a warp
     atomicMin(a.dbg + 9, static_cast<unsigned long long>(global_ns()));   // earliest
   }
+  if (a.cta_log != nullptr && lane == 0) atomicMax(a.cta_log + blockIdx.x * 4 + 2, static_cast<unsigned long long>(global_ns()));
   // park the fragments in this warp's own ring
   {
     float* dst = part + static_cast<size_t>(warp) * (ST * 512) + lane;
@@ -449,6 +458,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
     }
   }
   if (a.dbg != nullptr && lane == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));
+  if (a.cta_log != nullptr && threadIdx.x == 0) a.cta_log[blockIdx.x * 4 + 3] = global_ns();
 }
 
 }  // namespace thinfer

@@ -136,6 +136,8 @@ struct thinfer_ctx {
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
   int attn_waves = 1, attn_min_units = 2;  // split-KV schedule of decode attention (tuning aids)
+  int sk_max_tiles = 0;                    // tuning aid: cap on the tiles of a skinny share (0: the built-in limits)
+  int trace_cta_kid = -1;                  // kernel id whose CTAs log their own times while tracing is on
   // status word (pinned, mapped)
   int* status_host = nullptr;
   int* status_dev = nullptr;
@@ -245,7 +247,7 @@ ScratchPlan plan_scratch(const thinfer_config& c) {
     p.attn_partial = take((static_cast<size_t>(c.max_batch) * c.n_q_heads + kTcMaxCtas * 4) * (c.head_dim + 2) * 4);
     p.attn_counters = take(static_cast<size_t>(c.max_batch) * c.n_q_heads * 4);
     p.grid_bar = take(64);
-    p.timeline = take(256 * 8);
+    p.timeline = take((256 + 4 * 1024) * 8);  // 16 slots per kernel id, then 4 per CTA of one traced kernel
     p.mega_common = take(sizeof(MegaCommon));
     p.mega_layers = take(sizeof(MegaLayer) * c.n_layers);
   }
@@ -482,7 +484,9 @@ void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half
 // ----------------------------------------------------------------------------
 // skinny tensor-core streaming dispatch (decode, <= 16 tokens)
 // ----------------------------------------------------------------------------
-constexpr int kSkMaxTiles = 5;  // 16-row tiles per CTA share the kernels are instantiated for (1 .. 5)
+// 16-row tiles per CTA share the kernels are instantiated for: 1 .. 7 with one token tile (up to 8 requests),
+// 1 .. 6 with two (the accumulators of a share live in registers; beyond this they spill)
+constexpr int kSkMaxTiles1 = 7, kSkMaxTiles2 = 6;
 
 // Deals `grid` CTAs out to the matrices in proportion to their rows (every matrix with rows gets at least
 // one) and returns the largest number of tiles a CTA share has (mirrors the kernel's partition).
@@ -533,7 +537,12 @@ void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
     case 2: launch_skinny_tm<NT, 2, 4, EPI, NORM>(L, kid, grid, a); break;
     case 3: launch_skinny_tm<NT, 3, 4, EPI, NORM>(L, kid, grid, a); break;
     case 4: launch_skinny_tm<NT, 4, 4, EPI, NORM>(L, kid, grid, a); break;
-    default: launch_skinny_tm<NT, 5, 4, EPI, NORM>(L, kid, grid, a); break;
+    case 5: launch_skinny_tm<NT, 5, 4, EPI, NORM>(L, kid, grid, a); break;
+    case 6: launch_skinny_tm<NT, 6, 4, EPI, NORM>(L, kid, grid, a); break;
+    default:
+      if constexpr (NT == 1) launch_skinny_tm<NT, 7, 4, EPI, NORM>(L, kid, grid, a);
+      else L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection: %d tiles per share", a.tiles_max);
+      break;
   }
 }
 
@@ -560,6 +569,7 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
   a.e = e;
   if (L.c != nullptr && L.c->trace_unified && kid >= 0 && kid < 12) {
     a.dbg = L.c->timeline + 16 * kid;  // tracing aid: 16 slots per kernel id, reset at the start of the step
+    if (kid == L.c->trace_cta_kid) a.cta_log = L.c->timeline + 256;  // per-CTA times of this kernel (grid <= 1024)
   }
   const int units = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
   const bool swiglu = EPI == EPI_SWIGLU;
@@ -573,14 +583,19 @@ int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __hal
   const int by_work = std::max(units / 8, mats);
   if (grid > by_work) grid = by_work;
   a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
-  while (a.tiles_max > kSkMaxTiles && grid < 64 * sms) {
+  // A grid of two CTAs per SM is one wave of equal shares; more CTAs than that are dealt out as slots free up
+  // and some SMs end up with twice the work of others.  So the share grows before the grid does.
+  int max_tiles = rows <= 8 ? kSkMaxTiles1 : kSkMaxTiles2;
+  if (L.c != nullptr && L.c->sk_max_tiles > 0 && L.c->sk_max_tiles < max_tiles) max_tiles = L.c->sk_max_tiles;
+  while (a.tiles_max > max_tiles && grid < 64 * sms) {
     grid += sms;
     a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
   }
-  if (a.tiles_max > kSkMaxTiles) {
+  if (a.tiles_max > max_tiles) {
     L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection: %d tiles per share", a.tiles_max);
     return 0;
   }
+  if (grid > 1024) a.cta_log = nullptr;
   if (rows <= 8) launch_skinny<1, EPI, NORM>(L, kid, grid, a);
   else launch_skinny<2, EPI, NORM>(L, kid, grid, a);
   return grid;
@@ -1302,6 +1317,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     };
     c->attn_waves = env_int("THINFER_ATTN_WAVES", 1, 8, c->attn_waves);
     c->attn_min_units = env_int("THINFER_ATTN_MIN_UNITS", 1, 64, c->attn_min_units);
+    c->sk_max_tiles = env_int("THINFER_SK_MAX_TILES", 1, 7, 0);
+    c->trace_cta_kid = env_int("THINFER_TRACE_CTA_KID", 0, THINFER_K_COUNT - 1, -1);
   }
 
   auto cleanup = [&](int code) {
@@ -1597,7 +1614,7 @@ int thinfer_trace_unified(thinfer_ctx* c, int32_t enable, uint64_t* host_out, in
   if (c == nullptr) return THINFER_EINVAL;
   c->trace_unified = enable != 0;
   if (host_out != nullptr && max_entries > 0) {
-    const int n = max_entries < 256 ? max_entries : 256;
+    const int n = max_entries < 256 + 4 * 1024 ? max_entries : 256 + 4 * 1024;
     if (cudaMemcpy(host_out, c->timeline, static_cast<size_t>(n) * 8, cudaMemcpyDeviceToHost) != cudaSuccess)
       return fail(c, THINFER_ECUDA, "reading the timeline failed");
   }
