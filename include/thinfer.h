@@ -27,8 +27,13 @@
  *     synchronising.  Calls on one context must be issued from one thread at
  *     a time; work of one context must stay ordered on the device (use one
  *     stream, or order the streams with events).
- *   - Storage is IEEE FP16, accumulation and the norm / softmax reductions are
- *     FP32 (Section 3.2.4).  Matrices are row-major [out, in] (the paper's
+ *   - Storage is a 16-bit floating-point type, accumulation and the norm /
+ *     softmax reductions are FP32 (Section 3.2.4, which describes the operator
+ *     variants side by side: same kernels, different element type).  The
+ *     library is built once per storage type with the same exports:
+ *     libthinfer.so stores IEEE FP16, libthinfer_bf16.so stores BF16
+ *     (thinfer_storage_type() tells which one is loaded); wherever this
+ *     header says "FP16" the BF16 build reads and writes BF16 instead.  Matrices are row-major [out, in] (the paper's
  *     Y = X W, Section 3.2.1, with W stored transposed so that the contraction
  *     index is contiguous for both operands).
  *   - Device-side waits are bounded: a pipeline that does not make progress
@@ -85,6 +90,9 @@ typedef struct {
   const void *lm_head;                 /* device FP16 [vocab, hidden]; NULL when vocab == 0 */
 } thinfer_weights;
 
+/* Storage type of the loaded build (Section 3.2.4): 0 = IEEE FP16, 1 = BF16. */
+int thinfer_storage_type(void);
+
 /* Sizes of the two caller-allocated device regions.
  * kv_bytes: buf_slots x n_layers x {K,V} x [max_batch][n_kv_heads][max_seq][head_dim] FP16
  * (K is stored after RoPE, Algorithm 1).  scratch_bytes: activations, RoPE
@@ -130,6 +138,10 @@ int thinfer_prefill_ragged(thinfer_ctx* ctx, int32_t slot, const void* input, in
 /* Host query: positions each request of the slot holds (lens_out: host int32 [batch of the slot]). */
 int thinfer_slot_lengths(const thinfer_ctx* ctx, int32_t slot, int32_t* lens_out);
 
+/* Batch sizes.  Decode steps of up to 16 requests run on the weight-streaming skinny projections and are
+ * what the library is tuned and measured for (75 - 94 % of the device's copy bandwidth depending on the model);
+ * 17 .. 64 requests run on the stream-K tensor-core path, which is correct and tested but measured at 62 - 66 %
+ * (a step of 17 requests costs about 30 % more than one of 16).  Split larger batches into slots of 16. */
 /* One decode step for every request of `slot` (Section 3.4.1, selective
  * batching: projections batched over requests, attention per request).  The
  * new token sits at position cur_len (the number of positions the slot holds);

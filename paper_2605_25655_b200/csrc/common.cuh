@@ -3,11 +3,38 @@
 // pipelines (mbarrier, cp.async.bulk.tensor, tcgen05.alloc/mma/commit/ld/st).
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace thinfer {
+
+// ---------------------------------------------------------------- storage type
+// The library is compiled once per 16-bit storage type (Section 3.2.4 describes the operator variants side by
+// side: same kernel structure, different element type).  IEEE FP16 by default; -DTHINFER_BF16 gives the BF16
+// build.  Accumulation and every reduction are FP32 in both.  Everything below goes through these names:
+#ifdef THINFER_BF16
+using half_t = __nv_bfloat16;
+using half2_t = __nv_bfloat162;
+constexpr int kStorageType = 1;                 // thinfer_storage_type(): 1 = BF16
+constexpr unsigned int kTcOperandFormat = 1u;   // tcgen05 kind::f16 operand format field: BF16
+#define THINFER_MMA_SYNC_TYPES "bf16.bf16"
+__device__ __forceinline__ float2 h2_to_f2(half2_t v) { return __bfloat1622float2(v); }
+__device__ __forceinline__ float h_to_f(half_t v) { return __bfloat162float(v); }
+__device__ __forceinline__ half2_t f2_to_h2(float a, float b) { return __floats2bfloat162_rn(a, b); }
+__device__ __forceinline__ half_t f_to_h(float a) { return __float2bfloat16_rn(a); }
+#else
+using half_t = __half;
+using half2_t = __half2;
+constexpr int kStorageType = 0;                 // thinfer_storage_type(): 0 = IEEE FP16
+constexpr unsigned int kTcOperandFormat = 0u;   // tcgen05 kind::f16 operand format field: FP16
+#define THINFER_MMA_SYNC_TYPES "f16.f16"
+__device__ __forceinline__ float2 h2_to_f2(half2_t v) { return __half22float2(v); }
+__device__ __forceinline__ float h_to_f(half_t v) { return __half2float(v); }
+__device__ __forceinline__ half2_t f2_to_h2(float a, float b) { return __floats2half2_rn(a, b); }
+__device__ __forceinline__ half_t f_to_h(float a) { return __float2half_rn(a); }
+#endif
 
 constexpr int kErrTimeout = -6;  // THINFER_ETIMEOUT
 
@@ -25,16 +52,16 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // ------------------------------------------------------------- FP16 packing
 __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
+  const half2_t* h = reinterpret_cast<const half2_t*>(&v);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    float2 t = __half22float2(h[i]);
+    float2 t = h2_to_f2(h[i]);
     f[2 * i] = t.x;
     f[2 * i + 1] = t.y;
   }
 }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
-  __half2 h = __floats2half2_rn(a, b);
+  half2_t h = f2_to_h2(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
@@ -208,10 +235,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor for kind::f16 with FP16 A/B and FP32 D.
+// Instruction descriptor for kind::f16 with FP16 (or, in the BF16 build, BF16) A/B and FP32 D.
 // a_mn / b_mn: 0 = contraction index contiguous in shared memory, 1 = M (or N) index contiguous.
 __host__ __device__ constexpr uint32_t idesc_f16(int m, int n, int a_mn, int b_mn) {
-  return (1u << 4) | (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
+  return (1u << 4) | (kTcOperandFormat << 7) | (kTcOperandFormat << 10) | (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
          (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 

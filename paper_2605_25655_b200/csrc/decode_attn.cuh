@@ -19,10 +19,10 @@ constexpr int kAttnDecUnroll = 4;
 constexpr int kAttnMaxSplits = 32;
 
 struct AttnDecArgs {
-  const __half* q;        // [batch][n_q_heads][D], already rotated
-  const __half* k_cache;  // [max_batch][n_kv_heads][t_max][D]
-  const __half* v_cache;
-  __half* out;            // [batch][n_q_heads * D]
+  const half_t* q;        // [batch][n_q_heads][D], already rotated
+  const half_t* k_cache;  // [max_batch][n_kv_heads][t_max][D]
+  const half_t* v_cache;
+  half_t* out;            // [batch][n_q_heads * D]
   float* part_o;          // [batch][n_q_heads][kAttnMaxSplits][D]   un-normalised partial outputs of the segments
   float* part_ml;         // [batch][n_q_heads][kAttnMaxSplits][2]   (max in log2 units, sum)
   int* tickets;           // [batch][n_q_heads / G] arrival counters, zero between launches
@@ -39,7 +39,7 @@ struct AttnDecArgs {
 // Streams keys t_first, t_first + t_step, ... (< t_end) in groups of UN*KPL and folds them into the
 // running (max, sum, output) of this lane group.  kb / vb already point at this lane's 8 head elements.
 template <int D, int G, int UN = kAttnDecUnroll, bool PIPELINED = true>
-__device__ __forceinline__ void attn_stream_keys(const __half* kb, const __half* vb, const float (&q)[G][8], int t_first,
+__device__ __forceinline__ void attn_stream_keys(const half_t* kb, const half_t* vb, const float (&q)[G][8], int t_first,
                                                  int t_end, int t_step, int sub, float (&m)[G], float (&l)[G],
                                                  float (&o)[G][8]) {
   constexpr int LPK = D / 8;
@@ -169,7 +169,7 @@ __device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMe
       O += sm.o[w][g][i] * al;
     }
     if (n_seg == 1) {
-      a.out[(bh0 + g) * D + i] = __float2half_rn(O / L);
+      a.out[(bh0 + g) * D + i] = f_to_h(O / L);
     } else {
       const size_t p = (bh0 + g) * kAttnMaxSplits + seg;
       a.part_o[p * D + i] = O;
@@ -292,8 +292,8 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
 #pragma unroll
       for (int i = 0; i < 8; ++i) q[g][i] *= a.scale_log2;
     }
-    const __half* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
-    const __half* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+    const half_t* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
+    const half_t* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D + dl * 8;
 
     float m[G], l[G], o[G][8];
 #pragma unroll

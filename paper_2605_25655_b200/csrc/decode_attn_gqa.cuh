@@ -91,15 +91,15 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_gqa_kernel(con
     // 16 ks + 2t, +1 and 16 ks + 8 + 2t, +1
     uint32_t qa[KS][2];
     {
-      const __half* qrow = a.q + (static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D;
+      const half_t* qrow = a.q + (static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
         qa[ks][0] = g < G ? __ldg(reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * t)) : 0u;
         qa[ks][1] = g < G ? __ldg(reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * t)) : 0u;
       }
     }
-    const __half* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D;
-    const __half* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D;
+    const half_t* kb = a.k_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D;
+    const half_t* vb = a.v_cache + (static_cast<size_t>(b) * a.n_kv_heads + hk) * a.t_max * D;
 
     // blocks of 16 keys: this warp takes blocks warp, warp + 4, ... of the segment
     const int n_blocks = (t1 - t0 + kGqaChunk - 1) / kGqaChunk;          // <= 0 for an empty segment
@@ -166,8 +166,8 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_gqa_kernel(con
       float psum = 0.f;
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
-        const __half2 hp = __floats2half2_rn(exp2f(x[nt * 2] - m_new), exp2f(x[nt * 2 + 1] - m_new));
-        const float2 back = __half22float2(hp);       // the sum is taken over the rounded weights
+        const half2_t hp = f2_to_h2(exp2f(x[nt * 2] - m_new), exp2f(x[nt * 2 + 1] - m_new));
+        const float2 back = h2_to_f2(hp);       // the sum is taken over the rounded weights
         psum += back.x + back.y;
         pa[nt] = *reinterpret_cast<const uint32_t*>(&hp);
       }

@@ -18,13 +18,13 @@ constexpr int kGemvWarps = 8;
 constexpr int kGemvUnroll = 4;
 
 struct GemvArgs {
-  const __half* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
+  const half_t* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
   int n[3];            // rows of each matrix (0 for unused); every count is even
   int k;               // contraction length, multiple of 8
   int rows;            // tokens
-  const __half* x;     // [rows][ldx]
+  const half_t* x;     // [rows][ldx]
   int ldx;
-  const __half* gamma;  // RMSNorm gain [k] when NORM
+  const half_t* gamma;  // RMSNorm gain [k] when NORM
   float eps;
   int kslices;          // 1, 2, 4 or 8 warps share one feature pair
   EpiArgs e;
@@ -43,8 +43,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv_stream_kernel(const Gemv
   const int n_pairs = (EPI == EPI_SWIGLU) ? a.n[0] : (a.n[0] + a.n[1] + a.n[2]) / 2;
   const bool active = pair < n_pairs;
 
-  const __half* wa = nullptr;
-  const __half* wb = nullptr;
+  const half_t* wa = nullptr;
+  const half_t* wb = nullptr;
   if (active) {
     if (EPI == EPI_SWIGLU) {
       wa = a.w[0] + static_cast<size_t>(pair) * a.k;
@@ -149,13 +149,13 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv_stream_kernel(const Gemv
 
   const EpiArgs& e = a.e;
   if (EPI == EPI_SWIGLU) {
-    reinterpret_cast<__half*>(e.out)[static_cast<size_t>(r) * e.ld_out + pair] = __float2half_rn(silu_f(s0) * s1);
+    reinterpret_cast<half_t*>(e.out)[static_cast<size_t>(r) * e.ld_out + pair] = f_to_h(silu_f(s0) * s1);
   } else if (EPI == EPI_RESID) {
     const size_t o = static_cast<size_t>(r) * e.ld_out + 2 * pair;
-    const float2 x = __half22float2(*reinterpret_cast<const __half2*>(e.resid + o));
-    *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + o) = pack2(x.x + s0, x.y + s1);
+    const float2 x = h2_to_f2(*reinterpret_cast<const half2_t*>(e.resid + o));
+    *reinterpret_cast<uint32_t*>(reinterpret_cast<half_t*>(e.out) + o) = pack2(x.x + s0, x.y + s1);
   } else if (EPI == EPI_PLAIN_F16) {
-    *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + static_cast<size_t>(r) * e.ld_out + 2 * pair) =
+    *reinterpret_cast<uint32_t*>(reinterpret_cast<half_t*>(e.out) + static_cast<size_t>(r) * e.ld_out + 2 * pair) =
         pack2(s0, s1);
   } else if (EPI == EPI_PLAIN_F32) {
     *reinterpret_cast<float2*>(reinterpret_cast<float*>(e.out) + static_cast<size_t>(r) * e.ld_out + 2 * pair) =
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv_stream_kernel(const Gemv
       s0 = y0;
       s1 = y1;
     }
-    __half* dst = (kind == 0) ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
+    half_t* dst = (kind == 0) ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
     *reinterpret_cast<uint32_t*>(dst + o) = pack2(s0, s1);
   }
 }

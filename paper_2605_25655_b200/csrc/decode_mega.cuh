@@ -35,9 +35,9 @@ constexpr int kMegaABytes = kTcBM * 128;
 
 struct alignas(64) MegaLayer {
   CUtensorMap wq, wk, wv, wo, wg, wu, wd;
-  const __half* attn_norm;  // gain of the first RMSNorm (used by the prep unit of the first layer)
-  const __half* ffn_norm;   // gain folded into the O-projection epilogue
-  const __half* next_norm;  // gain folded into the down-projection epilogue (next layer's, or nullptr)
+  const half_t* attn_norm;  // gain of the first RMSNorm (used by the prep unit of the first layer)
+  const half_t* ffn_norm;   // gain folded into the O-projection epilogue
+  const half_t* next_norm;  // gain folded into the down-projection epilogue (next layer's, or nullptr)
 };
 struct alignas(64) MegaCommon {
   CUtensorMap x_qkv, x_o, x_gu, x_down;  // token-side operands: xg, attn, x1g, act  (boxes of BN rows)
@@ -49,10 +49,10 @@ struct MegaArgs {
   int n_layers, batch, pos;
   int hidden, ffn, n_q_heads, n_kv_heads, t_max;
   float eps;
-  const __half* x_in;  // [batch][hidden] input of the first layer
-  __half* x_out;       // output of the last layer
-  __half *xa, *xb;     // residual stream between layers (ping-pong)
-  __half *xg, *x1, *x1g, *qbuf, *attn, *act;
+  const half_t* x_in;  // [batch][hidden] input of the first layer
+  half_t* x_out;       // output of the last layer
+  half_t *xa, *xb;     // residual stream between layers (ping-pong)
+  half_t *xg, *x1, *x1g, *qbuf, *attn, *act;
   float *sumsq0, *sumsq1;  // [feature tiles][64]: sums of squares feeding the first / second RMSNorm
   uint8_t* kv_base;        // K of layer l: kv_base + ((slot * n_layers + l) * 2) * kv_layer_bytes, V one further
   size_t kv_layer_bytes;
@@ -103,8 +103,8 @@ template <int BN, int D>
 __device__ __forceinline__ void mega_gemm_desc(const MegaArgs& a, int layer, int phase, MegaGemm& m) {
   const MegaLayer& L = a.layers[layer];
   const int qd = a.n_q_heads * D, kvd = a.n_kv_heads * D;
-  const __half* in_l = layer == 0 ? a.x_in : ((layer & 1) ? a.xb : a.xa);
-  __half* out_l = layer == a.n_layers - 1 ? a.x_out : ((layer & 1) ? a.xa : a.xb);
+  const half_t* in_l = layer == 0 ? a.x_in : ((layer & 1) ? a.xb : a.xa);
+  half_t* out_l = layer == a.n_layers - 1 ? a.x_out : ((layer & 1) ? a.xa : a.xb);
   TcGemmArgs& g = m.g;
   g = TcGemmArgs{};
   g.rows = a.batch;
@@ -121,8 +121,8 @@ __device__ __forceinline__ void mega_gemm_desc(const MegaArgs& a, int layer, int
     g.k = a.hidden;
     uint8_t* kc = a.kv_base + (static_cast<size_t>(a.slot) * a.n_layers + layer) * 2 * a.kv_layer_bytes;
     e.q_out = a.qbuf;
-    e.k_cache = reinterpret_cast<__half*>(kc);
-    e.v_cache = reinterpret_cast<__half*>(kc + a.kv_layer_bytes);
+    e.k_cache = reinterpret_cast<half_t*>(kc);
+    e.v_cache = reinterpret_cast<half_t*>(kc + a.kv_layer_bytes);
     e.rope_cos = a.rope_cos; e.rope_sin = a.rope_sin;
     e.n_q = qd; e.n_kv = kvd; e.head_dim = D; e.n_q_heads = a.n_q_heads; e.n_kv_heads = a.n_kv_heads;
     e.seq_len = 1; e.pos0 = a.pos; e.t_max = a.t_max;
@@ -334,12 +334,12 @@ __device__ __forceinline__ void mega_rstd(const MegaArgs& a, const MegaShared& s
 
 // ------------------------------------------------------------------ prep unit (first layer's RMSNorm input)
 __device__ __forceinline__ void mega_prep(const MegaArgs& a, float* red, int wtid) {
-  const __half* gain = a.layers[0].attn_norm;
+  const half_t* gain = a.layers[0].attn_norm;
   const int chunks = a.hidden >> 3;
   const int parts = (a.hidden + kTcBM - 1) / kTcBM;
   for (int b = blockIdx.x; b < a.batch; b += gridDim.x) {
-    const __half* xr = a.x_in + static_cast<size_t>(b) * a.hidden;
-    __half* gr = a.xg + static_cast<size_t>(b) * a.hidden;
+    const half_t* xr = a.x_in + static_cast<size_t>(b) * a.hidden;
+    half_t* gr = a.xg + static_cast<size_t>(b) * a.hidden;
     float ss = 0.f;
     for (int c = wtid; c < chunks; c += kMegaWorkers) {
       float f[8], g[8];
@@ -385,8 +385,8 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
   const long long per = (total + gridDim.x - 1) / gridDim.x;
   long long cur = per * blockIdx.x;
   const long long end = (cur + per < total) ? cur + per : total;
-  const __half* kcache = reinterpret_cast<const __half*>(kc_bytes);
-  const __half* vcache = reinterpret_cast<const __half*>(kc_bytes + a.kv_layer_bytes);
+  const half_t* kcache = reinterpret_cast<const half_t*>(kc_bytes);
+  const half_t* vcache = reinterpret_cast<const half_t*>(kc_bytes + a.kv_layer_bytes);
   const float scale_log2 = 1.4426950408889634f * rsqrtf(static_cast<float>(D));
   while (cur < end) {
     const int item = static_cast<int>(cur / T);
@@ -446,7 +446,7 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
         O += sm.o[w][g][i] * al;
       }
       if (n_seg == 1) {
-        a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = __float2half_rn(O / L);
+        a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = f_to_h(O / L);
       } else {
         slot[g * (D + 2) + i] = O;
         if (i == 0) {
@@ -494,7 +494,7 @@ __device__ __forceinline__ void mega_attention(const MegaArgs& a, const MegaShar
               L += __ldcg(p + D + 1) * al;
               O += __ldcg(p + i) * al;
             }
-            a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = __float2half_rn(O / L);
+            a.attn[(static_cast<size_t>(b) * a.n_q_heads + h0 + g) * D + i] = f_to_h(O / L);
           }
           if (wtid == 0) a.attn_counters[item] = 0;
         } else {

@@ -34,12 +34,12 @@ constexpr int kSkTokMax = 16;
 // ring depth per warp is the template parameter ST; one stage = 16 rows x 64 elements = 2 KB
 
 struct SkinnyArgs {
-  const __half* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
+  const half_t* w[3];  // QKV: wq, wk, wv.  SWIGLU: gate, up.  Others: one matrix.
   int n[3];            // rows of each matrix (0 for unused); every count is even
   int cta0[4];         // CTAs cta0[m] .. cta0[m+1]-1 share matrix m (SWIGLU: everything is "matrix" 0)
   int k;               // contraction length, multiple of 64
   int rows;            // tokens, <= 8 * NT
-  const __half* x;     // [rows][ldx]
+  const half_t* x;     // [rows][ldx]
   int ldx;
   // folded RMSNorm of the token operand: sums of squares per (part, token), [sumsq_parts][16], as the
   // RESID epilogue of this kernel leaves them (one part per CTA)
@@ -50,7 +50,7 @@ struct SkinnyArgs {
   // NORM kernels instead take the raw rows in x and the gain here: RMSNorm as a prologue.  Every CTA reads
   // all of x anyway, so the sums of squares come from the token fragments it already holds, the gain is
   // multiplied in (FP16, the rounding of a stored normalised operand) and 1/rms scales the finished sums.
-  const __half* gamma;
+  const half_t* gamma;
   int tiles_max;       // row tiles of the largest CTA share (<= TM)
   EpiArgs e;           // RESID with outg: e.sumsq receives [gridDim.x][16]
   unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
@@ -60,7 +60,7 @@ struct SkinnyArgs {
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                           uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      "mma.sync.aligned.m16n8k16.row.col.f32." THINFER_MMA_SYNC_TYPES ".f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -77,9 +77,9 @@ __device__ __forceinline__ void cp_async_wait_group() {
 // element-wise FP16 product of two groups of 8 halves
 __device__ __forceinline__ uint4 hmul2x4(const uint4& a, const uint4& b) {
   uint4 r;
-  const __half2* pa = reinterpret_cast<const __half2*>(&a);
-  const __half2* pb = reinterpret_cast<const __half2*>(&b);
-  __half2* pr = reinterpret_cast<__half2*>(&r);
+  const half2_t* pa = reinterpret_cast<const half2_t*>(&a);
+  const half2_t* pb = reinterpret_cast<const half2_t*>(&b);
+  half2_t* pr = reinterpret_cast<half2_t*>(&r);
 #pragma unroll
   for (int i = 0; i < 4; ++i) pr[i] = __hmul2(pa[i], pb[i]);
   return r;
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   const uint32_t coop_dst = smem_u32(ring) + crow * 128 + ((cchunk ^ ((crow & 1) << 2)) << 4);
   const size_t coop_off = static_cast<size_t>(warp) * 64 + cchunk * 8;
   const int lim_hi = r_hi - r_lo - crow;  // tile row TR * tile + 4 j (+ crow) is in the share iff TR * tile + 4 j < lim_hi
-  const __half* tb[TM];  // plain: row crow of the tile, at this lane's chunk of block `warp`
+  const half_t* tb[TM];  // plain: row crow of the tile, at this lane's chunk of block `warp`
   if (EPI != EPI_SWIGLU) {
 #pragma unroll
     for (int tile = 0; tile < TM; ++tile)
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
       cp_async_16(dst + 1024, a.w[1] + o0, s0);
       cp_async_16(dst + 1536, a.w[1] + o1, s1);
     } else {
-      const __half* src = tb[tile] + off;
+      const half_t* src = tb[tile] + off;
       const size_t k4 = static_cast<size_t>(4) * a.k;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   // token fragments: XB buffers, requested XB - 1 blocks ahead (the fewer tiles a block has, the further)
   constexpr int XB = TM == 1 ? 4 : (TM <= 3 ? 3 : 2);
   const uint4 zero = make_uint4(0, 0, 0, 0);
-  const __half* xrow[NT];
+  const half_t* xrow[NT];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt)
     xrow[nt] = (nt * 8 + g < a.rows) ? a.x + static_cast<size_t>(nt * 8 + g) * a.ldx + static_cast<size_t>(warp) * 64 + t * 8
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
   float ssx[NT];  // NORM: this lane's share of the sum of squares of token nt * 8 + g
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) ssx[nt] = 0.f;
-  const __half* grow = NORM ? a.gamma + static_cast<size_t>(warp) * 64 + t * 8 : nullptr;
+  const half_t* grow = NORM ? a.gamma + static_cast<size_t>(warp) * 64 + t * 8 : nullptr;
 
   int stage = 0;
   const int frag0 = g * 8 + (t ^ ((g & 1) << 2));  // row g, chunk t (chunk 4 + t: position ^ 4; row g + 8: + 64)
@@ -370,9 +370,9 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
     if (EPI == EPI_SWIGLU) {
       const int f = row0 + g;
       if (f < r_hi) {
-        __half* o = reinterpret_cast<__half*>(e.out);
-        if (ta < a.rows) o[static_cast<size_t>(ta) * e.ld_out + f] = __float2half_rn(silu_f(c[0]) * c[2]);
-        if (tb < a.rows) o[static_cast<size_t>(tb) * e.ld_out + f] = __float2half_rn(silu_f(c[1]) * c[3]);
+        half_t* o = reinterpret_cast<half_t*>(e.out);
+        if (ta < a.rows) o[static_cast<size_t>(ta) * e.ld_out + f] = f_to_h(silu_f(c[0]) * c[2]);
+        if (tb < a.rows) o[static_cast<size_t>(tb) * e.ld_out + f] = f_to_h(silu_f(c[1]) * c[3]);
       }
     } else if (EPI == EPI_QKV_ROPE) {
       // rows g and g + 8 have the parity of g; the other half of a rotation pair sits in lane ^ 4
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
           }
           const float y_odd = __shfl_xor_sync(0xffffffffu, y, 4);
           if (ok && !(g & 1)) {
-            __half* dst = (kind == 0) ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
+            half_t* dst = (kind == 0) ? e.q_out : (kind == 1 ? e.k_cache : e.v_cache);
             *reinterpret_cast<uint32_t*>(dst + off) = pack2(y, y_odd);
           }
         }
@@ -420,14 +420,14 @@ __global__ void __launch_bounds__(kSkWarps * 32, 2) skinny_mma_kernel(const Skin
           if (EPI == EPI_PLAIN_F32) {
             *reinterpret_cast<float2*>(reinterpret_cast<float*>(e.out) + off) = make_float2(v0, v1);
           } else if (EPI == EPI_PLAIN_F16) {
-            *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + off) = pack2(v0, v1);
+            *reinterpret_cast<uint32_t*>(reinterpret_cast<half_t*>(e.out) + off) = pack2(v0, v1);
           } else {  // EPI_RESID
-            const float2 x = __half22float2(*reinterpret_cast<const __half2*>(e.resid + off));
+            const float2 x = h2_to_f2(*reinterpret_cast<const half2_t*>(e.resid + off));
             const uint32_t yh = pack2(x.x + v0, x.y + v1);
-            *reinterpret_cast<uint32_t*>(reinterpret_cast<__half*>(e.out) + off) = yh;
+            *reinterpret_cast<uint32_t*>(reinterpret_cast<half_t*>(e.out) + off) = yh;
             if (e.outg != nullptr) {  // folded RMSNorm of the next sub-layer (gain here, 1/rms there)
-              const float2 y = __half22float2(*reinterpret_cast<const __half2*>(&yh));
-              const float2 gn = __half22float2(*reinterpret_cast<const __half2*>(e.gain_next + r_cat + row));
+              const float2 y = h2_to_f2(*reinterpret_cast<const half2_t*>(&yh));
+              const float2 gn = h2_to_f2(*reinterpret_cast<const half2_t*>(e.gain_next + r_cat + row));
               *reinterpret_cast<uint32_t*>(e.outg + off) = pack2(y.x * gn.x, y.y * gn.y);
               sq[j] = fmaf(y.x, y.x, fmaf(y.y, y.y, sq[j]));
             }

@@ -18,12 +18,12 @@ enum Epi : int {
 
 struct EpiArgs {
   void* out;            // PLAIN / RESID / SWIGLU destination, row-major [rows][ld_out]
-  const __half* resid;  // RESID: residual stream, same layout as out
+  const half_t* resid;  // RESID: residual stream, same layout as out
   int ld_out;
   // QKV + RoPE + cache append
-  __half* q_out;        // [batch][n_q_heads][seq_len][head_dim]
-  __half* k_cache;      // [max_batch][n_kv_heads][t_max][head_dim], K after rotation
-  __half* v_cache;
+  half_t* q_out;        // [batch][n_q_heads][seq_len][head_dim]
+  half_t* k_cache;      // [max_batch][n_kv_heads][t_max][head_dim], K after rotation
+  half_t* v_cache;
   const float* rope_cos;  // [max_seq][head_dim/2]
   const float* rope_sin;
   int n_q;              // n_q_heads * head_dim   (rows of wq)
@@ -37,8 +37,8 @@ struct EpiArgs {
   // y = resid + acc the kernel writes outg = y * gain_next (the operand the next projection reads)
   // and, per 128-feature tile and token, the sum of y^2 (sumsq[feature_tile][64 tokens]); the next
   // projection multiplies its result by rsqrt(sum over tiles / n + eps) per token.
-  __half* outg;
-  const __half* gain_next;
+  half_t* outg;
+  const half_t* gain_next;
   float* sumsq;
 };
 

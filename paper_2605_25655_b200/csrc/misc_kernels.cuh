@@ -8,15 +8,15 @@ namespace thinfer {
 
 // y[r][:] = x[r][:] * gain / sqrt(mean(x[r]^2) + eps); FP32 inside (Section 3.2.4).
 // One warp per row, 128-bit accesses; n is a multiple of 8.
-__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __half* __restrict__ x, const __half* __restrict__ gain,
-                                                           __half* __restrict__ y, int rows, int n, float eps) {
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const half_t* __restrict__ x, const half_t* __restrict__ gain,
+                                                           half_t* __restrict__ y, int rows, int n, float eps) {
   pdl_launch_dependents();
   pdl_wait();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
-  const __half* xr = x + static_cast<size_t>(row) * n;
-  __half* yr = y + static_cast<size_t>(row) * n;
+  const half_t* xr = x + static_cast<size_t>(row) * n;
+  half_t* yr = y + static_cast<size_t>(row) * n;
   const int chunks = n >> 3;
   float ss = 0.f;
   for (int c = lane; c < chunks; c += 32) {
@@ -43,14 +43,14 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __half* __restr
 // The same operator for few rows (decode): one CTA per row, the row is read once into registers.
 // n <= 8 * 256 * kRmsSmallChunks.
 constexpr int kRmsSmallChunks = 8;
-__global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const __half* __restrict__ x,
-                                                               const __half* __restrict__ gain, __half* __restrict__ y,
+__global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const half_t* __restrict__ x,
+                                                               const half_t* __restrict__ gain, half_t* __restrict__ y,
                                                                int n, float eps) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ float red[8];
-  const __half* xr = x + static_cast<size_t>(blockIdx.x) * n;
-  __half* yr = y + static_cast<size_t>(blockIdx.x) * n;
+  const half_t* xr = x + static_cast<size_t>(blockIdx.x) * n;
+  half_t* yr = y + static_cast<size_t>(blockIdx.x) * n;
   const int chunks = n >> 3;
   uint4 xv[kRmsSmallChunks], gv[kRmsSmallChunks];
 #pragma unroll
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(256) rmsnorm_few_rows_kernel(const __half* __r
 
 // dst[r][:] = table[ids[r]][:]  (embedding).  One warp per row.
 __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __restrict__ ids,
-                                                           const __half* __restrict__ table, __half* __restrict__ dst,
+                                                           const half_t* __restrict__ table, half_t* __restrict__ dst,
                                                            int rows, int n, int vocab) {
   pdl_launch_dependents();
   pdl_wait();
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* __rest
 }
 
 // dst[b][:] = src[b][seq_len-1][:]  (the last prompt position feeds the LM head).
-__global__ void __launch_bounds__(256) gather_last_rows_kernel(const __half* __restrict__ src, __half* __restrict__ dst,
+__global__ void __launch_bounds__(256) gather_last_rows_kernel(const half_t* __restrict__ src, half_t* __restrict__ dst,
                                                                int batch, int seq_len, int n,
                                                                const int* __restrict__ lens) {
   pdl_launch_dependents();

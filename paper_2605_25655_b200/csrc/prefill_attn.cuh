@@ -32,7 +32,7 @@ constexpr int kAttnBK = 64;    // keys per tile
 constexpr int kAttnThreads = 288;  // two softmax groups of 128 + the issuing warp
 
 struct AttnPreArgs {
-  __half* out;  // [batch][seq_len][n_q_heads * D]
+  half_t* out;  // [batch][seq_len][n_q_heads * D]
   int n_q_heads, n_kv_heads, seq_len;
   float scale_log2;  // log2(e) / sqrt(D)
   int* status;
@@ -259,8 +259,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             if (kbase + half * 32 + c > row) p0 = 0.f;
             if (kbase + half * 32 + c + 1 > row) p1 = 0.f;
           }
-          const __half2 hp = __floats2half2_rn(p0, p1);
-          const float2 back = __half22float2(hp);
+          const half2_t hp = f2_to_h2(p0, p1);
+          const float2 back = h2_to_f2(hp);
           sum4[(c >> 1) & 3] += back.x + back.y;
           pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&hp);
         }
@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         tmem_ld32(lane_addr + TM_O[t] + c0, r);
         tmem_ld_wait();
         if (qrow < a.seq_len) {
-          __half* dst = a.out + (static_cast<size_t>(b) * a.seq_len + qrow) * (a.n_q_heads * D) + h * D + c0;
+          half_t* dst = a.out + (static_cast<size_t>(b) * a.seq_len + qrow) * (a.n_q_heads * D) + h * D + c0;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             uint4 o;

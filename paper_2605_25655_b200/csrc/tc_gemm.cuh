@@ -167,7 +167,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
                                               const float (&v)[CW], const float (&v2)[CW], int tok_base) {
   const EpiArgs& e = a.e;
   constexpr bool F32 = tc_epi_fp32_stage(EPI);
-  __half* st16 = reinterpret_cast<__half*>(stage);
+  half_t* st16 = reinterpret_cast<half_t*>(stage);
   float* st32 = reinterpret_cast<float*>(stage);
 
   // RESID: the residual pieces this thread adds in phase B are requested now, so that their latency runs
@@ -183,7 +183,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
       const int r = tok_base + c, n0 = t.feat0 + piece * 8;
       rx[it] = make_uint4(0, 0, 0, 0);
       if (idx < CW * 16 && r < a.rows && a.n_feat[t.mat] - n0 >= 8) {
-        const __half* src = e.resid + static_cast<size_t>(r) * e.ld_out + n0;
+        const half_t* src = e.resid + static_cast<size_t>(r) * e.ld_out + n0;
         rx[it] = a.static_finisher ? __ldcg(reinterpret_cast<const uint4*>(src))  // written earlier in the same kernel
                                    : *reinterpret_cast<const uint4*>(src);        // written by an earlier kernel
       }
@@ -195,8 +195,8 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
       if (F32) st32[c * kTcBM + row] = v[c];
-      else if (EPI == EPI_SWIGLU) st16[c * kTcBM + row] = __float2half_rn(silu_f(v[c]) * v2[c]);
-      else st16[c * kTcBM + row] = __float2half_rn(v[c]);
+      else if (EPI == EPI_SWIGLU) st16[c * kTcBM + row] = f_to_h(silu_f(v[c]) * v2[c]);
+      else st16[c * kTcBM + row] = f_to_h(v[c]);
     }
   }
   epi_bar();
@@ -213,7 +213,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
       if (r < a.rows && n0 < n_feat) {
         const float* g = st32 + c * kTcBM + piece * 8;
         const float* u = g + 64;
-        __half* dst = reinterpret_cast<__half*>(e.out) + static_cast<size_t>(r) * e.ld_out + n0;
+        half_t* dst = reinterpret_cast<half_t*>(e.out) + static_cast<size_t>(r) * e.ld_out + n0;
         if (n_feat - n0 >= 8 && (e.ld_out & 7) == 0) {
           uint4 o;
           o.x = pack2(silu_f(g[0]) * u[0], silu_f(g[1]) * u[1]);
@@ -222,7 +222,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
           o.w = pack2(silu_f(g[6]) * u[6], silu_f(g[7]) * u[7]);
           *reinterpret_cast<uint4*>(dst) = o;
         } else {
-          for (int j = 0; j < min(8, n_feat - n0); ++j) dst[j] = __float2half_rn(silu_f(g[j]) * u[j]);
+          for (int j = 0; j < min(8, n_feat - n0); ++j) dst[j] = f_to_h(silu_f(g[j]) * u[j]);
         }
       }
     }
@@ -243,7 +243,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
     if (EPI == EPI_QKV_ROPE) {
       const int b = r / e.seq_len, s = r - b * e.seq_len;
       const int h = n0 / e.head_dim, i = n0 - h * e.head_dim;
-      __half* dst;
+      half_t* dst;
       if (t.mat == 0) dst = e.q_out + ((static_cast<size_t>(b) * e.n_q_heads + h) * e.seq_len + s) * e.head_dim + i;
       else dst = (t.mat == 1 ? e.k_cache : e.v_cache) +
                  ((static_cast<size_t>(b) * e.n_kv_heads + h) * e.t_max + e.pos0 + s +
@@ -286,7 +286,7 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
           for (int j = 0; j < valid; ++j) dst[j] = src[j];
         }
       } else if (EPI == EPI_RESID) {
-        __half* dst = reinterpret_cast<__half*>(e.out) + off;
+        half_t* dst = reinterpret_cast<half_t*>(e.out) + off;
         const float* src = st32 + c * kTcBM + piece * 8;
         if (vec) {
           float x[8];
@@ -312,18 +312,18 @@ __device__ __forceinline__ void tc_emit_chunk(const TcGemmArgs& a, const TcTile&
           }
         } else {
           for (int j = 0; j < valid; ++j) {
-            const __half yh = __float2half_rn(__half2float(__ldcg(e.resid + off + j)) + src[j]);
+            const half_t yh = f_to_h(h_to_f(__ldcg(e.resid + off + j)) + src[j]);
             dst[j] = yh;
             if (e.outg != nullptr) {
-              const float y = __half2float(yh);
-              e.outg[off + j] = __float2half_rn(y * __half2float(e.gain_next[n0 + j]));
+              const float y = h_to_f(yh);
+              e.outg[off + j] = f_to_h(y * h_to_f(e.gain_next[n0 + j]));
               sq = fmaf(y, y, sq);
             }
           }
         }
       } else {  // PLAIN_F16, SWIGLU
-        __half* dst = reinterpret_cast<__half*>(e.out) + off;
-        const __half* src = st16 + c * kTcBM + piece * 8;
+        half_t* dst = reinterpret_cast<half_t*>(e.out) + off;
+        const half_t* src = st16 + c * kTcBM + piece * 8;
         if (vec) {
           *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
         } else {

@@ -46,7 +46,7 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// FP16 tensor [d2][d1][d0] (d0 contiguous), box [1][box1][64], 128-byte swizzle, zero fill outside.
+// 16-bit tensor [d2][d1][d0] (d0 contiguous), box [1][box1][64], 128-byte swizzle, zero fill outside.
 // stride1 / stride2 in elements.
 bool make_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1,
               uint64_t stride2, uint32_t box1, int rank) {
@@ -56,7 +56,7 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64
   cuuint64_t strides[2] = {stride1 * 2, stride2 * 2};
   cuuint32_t box[3] = {64, box1, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base), dims,
+  CUresult r = fn(m, kStorageType == 1 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base), dims,
                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -95,7 +95,7 @@ struct ProfEvent {
 struct thinfer_ctx {
   thinfer_config cfg{};
   std::vector<thinfer_layer_weights> layers;
-  const __half *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+  const half_t *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
   std::vector<LayerMaps> maps;
   CUtensorMap map_head{};
   uint8_t* kv = nullptr;
@@ -103,13 +103,13 @@ struct thinfer_ctx {
   std::vector<Slot> slots;
   // scratch carve-up
   float *rope_cos = nullptr, *rope_sin = nullptr;
-  __half *h = nullptr, *qbuf = nullptr, *attn = nullptr, *x1 = nullptr, *act = nullptr, *xa = nullptr, *xb = nullptr;
-  __half* last = nullptr;
+  half_t *h = nullptr, *qbuf = nullptr, *attn = nullptr, *x1 = nullptr, *act = nullptr, *xa = nullptr, *xb = nullptr;
+  half_t* last = nullptr;
   float* logits = nullptr;
   int32_t* ids_out = nullptr;
   // the decode path has its own (small) activation buffers, so that a prefill of one slot and decode steps of
   // another may run on different streams at the same time (the two stages of the pipeline, Section 3.4.2)
-  __half *d_h = nullptr, *d_qbuf = nullptr, *d_attn = nullptr, *d_x1 = nullptr, *d_act = nullptr, *d_xa = nullptr,
+  half_t *d_h = nullptr, *d_qbuf = nullptr, *d_attn = nullptr, *d_x1 = nullptr, *d_act = nullptr, *d_xa = nullptr,
          *d_xb = nullptr;
   float* d_logits = nullptr;
   uint8_t *d_stage_in = nullptr, *d_stage_out = nullptr;
@@ -121,7 +121,7 @@ struct thinfer_ctx {
   // inspection: copies of the hidden state behind chosen layers (thinfer_capture_hidden)
   std::vector<std::pair<int, void*>> captures;
   // unified decode kernel
-  __half *xg = nullptr, *x1g = nullptr;
+  half_t *xg = nullptr, *x1g = nullptr;
   float *sumsq0 = nullptr, *sumsq1 = nullptr, *attn_partial = nullptr;
   int sumsq0_parts = 0, sumsq1_parts = 0;  // parts the last skinny down / O projection left in sumsq0 / sumsq1
   bool skinny_ok = true;    // hidden, ffn and the head widths suit the skinny decode projections
@@ -408,7 +408,7 @@ void launch_tc_bn(Launcher& L, int kid, int bn, const CUtensorMap& w0, const CUt
 // x: activations [rows][k]; the token-side tensor map is encoded per call (host only, no device work)
 template <int EPI>
 void tc_linear(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& w2,
-               const __half* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e, bool stream_k = false,
+               const half_t* x, int rows, int k, const int (&n_feat)[3], const EpiArgs& e, bool stream_k = false,
                const float* sumsq_in = nullptr, float norm_eps = 0.f) {
   if (L.rc != THINFER_OK) return;
   const int bn = pick_bn(rows, EPI);
@@ -452,8 +452,8 @@ int pick_kslices(int n_pairs, int k, int sm_count) {
 }
 
 template <int EPI, bool NORM>
-void gemv(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
-          const __half* x, int ldx, int rows, const __half* gamma, float eps, const EpiArgs& e) {
+void gemv(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_t* w2, const int (&n)[3], int k,
+          const half_t* x, int ldx, int rows, const half_t* gamma, float eps, const EpiArgs& e) {
   if (L.rc != THINFER_OK) return;
   GemvArgs a{};
   a.w[0] = w0;
@@ -548,9 +548,9 @@ void launch_skinny(Launcher& L, int kid, int grid, const SkinnyArgs& a) {
 
 // Returns the grid size: a RESID producer leaves one sum-of-squares part per CTA.
 template <int EPI, bool NORM = false>
-int skinny(Launcher& L, int kid, const __half* w0, const __half* w1, const __half* w2, const int (&n)[3], int k,
-           const __half* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, float eps, const EpiArgs& e,
-           const __half* gamma = nullptr) {
+int skinny(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_t* w2, const int (&n)[3], int k,
+           const half_t* x, int ldx, int rows, const float* sumsq_in, int sumsq_parts, float eps, const EpiArgs& e,
+           const half_t* gamma = nullptr) {
   if (L.rc != THINFER_OK) return 0;
   SkinnyArgs a{};
   a.w[0] = w0;
@@ -662,7 +662,7 @@ void attn_decode_d(Launcher& L, thinfer_ctx* c, const AttnDecArgs& a, int batch,
 
 // t_len: keys the longest request attends (the unit count of the schedule); with `len_arr` (ragged slots) request b
 // attends len_arr[b] + len_add keys
-void attn_decode(Launcher& L, thinfer_ctx* c, const __half* q, const __half* kc, const __half* vc, __half* out,
+void attn_decode(Launcher& L, thinfer_ctx* c, const half_t* q, const half_t* kc, const half_t* vc, half_t* out,
                  int batch, int t_len, const int* len_arr = nullptr, int len_add = 0) {
   if (L.rc != THINFER_OK) return;
   const thinfer_config& cf = c->cfg;
@@ -699,7 +699,7 @@ void attn_prefill_d(Launcher& L, const CUtensorMap& mq, const CUtensorMap& mk, c
   L.go(THINFER_K_ATTN, attn_prefill_kernel<D>, dim3((n_qt + 1) / 2, a.n_q_heads, batch), dim3(kAttnThreads), smem, mq, mk, mv, a);
 }
 
-void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v, __half* out, int batch, int n_q_heads,
+void attn_prefill(Launcher& L, const half_t* q, const half_t* k, const half_t* v, half_t* out, int batch, int n_q_heads,
                   int n_kv_heads, int seq, int kv_stride, int head_dim, int* status) {
   if (L.rc != THINFER_OK) return;
   CUtensorMap mq, mk, mv;
@@ -725,7 +725,7 @@ void attn_prefill(Launcher& L, const __half* q, const __half* k, const __half* v
   else attn_prefill_d<64>(L, mq, mk, mv, a, batch);
 }
 
-void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int rows, int n, float eps) {
+void rmsnorm_rows(Launcher& L, const half_t* x, const half_t* g, half_t* y, int rows, int n, float eps) {
   if (rows <= 256 && n <= 8 * 256 * kRmsSmallChunks) {
     L.go(THINFER_K_RMSNORM, rmsnorm_few_rows_kernel, dim3(rows), dim3(256), 0, x, g, y, n, eps);
     return;
@@ -736,7 +736,7 @@ void rmsnorm_rows(Launcher& L, const __half* x, const __half* g, __half* y, int 
 // ----------------------------------------------------------------------------
 // the layer sequences
 // ----------------------------------------------------------------------------
-EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_len, int pos0,
+EpiArgs qkv_epi(thinfer_ctx* c, half_t* qbuf, half_t* kc, half_t* vc, int seq_len, int pos0,
                 const int* pos_arr = nullptr) {
   const thinfer_config& cf = c->cfg;
   EpiArgs e{};
@@ -757,22 +757,22 @@ EpiArgs qkv_epi(thinfer_ctx* c, __half* qbuf, __half* kc, __half* vc, int seq_le
   return e;
 }
 
-__half* kv_ptr(thinfer_ctx* c, int slot, int layer, int which) {
+half_t* kv_ptr(thinfer_ctx* c, int slot, int layer, int which) {
   const size_t idx = (static_cast<size_t>(slot) * c->cfg.n_layers + layer) * 2 + which;
-  return reinterpret_cast<__half*>(c->kv + idx * c->kv_layer_bytes);
+  return reinterpret_cast<half_t*>(c->kv + idx * c->kv_layer_bytes);
 }
 
-void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half* x_in, __half* x_out, int batch,
+void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const half_t* x_in, half_t* x_out, int batch,
                    int seq) {
   const thinfer_config& cf = c->cfg;
   const thinfer_layer_weights& w = c->layers[layer];
   const LayerMaps& m = c->maps[layer];
   const int rows = batch * seq;
   const int qd = cf.n_q_heads * cf.head_dim, kvd = cf.n_kv_heads * cf.head_dim;
-  __half* kc = kv_ptr(c, slot, layer, 0);
-  __half* vc = kv_ptr(c, slot, layer, 1);
+  half_t* kc = kv_ptr(c, slot, layer, 0);
+  half_t* vc = kv_ptr(c, slot, layer, 1);
 
-  rmsnorm_rows(L, x_in, static_cast<const __half*>(w.attn_norm), c->h, rows, cf.hidden, cf.rms_eps);
+  rmsnorm_rows(L, x_in, static_cast<const half_t*>(w.attn_norm), c->h, rows, cf.hidden, cf.rms_eps);
   {
     const int nf[3] = {qd, kvd, kvd};
     tc_linear<EPI_QKV_ROPE>(L, THINFER_K_QKV, m.wq, m.wk, m.wv, c->h, rows, cf.hidden, nf, qkv_epi(c, c->qbuf, kc, vc, seq, 0));
@@ -787,7 +787,7 @@ void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __hal
     const int nf[3] = {cf.hidden, 0, 0};
     tc_linear<EPI_RESID>(L, THINFER_K_OPROJ, m.wo, m.wo, m.wo, c->attn, rows, qd, nf, e);
   }
-  rmsnorm_rows(L, c->x1, static_cast<const __half*>(w.ffn_norm), c->h, rows, cf.hidden, cf.rms_eps);
+  rmsnorm_rows(L, c->x1, static_cast<const half_t*>(w.ffn_norm), c->h, rows, cf.hidden, cf.rms_eps);
   {
     EpiArgs e{};
     e.out = c->act;
@@ -808,14 +808,14 @@ void layer_prefill(Launcher& L, thinfer_ctx* c, int slot, int layer, const __hal
 
 // pos: position of the new token (uniform slots), or the number of decode steps so far when `lens` (device,
 // per-request prompt lengths of a ragged slot) is given; max_t: keys the longest request attends.
-void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half* x_in, __half* x_out, int batch,
+void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const half_t* x_in, half_t* x_out, int batch,
                   int pos, const int* lens, int max_t) {
   const thinfer_config& cf = c->cfg;
   const thinfer_layer_weights& w = c->layers[layer];
   const int qd = cf.n_q_heads * cf.head_dim, kvd = cf.n_kv_heads * cf.head_dim;
-  __half* kc = kv_ptr(c, slot, layer, 0);
-  __half* vc = kv_ptr(c, slot, layer, 1);
-  auto H = [](const void* p) { return static_cast<const __half*>(p); };
+  half_t* kc = kv_ptr(c, slot, layer, 0);
+  half_t* vc = kv_ptr(c, slot, layer, 1);
+  auto H = [](const void* p) { return static_cast<const half_t*>(p); };
   if (batch <= kSkTokMax && c->skinny_ok) {
     // Up to 16 tokens: every projection is a balanced weight stream into warp-level tensor-core fragments
     // (no partial sums across CTAs, no tensor memory, so the CTAs of the next projection move in as this
@@ -823,7 +823,7 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     // is folded into the projection before it (gain there, 1/rms here); the first norm of a step has no
     // projection in front of it and runs as a prologue of the QKV projection.
     const bool first_norm_folded = layer > 0;
-    const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
+    const half_t* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
     {
       const int n[3] = {qd, kvd, kvd};
       if (first_norm_folded)
@@ -878,7 +878,7 @@ void layer_decode(Launcher& L, thinfer_ctx* c, int slot, int layer, const __half
     // epilogue also writes (output x next gain) and the per-tile sums of squares; the consumer multiplies
     // its sums by 1/rms.  Only the first norm of a step still needs its own small kernel.
     const bool first_norm_folded = layer > 0;
-    const __half* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
+    const half_t* next_gain = layer + 1 < cf.n_layers ? H(c->layers[layer + 1].attn_norm) : nullptr;
     if (!first_norm_folded) rmsnorm_rows(L, x_in, H(w.attn_norm), c->d_h, batch, cf.hidden, cf.rms_eps);
     {
       const int nf[3] = {qd, kvd, kvd};
@@ -971,7 +971,7 @@ void launch_mega(Launcher& L, thinfer_ctx* c, const MegaArgs& a) {
 
 bool mega_supported(const thinfer_ctx* c, int batch) { return batch <= 16; }
 
-void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* x_in, __half* x_out, int batch, int pos) {
+void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const half_t* x_in, half_t* x_out, int batch, int pos) {
   const thinfer_config& cf = c->cfg;
   MegaArgs a{};
   a.common = c->mega_common;
@@ -1028,11 +1028,11 @@ void layers_decode_unified(Launcher& L, thinfer_ctx* c, int slot, const __half* 
 }
 
 // final RMSNorm + LM head + greedy argmax on `batch` rows of x [batch][hidden]
-void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, int32_t* ids_out, float* logits_out,
+void head_and_argmax(Launcher& L, thinfer_ctx* c, const half_t* x, int batch, int32_t* ids_out, float* logits_out,
                      bool decode) {
   const thinfer_config& cf = c->cfg;
   float* lg = logits_out != nullptr ? logits_out : (decode ? c->d_logits : c->logits);
-  __half* hbuf = decode ? c->d_h : c->h;
+  half_t* hbuf = decode ? c->d_h : c->h;
   EpiArgs e{};
   e.out = lg;
   e.ld_out = cf.vocab;
@@ -1054,7 +1054,7 @@ void head_and_argmax(Launcher& L, thinfer_ctx* c, const __half* x, int batch, in
 }
 
 // inspection hook: a copy of the hidden state behind `layer` (-1: the input of layer 0), enqueued on the stream
-void capture_hidden(Launcher& L, thinfer_ctx* c, int layer, const __half* x, size_t rows) {
+void capture_hidden(Launcher& L, thinfer_ctx* c, int layer, const half_t* x, size_t rows) {
   if (L.rc != THINFER_OK) return;
   for (const auto& cap : c->captures) {
     if (cap.first != layer) continue;
@@ -1070,18 +1070,18 @@ int run_prefill(thinfer_ctx* c, int slot, const void* input, int batch, int seq,
   L.prefill_stage = true;
   if (c->trace_unified) L.go(-3, trace_reset_kernel, dim3(1), dim3(256), 0, c->timeline, 12);
   const int rows = batch * seq;
-  const __half* x = nullptr;
+  const half_t* x = nullptr;
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((rows + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
          c->embed, c->xa, rows, cf.hidden, cf.vocab);
     x = c->xa;
   } else {
-    x = static_cast<const __half*>(input);
+    x = static_cast<const half_t*>(input);
   }
-  __half* pong[2] = {c->xb, c->xa};
+  half_t* pong[2] = {c->xb, c->xa};
   if (!c->captures.empty()) capture_hidden(L, c, -1, x, rows);
   for (int l = 0; l < cf.n_layers; ++l) {
-    __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
+    half_t* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<half_t*>(out_primary) : pong[l & 1];
     layer_prefill(L, c, slot, l, x, dst, batch, seq);
     x = dst;
     if (!c->captures.empty()) capture_hidden(L, c, l, x, rows);
@@ -1099,15 +1099,15 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
   const thinfer_config& cf = c->cfg;
   Launcher L{c, st};
   if (c->trace_unified) L.go(-3, trace_reset_kernel, dim3(1), dim3(256), 0, c->timeline, 12);
-  const __half* x = nullptr;
+  const half_t* x = nullptr;
   if (cf.vocab > 0) {
     L.go(THINFER_K_EMBED, embed_gather_kernel, dim3((batch + 7) / 8), dim3(256), 0, static_cast<const int32_t*>(input),
          c->embed, c->d_xa, batch, cf.hidden, cf.vocab);
     x = c->d_xa;
   } else {
-    x = static_cast<const __half*>(input);
+    x = static_cast<const half_t*>(input);
   }
-  __half* pong[2] = {c->d_xb, c->d_xa};
+  half_t* pong[2] = {c->d_xb, c->d_xa};
   const Slot& sl = c->slots[slot];
   const int* lens = sl.ragged ? c->slot_lens + static_cast<size_t>(slot) * cf.max_batch : nullptr;
   const int step_pos = sl.ragged ? sl.steps : pos;  // ragged: every request adds its own prompt length on the device
@@ -1117,13 +1117,13 @@ int run_decode(thinfer_ctx* c, int slot, const void* input, int batch, int pos, 
       if (cap.first >= 0 && cap.first != cf.n_layers - 1)
         return fail(c, THINFER_EUNSUPPORTED, "launch mode 2 runs all layers in one kernel: only the last layer's "
                                              "hidden state can be captured");
-    __half* dst = cf.vocab == 0 ? static_cast<__half*>(out_primary) : pong[(cf.n_layers - 1) & 1];
+    half_t* dst = cf.vocab == 0 ? static_cast<half_t*>(out_primary) : pong[(cf.n_layers - 1) & 1];
     layers_decode_unified(L, c, slot, x, dst, batch, pos);
     x = dst;
     if (!c->captures.empty()) capture_hidden(L, c, cf.n_layers - 1, x, batch);
   } else {
     for (int l = 0; l < cf.n_layers; ++l) {
-      __half* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<__half*>(out_primary) : pong[l & 1];
+      half_t* dst = (cf.vocab == 0 && l == cf.n_layers - 1) ? static_cast<half_t*>(out_primary) : pong[l & 1];
       layer_decode(L, c, slot, l, x, dst, batch, step_pos, lens, pos + 1);
       x = dst;
       if (!c->captures.empty()) capture_hidden(L, c, l, x, batch);
@@ -1201,6 +1201,8 @@ int check_decode_args(thinfer_ctx* c, int slot, const void* input, void* out_pri
 // ============================================================================
 extern "C" {
 
+int thinfer_storage_type(void) { return kStorageType; }
+
 int thinfer_workspace_bytes(const thinfer_config* cfg, size_t* kv_bytes, size_t* scratch_bytes) {
   int rc = validate_config(cfg, &g_global_err);
   if (rc != THINFER_OK) return rc;
@@ -1245,9 +1247,9 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->sm_count = prop.multiProcessorCount;
   c->skinny_ok = cfg->hidden % 64 == 0 && cfg->ffn % 64 == 0 && (cfg->n_q_heads * cfg->head_dim) % 64 == 0;
   c->layers.assign(weights->layers, weights->layers + cfg->n_layers);
-  c->embed = static_cast<const __half*>(weights->embed);
-  c->final_norm = static_cast<const __half*>(weights->final_norm);
-  c->lm_head = static_cast<const __half*>(weights->lm_head);
+  c->embed = static_cast<const half_t*>(weights->embed);
+  c->final_norm = static_cast<const half_t*>(weights->final_norm);
+  c->lm_head = static_cast<const half_t*>(weights->lm_head);
   c->kv = static_cast<uint8_t*>(kv_workspace);
   c->kv_layer_bytes = kv_layer_bytes_of(*cfg);
   c->slots.assign(cfg->buf_slots, Slot{});
@@ -1267,14 +1269,14 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   uint8_t* s = static_cast<uint8_t*>(scratch);
   c->rope_cos = reinterpret_cast<float*>(s + p.rope_cos);
   c->rope_sin = reinterpret_cast<float*>(s + p.rope_sin);
-  c->h = reinterpret_cast<__half*>(s + p.h);
-  c->qbuf = reinterpret_cast<__half*>(s + p.qbuf);
-  c->attn = reinterpret_cast<__half*>(s + p.attn);
-  c->x1 = reinterpret_cast<__half*>(s + p.x1);
-  c->act = reinterpret_cast<__half*>(s + p.act);
-  c->xa = reinterpret_cast<__half*>(s + p.xa);
-  c->xb = reinterpret_cast<__half*>(s + p.xb);
-  c->last = reinterpret_cast<__half*>(s + p.last);
+  c->h = reinterpret_cast<half_t*>(s + p.h);
+  c->qbuf = reinterpret_cast<half_t*>(s + p.qbuf);
+  c->attn = reinterpret_cast<half_t*>(s + p.attn);
+  c->x1 = reinterpret_cast<half_t*>(s + p.x1);
+  c->act = reinterpret_cast<half_t*>(s + p.act);
+  c->xa = reinterpret_cast<half_t*>(s + p.xa);
+  c->xb = reinterpret_cast<half_t*>(s + p.xb);
+  c->last = reinterpret_cast<half_t*>(s + p.last);
   c->logits = reinterpret_cast<float*>(s + p.logits);
   c->ids_out = reinterpret_cast<int32_t*>(s + p.ids_out);
   c->part_o = reinterpret_cast<float*>(s + p.part_o);
@@ -1283,8 +1285,8 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->splitk_counters = reinterpret_cast<int*>(s + p.splitk_counters);
   c->pf_splitk_ws = reinterpret_cast<float*>(s + p.pf_splitk_ws);
   c->pf_splitk_counters = reinterpret_cast<int*>(s + p.pf_splitk_counters);
-  c->xg = reinterpret_cast<__half*>(s + p.xg);
-  c->x1g = reinterpret_cast<__half*>(s + p.x1g);
+  c->xg = reinterpret_cast<half_t*>(s + p.xg);
+  c->x1g = reinterpret_cast<half_t*>(s + p.x1g);
   c->sumsq0 = reinterpret_cast<float*>(s + p.sumsq0);
   c->sumsq1 = reinterpret_cast<float*>(s + p.sumsq1);
   c->attn_partial = reinterpret_cast<float*>(s + p.attn_partial);
@@ -1296,13 +1298,13 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
   c->stage_in = s + p.stage_in;
   c->stage_out = s + p.stage_out;
   c->slot_lens = reinterpret_cast<int*>(s + p.slot_lens);
-  c->d_h = reinterpret_cast<__half*>(s + p.d_h);
-  c->d_qbuf = reinterpret_cast<__half*>(s + p.d_qbuf);
-  c->d_attn = reinterpret_cast<__half*>(s + p.d_attn);
-  c->d_x1 = reinterpret_cast<__half*>(s + p.d_x1);
-  c->d_act = reinterpret_cast<__half*>(s + p.d_act);
-  c->d_xa = reinterpret_cast<__half*>(s + p.d_xa);
-  c->d_xb = reinterpret_cast<__half*>(s + p.d_xb);
+  c->d_h = reinterpret_cast<half_t*>(s + p.d_h);
+  c->d_qbuf = reinterpret_cast<half_t*>(s + p.d_qbuf);
+  c->d_attn = reinterpret_cast<half_t*>(s + p.d_attn);
+  c->d_x1 = reinterpret_cast<half_t*>(s + p.d_x1);
+  c->d_act = reinterpret_cast<half_t*>(s + p.d_act);
+  c->d_xa = reinterpret_cast<half_t*>(s + p.d_xa);
+  c->d_xb = reinterpret_cast<half_t*>(s + p.d_xb);
   c->d_logits = reinterpret_cast<float*>(s + p.d_logits);
   c->d_stage_in = s + p.d_stage_in;
   c->d_stage_out = s + p.d_stage_out;
@@ -1369,9 +1371,9 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     for (int l = 0; l < cfg->n_layers; ++l) {
       const LayerMaps& m = c->maps[l];
       ml[l].wq = m.wq; ml[l].wk = m.wk; ml[l].wv = m.wv; ml[l].wo = m.wo; ml[l].wg = m.wg; ml[l].wu = m.wu; ml[l].wd = m.wd;
-      ml[l].attn_norm = static_cast<const __half*>(c->layers[l].attn_norm);
-      ml[l].ffn_norm = static_cast<const __half*>(c->layers[l].ffn_norm);
-      ml[l].next_norm = l + 1 < cfg->n_layers ? static_cast<const __half*>(c->layers[l + 1].attn_norm) : nullptr;
+      ml[l].attn_norm = static_cast<const half_t*>(c->layers[l].attn_norm);
+      ml[l].ffn_norm = static_cast<const half_t*>(c->layers[l].ffn_norm);
+      ml[l].next_norm = l + 1 < cfg->n_layers ? static_cast<const half_t*>(c->layers[l + 1].attn_norm) : nullptr;
     }
     MegaCommon mc;
     const uint64_t rows = cfg->max_batch;
@@ -1652,24 +1654,24 @@ int thinfer_op_linear(const void* x, const void* w, void* y, int32_t rows, int32
   if (path == 1) {
     if (rows > 16) return THINFER_EUNSUPPORTED;
     if (out_fp32)
-      gemv<EPI_PLAIN_F32, false>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k,
-                                 static_cast<const __half*>(x), k, rows, nullptr, 0.f, e);
+      gemv<EPI_PLAIN_F32, false>(L, -2, static_cast<const half_t*>(w), nullptr, nullptr, n, k,
+                                 static_cast<const half_t*>(x), k, rows, nullptr, 0.f, e);
     else
-      gemv<EPI_PLAIN_F16, false>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k,
-                                 static_cast<const __half*>(x), k, rows, nullptr, 0.f, e);
+      gemv<EPI_PLAIN_F16, false>(L, -2, static_cast<const half_t*>(w), nullptr, nullptr, n, k,
+                                 static_cast<const half_t*>(x), k, rows, nullptr, 0.f, e);
   } else if (path == 2) {
     if (rows > kSkTokMax || k % 64 != 0) return THINFER_EUNSUPPORTED;
     if (out_fp32)
-      skinny<EPI_PLAIN_F32>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
+      skinny<EPI_PLAIN_F32>(L, -2, static_cast<const half_t*>(w), nullptr, nullptr, n, k, static_cast<const half_t*>(x), k,
                             rows, nullptr, 0, 0.f, e);
     else
-      skinny<EPI_PLAIN_F16>(L, -2, static_cast<const __half*>(w), nullptr, nullptr, n, k, static_cast<const __half*>(x), k,
+      skinny<EPI_PLAIN_F16>(L, -2, static_cast<const half_t*>(w), nullptr, nullptr, n, k, static_cast<const half_t*>(x), k,
                             rows, nullptr, 0, 0.f, e);
   } else if (path == 0) {
     CUtensorMap mw;
     if (!make_map_2d(&mw, w, k, n_out, 128)) return THINFER_ECUDA;
-    if (out_fp32) tc_linear<EPI_PLAIN_F32>(L, -2, mw, mw, mw, static_cast<const __half*>(x), rows, k, n, e);
-    else tc_linear<EPI_PLAIN_F16>(L, -2, mw, mw, mw, static_cast<const __half*>(x), rows, k, n, e);
+    if (out_fp32) tc_linear<EPI_PLAIN_F32>(L, -2, mw, mw, mw, static_cast<const half_t*>(x), rows, k, n, e);
+    else tc_linear<EPI_PLAIN_F16>(L, -2, mw, mw, mw, static_cast<const half_t*>(x), rows, k, n, e);
   } else {
     return THINFER_EINVAL;
   }
@@ -1748,8 +1750,8 @@ int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, vo
     return THINFER_EINVAL;
   if ((head_dim != 64 && head_dim != 128) || n_q_heads % n_kv_heads != 0) return THINFER_EUNSUPPORTED;
   Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
-  attn_prefill(L, static_cast<const __half*>(q), static_cast<const __half*>(k), static_cast<const __half*>(v),
-               static_cast<__half*>(out), batch, n_q_heads, n_kv_heads, seq, kv_stride, head_dim, nullptr);
+  attn_prefill(L, static_cast<const half_t*>(q), static_cast<const half_t*>(k), static_cast<const half_t*>(v),
+               static_cast<half_t*>(out), batch, n_q_heads, n_kv_heads, seq, kv_stride, head_dim, nullptr);
   return L.rc;
 }
 
@@ -1764,7 +1766,7 @@ int thinfer_op_rmsnorm(const void* x, const void* gain, void* y, int32_t rows, i
   if (x == nullptr || gain == nullptr || y == nullptr || rows <= 0 || n <= 0) return THINFER_EINVAL;
   if (n % 8 != 0) return THINFER_EUNSUPPORTED;
   Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};
-  rmsnorm_rows(L, static_cast<const __half*>(x), static_cast<const __half*>(gain), static_cast<__half*>(y), rows, n, eps);
+  rmsnorm_rows(L, static_cast<const half_t*>(x), static_cast<const half_t*>(gain), static_cast<half_t*>(y), rows, n, eps);
   return L.rc;
 }
 

@@ -121,11 +121,11 @@ def token_ids(shape: Shape, seed: int, dims, stream: int = 0) -> np.ndarray:
 # --------------------------------------------------------------------------- #
 # the same recipe drawn on the device (full-depth configurations)
 # --------------------------------------------------------------------------- #
-def _device_normal16(shape_, mean, std, key, device):
+def _device_normal16(shape_, mean, std, key, device, dtype=None):
     import torch
     g = torch.Generator(device=device)
     g.manual_seed(int(key))
-    t = torch.empty(shape_, dtype=torch.float16, device=device)
+    t = torch.empty(shape_, dtype=dtype or torch.float16, device=device)
     t.normal_(mean, std, generator=g)
     return t
 
@@ -134,22 +134,22 @@ def _key(seed, layer, tensor_id):
     return (int(seed) * 1_000_003 + int(layer)) * 1_009 + int(tensor_id) + 12_345
 
 
-def device_layer_weights(shape: Shape, seed: int, layer: int, device="cuda:0") -> dict:
-    """The nine tensors of one layer as CUDA FP16 tensors drawn on the device."""
+def device_layer_weights(shape: Shape, seed: int, layer: int, device="cuda:0", dtype=None) -> dict:
+    """The nine tensors of one layer as CUDA tensors drawn on the device (float16, or dtype=torch.bfloat16)."""
     out = {}
     for tid, name in enumerate(LAYER_TENSORS):
         mean = 1.0 if name.endswith("_norm") else 0.0
-        out[name] = _device_normal16(layer_tensor_shape(shape, name), mean, 0.02, _key(seed, layer, tid), device)
+        out[name] = _device_normal16(layer_tensor_shape(shape, name), mean, 0.02, _key(seed, layer, tid), device, dtype)
     return out
 
 
-def device_stack_weights(shape: Shape, seed: int = 0, device="cuda:0") -> dict:
+def device_stack_weights(shape: Shape, seed: int = 0, device="cuda:0", dtype=None) -> dict:
     """Whole model on the device: {"layers": [dict per layer], "embed", "final_norm", "lm_head"}."""
-    out = {"layers": [device_layer_weights(shape, seed, l, device) for l in range(shape.n_layers)]}
+    out = {"layers": [device_layer_weights(shape, seed, l, device, dtype) for l in range(shape.n_layers)]}
     for i, name in enumerate(_STACK_TENSORS):
         dims = (shape.hidden,) if name == "final_norm" else (shape.vocab, shape.hidden)
         out[name] = _device_normal16(dims, 1.0 if name == "final_norm" else 0.0, 0.02,
-                                     _key(seed, 1 << 20, 50 + i), device)
+                                     _key(seed, 1 << 20, 50 + i), device, dtype)
     return out
 
 

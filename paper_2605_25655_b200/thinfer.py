@@ -11,6 +11,8 @@ import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libthinfer.so")
+# one build per 16-bit storage type, same exports (include/thinfer.h)
+LIB_PATHS = {"f16": LIB_PATH, "bf16": os.path.join(_HERE, "libthinfer_bf16.so")}
 
 OK, EINVAL, EUNSUPPORTED, ECAPACITY, EBUSY, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 ERR_NAMES = {OK: "THINFER_OK", EINVAL: "THINFER_EINVAL", EUNSUPPORTED: "THINFER_EUNSUPPORTED",
@@ -19,7 +21,7 @@ ERR_NAMES = {OK: "THINFER_OK", EINVAL: "THINFER_EINVAL", EUNSUPPORTED: "THINFER_
 K_RMSNORM, K_QKV, K_ATTN, K_ATTN_COMBINE, K_OPROJ, K_GATEUP, K_DOWN, K_HEAD, K_EMBED, K_ARGMAX, K_DECODE_UNIFIED = range(11)
 
 EXPORTS = (
-    "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_prefill_ragged", "thinfer_slot_lengths",
+    "thinfer_storage_type", "thinfer_workspace_bytes", "thinfer_create", "thinfer_prefill", "thinfer_prefill_ragged", "thinfer_slot_lengths",
     "thinfer_decode_step",
     "thinfer_prefill_host", "thinfer_decode_step_host", "thinfer_release_slot", "thinfer_slot_state",
     "thinfer_kv_pointer", "thinfer_status", "thinfer_clear_status", "thinfer_capture_hidden", "thinfer_set_launch_mode", "thinfer_profile_select",
@@ -52,18 +54,30 @@ class Weights(C.Structure):
                 ("lm_head", C.c_void_p)]
 
 
-_lib = None
+_libs = {}
 
 
-def lib():
-    """Loads the shared library (once).  Fails loudly when it has not been built."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
-        raise ThinferError(ECUDA, f"{LIB_PATH} is missing: build it with "
+def storage_of(tensor) -> str:
+    """'f16' or 'bf16' for a torch tensor of a storage type the library is built for."""
+    import torch
+    if tensor.dtype == torch.float16:
+        return "f16"
+    if tensor.dtype == torch.bfloat16:
+        return "bf16"
+    raise ThinferError(EUNSUPPORTED, f"storage type {tensor.dtype}: the library is built for float16 and bfloat16")
+
+
+def lib(storage="f16"):
+    """Loads the shared library of a storage type (once).  Fails loudly when it has not been built."""
+    if storage in _libs:
+        return _libs[storage]
+    path = LIB_PATHS[storage]
+    if not os.path.exists(path):
+        raise ThinferError(ECUDA, f"{path} is missing: build it with "
                                   "`python -m paper_2605_25655_b200._build` (needs nvcc)")
-    L = C.CDLL(LIB_PATH)
+    L = C.CDLL(path)
+    L.thinfer_storage_type.argtypes = []
+    assert L.thinfer_storage_type() == {"f16": 0, "bf16": 1}[storage], path
     vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
     L.thinfer_workspace_bytes.argtypes = [C.POINTER(Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.thinfer_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
@@ -95,13 +109,13 @@ def lib():
     L.thinfer_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, C.c_float, vp]
     L.thinfer_op_argmax.argtypes = [vp, vp, i32, i32, vp]
     L.thinfer_selftest_bounded_wait.argtypes = [vp, i64, vp]
-    _lib = L
+    _libs[storage] = L
     return L
 
 
-def _check(rc, ctx=None):
+def _check(rc, ctx=None, storage="f16"):
     if rc != OK:
-        msg = lib().thinfer_last_error(ctx)
+        msg = lib(storage).thinfer_last_error(ctx)
         raise ThinferError(rc, msg.decode() if msg else "")
 
 
@@ -117,16 +131,16 @@ def make_config(shape, max_batch, max_seq, buf_slots=1) -> Config:
                   shape.vocab, shape.rms_eps, shape.rope_base, max_batch, max_seq, buf_slots)
 
 
-def workspace_bytes(cfg: Config):
+def workspace_bytes(cfg: Config, storage="f16"):
     kv, sc = C.c_size_t(0), C.c_size_t(0)
-    _check(lib().thinfer_workspace_bytes(C.byref(cfg), C.byref(kv), C.byref(sc)))
+    _check(lib(storage).thinfer_workspace_bytes(C.byref(cfg), C.byref(kv), C.byref(sc)), None, storage)
     return kv.value, sc.value
 
 
 class Context:
     """One thinfer_ctx plus the torch tensors that back its caller-owned memory.
 
-    layers: list of dicts name -> CUDA FP16 tensor (names of thinfer_layer_weights);
+    layers: list of dicts name -> CUDA float16 (or bfloat16) tensor (names of thinfer_layer_weights);
     stack:  dict with embed / final_norm / lm_head when shape.vocab > 0.
     """
 
@@ -136,7 +150,10 @@ class Context:
         self.shape = shape
         self.device = torch.device(device)
         self.cfg = make_config(shape, max_batch, max_seq, buf_slots)
-        kv_bytes, scratch_bytes = workspace_bytes(self.cfg)
+        self.storage = storage_of(layers[0]["wq"])         # the weights decide which build serves this context
+        self.dtype = layers[0]["wq"].dtype
+        self.L = lib(self.storage)
+        kv_bytes, scratch_bytes = workspace_bytes(self.cfg, self.storage)
         with torch.cuda.device(self.device):
             self.kv = torch.empty(kv_bytes, dtype=torch.uint8, device=self.device)
             self.scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=self.device)
@@ -145,14 +162,14 @@ class Context:
             for l, w in enumerate(layers):
                 for name, _ in LayerWeights._fields_:
                     t = w[name]
-                    assert t.is_cuda and t.dtype == torch.float16 and t.is_contiguous(), name
+                    assert t.is_cuda and t.dtype == self.dtype and t.is_contiguous(), name
                     setattr(arr[l], name, t.data_ptr())
             wts = Weights(arr, None, None, None)
             if shape.vocab > 0:
                 wts.embed, wts.final_norm, wts.lm_head = (stack[n].data_ptr() for n in ("embed", "final_norm", "lm_head"))
             h = C.c_void_p(None)
-            _check(lib().thinfer_create(C.byref(self.cfg), C.byref(wts), self.kv.data_ptr(), kv_bytes,
-                                        self.scratch.data_ptr(), scratch_bytes, C.byref(h)))
+            _check(self.L.thinfer_create(C.byref(self.cfg), C.byref(wts), self.kv.data_ptr(), kv_bytes,
+                                         self.scratch.data_ptr(), scratch_bytes, C.byref(h)), None, self.storage)
         self.h = h
 
     # -- device-buffer calls ------------------------------------------------
@@ -161,16 +178,16 @@ class Context:
         batch, seq = int(inp.shape[0]), int(inp.shape[1])
         assert inp.is_cuda and inp.is_contiguous()
         if self.shape.vocab == 0:
-            assert inp.dtype == torch.float16
+            assert inp.dtype == self.dtype
             out = torch.empty_like(inp)
-            _check(lib().thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, out.data_ptr(), None,
-                                         _stream_ptr(stream)), self.h)
+            _check(self.L.thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, out.data_ptr(), None,
+                                         _stream_ptr(stream)), self.h, self.storage)
             return out
         assert inp.dtype == torch.int32
         ids = torch.empty(batch, dtype=torch.int32, device=self.device)
         logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
-        _check(lib().thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, ids.data_ptr(),
-                                     logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        _check(self.L.thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, ids.data_ptr(),
+                                     logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h, self.storage)
         return (ids, logits) if want_logits else ids
 
     def prefill_ragged(self, inp, seq_lens, slot=0, stream=None, want_logits=False):
@@ -181,19 +198,19 @@ class Context:
         assert inp.is_cuda and inp.is_contiguous()
         if self.shape.vocab == 0:
             out = torch.empty_like(inp)
-            _check(lib().thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, out.data_ptr(), None,
-                                                _stream_ptr(stream)), self.h)
+            _check(self.L.thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, out.data_ptr(), None,
+                                                _stream_ptr(stream)), self.h, self.storage)
             return out
         ids = torch.empty(batch, dtype=torch.int32, device=self.device)
         logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
-        _check(lib().thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, ids.data_ptr(),
-                                            logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        _check(self.L.thinfer_prefill_ragged(self.h, slot, inp.data_ptr(), batch, seq, lens, ids.data_ptr(),
+                                            logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h, self.storage)
         return (ids, logits) if want_logits else ids
 
     def slot_lengths(self, slot=0):
         b, _ = self.slot_state(slot)
         buf = (C.c_int32 * max(b, 1))()
-        _check(lib().thinfer_slot_lengths(self.h, slot, buf), self.h)
+        _check(self.L.thinfer_slot_lengths(self.h, slot, buf), self.h, self.storage)
         return list(buf)[:b]
 
     def decode_step(self, inp, slot=0, stream=None, want_logits=False, out=None):
@@ -201,56 +218,56 @@ class Context:
         assert inp.is_cuda and inp.is_contiguous()
         if self.shape.vocab == 0:
             out = torch.empty_like(inp) if out is None else out
-            _check(lib().thinfer_decode_step(self.h, slot, inp.data_ptr(), out.data_ptr(), None,
-                                             _stream_ptr(stream)), self.h)
+            _check(self.L.thinfer_decode_step(self.h, slot, inp.data_ptr(), out.data_ptr(), None,
+                                             _stream_ptr(stream)), self.h, self.storage)
             return out
         batch = int(inp.shape[0])
         ids = torch.empty(batch, dtype=torch.int32, device=self.device) if out is None else out
         logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
-        _check(lib().thinfer_decode_step(self.h, slot, inp.data_ptr(), ids.data_ptr(),
-                                         logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h)
+        _check(self.L.thinfer_decode_step(self.h, slot, inp.data_ptr(), ids.data_ptr(),
+                                         logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h, self.storage)
         return (ids, logits) if want_logits else ids
 
     # -- host-buffer calls (pinned tensors make the copies asynchronous) -----
     def prefill_host(self, host_in, host_out, slot=0, stream=None, host_logits=None):
         batch, seq = int(host_in.shape[0]), int(host_in.shape[1])
-        _check(lib().thinfer_prefill_host(self.h, slot, host_in.data_ptr(), batch, seq, host_out.data_ptr(),
+        _check(self.L.thinfer_prefill_host(self.h, slot, host_in.data_ptr(), batch, seq, host_out.data_ptr(),
                                           host_logits.data_ptr() if host_logits is not None else None,
-                                          _stream_ptr(stream)), self.h)
+                                          _stream_ptr(stream)), self.h, self.storage)
 
     def decode_step_host(self, host_in, host_out, slot=0, stream=None, host_logits=None):
-        _check(lib().thinfer_decode_step_host(self.h, slot, host_in.data_ptr(), host_out.data_ptr(),
+        _check(self.L.thinfer_decode_step_host(self.h, slot, host_in.data_ptr(), host_out.data_ptr(),
                                               host_logits.data_ptr() if host_logits is not None else None,
-                                              _stream_ptr(stream)), self.h)
+                                              _stream_ptr(stream)), self.h, self.storage)
 
     # -- bookkeeping ----------------------------------------------------------
     def release_slot(self, slot=0, stream=None):
-        _check(lib().thinfer_release_slot(self.h, slot, _stream_ptr(stream)), self.h)
+        _check(self.L.thinfer_release_slot(self.h, slot, _stream_ptr(stream)), self.h, self.storage)
 
     def slot_state(self, slot=0):
         b, n = C.c_int32(0), C.c_int32(0)
-        _check(lib().thinfer_slot_state(self.h, slot, C.byref(b), C.byref(n)), self.h)
+        _check(self.L.thinfer_slot_state(self.h, slot, C.byref(b), C.byref(n)), self.h, self.storage)
         return b.value, n.value
 
     def kv_view(self, slot, layer, which):
         """Strided torch view [max_batch][n_kv_heads][max_seq][head_dim] of K (0) or V (1)."""
         p = C.c_void_p(None)
-        _check(lib().thinfer_kv_pointer(self.h, slot, layer, which, C.byref(p)), self.h)
+        _check(self.L.thinfer_kv_pointer(self.h, slot, layer, which, C.byref(p)), self.h, self.storage)
         off = p.value - self.kv.data_ptr()
         n = self.cfg.max_batch * self.cfg.n_kv_heads * self.cfg.max_seq * self.cfg.head_dim
-        return self.kv[off:off + 2 * n].view(self.torch.float16).view(
+        return self.kv[off:off + 2 * n].view(self.dtype).view(
             self.cfg.max_batch, self.cfg.n_kv_heads, self.cfg.max_seq, self.cfg.head_dim)
 
     def status(self):
         v = C.c_int32(0)
-        _check(lib().thinfer_status(self.h, C.byref(v)), self.h)
+        _check(self.L.thinfer_status(self.h, C.byref(v)), self.h, self.storage)
         return v.value
 
     def clear_status(self):
-        _check(lib().thinfer_clear_status(self.h), self.h)
+        _check(self.L.thinfer_clear_status(self.h), self.h, self.storage)
 
     def selftest_bounded_wait(self, limit_ns=1_000_000, stream=None):
-        _check(lib().thinfer_selftest_bounded_wait(self.h, int(limit_ns), _stream_ptr(stream)), self.h)
+        _check(self.L.thinfer_selftest_bounded_wait(self.h, int(limit_ns), _stream_ptr(stream)), self.h, self.storage)
 
     def capture_hidden(self, captures):
         """captures: dict layer index (-1 = input of layer 0) -> CUDA FP16 tensor that receives the hidden
@@ -260,31 +277,31 @@ class Context:
         layers = (C.c_int32 * max(n, 1))(*[int(l) for l in captures])
         bufs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in captures.values()])
         self._captures = captures                      # keeps the tensors alive
-        _check(lib().thinfer_capture_hidden(self.h, n, layers, bufs), self.h)
+        _check(self.L.thinfer_capture_hidden(self.h, n, layers, bufs), self.h, self.storage)
 
     def set_launch_mode(self, mode):
-        _check(lib().thinfer_set_launch_mode(self.h, mode), self.h)
+        _check(self.L.thinfer_set_launch_mode(self.h, mode), self.h, self.storage)
 
     def profile_select(self, kernel_id):
-        _check(lib().thinfer_profile_select(self.h, kernel_id), self.h)
+        _check(self.L.thinfer_profile_select(self.h, kernel_id), self.h, self.storage)
 
     def profile_read(self):
         n, ms = C.c_int32(0), C.c_float(0)
-        _check(lib().thinfer_profile_read(self.h, C.byref(n), C.byref(ms)), self.h)
+        _check(self.L.thinfer_profile_read(self.h, C.byref(n), C.byref(ms)), self.h, self.storage)
         return n.value, ms.value
 
     def trace_unified(self, enable=True, read=0):
         """Switches the unit-boundary trace of the unified decode kernel on/off; returns `read` entries (ns)."""
         buf = (C.c_uint64 * max(read, 1))()
-        _check(lib().thinfer_trace_unified(self.h, int(enable), buf if read else None, read), self.h)
+        _check(self.L.thinfer_trace_unified(self.h, int(enable), buf if read else None, read), self.h, self.storage)
         return list(buf)[:read]
 
     def launch_count(self):
-        return int(lib().thinfer_launch_count(self.h))
+        return int(self.L.thinfer_launch_count(self.h))
 
     def close(self):
         if self.h is not None and self.h.value:
-            lib().thinfer_destroy(self.h)
+            self.L.thinfer_destroy(self.h)
             self.h = None
 
     def __del__(self):
@@ -302,9 +319,10 @@ def op_linear(x, w, out_fp32=False, path=0, stream=None, out=None):
     if out is not None:
         y, out_fp32 = out, out.dtype == torch.float32
     else:
-        y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else torch.float16, device=x.device)
-    _check(lib().thinfer_op_linear(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k, int(out_fp32), path,
-                                   _stream_ptr(stream)))
+        y = torch.empty(rows, n_out, dtype=torch.float32 if out_fp32 else x.dtype, device=x.device)
+    st = storage_of(x)
+    _check(lib(st).thinfer_op_linear(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k, int(out_fp32), path,
+                                     _stream_ptr(stream)), None, st)
     return y
 
 
@@ -316,8 +334,9 @@ def op_linear_noalloc(x, w, y, stream=None):
     rows, k = x.shape
     n_out = w.shape[0]
     assert y.shape == (rows, n_out) and y.is_contiguous()
-    _check(lib().thinfer_op_linear_noalloc(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k,
-                                           int(y.dtype == torch.float32), _stream_ptr(stream)))
+    st = storage_of(x)
+    _check(lib(st).thinfer_op_linear_noalloc(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, n_out, k,
+                                             int(y.dtype == torch.float32), _stream_ptr(stream)), None, st)
     return y
 
 
@@ -327,9 +346,10 @@ def op_attention_prefill(q, k, v, seq=None, stream=None, out=None):
     b, hq, s, d = q.shape
     hkv, t = k.shape[1], k.shape[2]
     if out is None:
-        out = torch.empty(b, s, hq * d, dtype=torch.float16, device=q.device)
-    _check(lib().thinfer_op_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), b, hq, hkv,
-                                              s, t, d, _stream_ptr(stream)))
+        out = torch.empty(b, s, hq * d, dtype=q.dtype, device=q.device)
+    st = storage_of(q)
+    _check(lib(st).thinfer_op_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), b, hq, hkv,
+                                                s, t, d, _stream_ptr(stream)), None, st)
     return out
 
 
@@ -337,7 +357,8 @@ def op_rmsnorm(x, gain, eps, stream=None):
     import torch
     rows, n = x.shape
     y = torch.empty_like(x)
-    _check(lib().thinfer_op_rmsnorm(x.data_ptr(), gain.data_ptr(), y.data_ptr(), rows, n, eps, _stream_ptr(stream)))
+    st = storage_of(x)
+    _check(lib(st).thinfer_op_rmsnorm(x.data_ptr(), gain.data_ptr(), y.data_ptr(), rows, n, eps, _stream_ptr(stream)), None, st)
     return y
 
 

@@ -26,8 +26,11 @@ def _declared():
 def test_every_declared_symbol_is_exported(lib):
     names = _declared()
     assert set(names) == set(thinfer.EXPORTS)
-    for n in names:
-        assert hasattr(lib, n), n
+    for storage, code in (("f16", 0), ("bf16", 1)):          # one build per storage type, the same exports
+        L = thinfer.lib(storage)
+        for n in names:
+            assert hasattr(L, n), (storage, n)
+        assert L.thinfer_storage_type() == code
     for n in ("thinfer_create", "thinfer_prefill", "thinfer_decode_step", "thinfer_destroy"):
         assert n in names
 
