@@ -274,13 +274,14 @@ def whole_job_rate(units_per_rank, world, seconds):
 class Runner:
     """One workload on one device: weights, context, inputs, and the step functions the legs time."""
 
-    def __init__(self, wl, batch, dev, torch, thinfer):
+    def __init__(self, wl, batch, dev, torch, thinfer, storage="f16"):
         self.wl, self.B, self.dev, self.torch, self.thinfer = wl, batch, dev, torch, thinfer
         s, B = wl.shape, batch
+        dt = torch.bfloat16 if storage == "bf16" else torch.float16
         self.steps_dec = wl.decode_steps
         max_seq = wl.prompt + wl.decode_steps
         if wl.stack:
-            sw = synth.device_stack_weights(s, seed=0, device=dev)
+            sw = synth.device_stack_weights(s, seed=0, device=dev, dtype=dt)
             self.sw = sw
             self.ctx = thinfer.Context(s, sw["layers"], {n: sw[n] for n in ("embed", "final_norm", "lm_head")},
                                        max_batch=B, max_seq=max_seq, device=dev)
@@ -292,16 +293,19 @@ class Runner:
             self.h_ids_out = torch.zeros(B, dtype=torch.int32).pin_memory()
             self.h2d, self.d2h = B * 4, B * 4
         else:
-            self.layers = thinfer.to_device_layers([synth.layer_weights(s, seed=0)], device=dev)
+            if storage == "bf16":
+                self.layers = [synth.device_layer_weights(s, 0, 0, device=dev, dtype=dt)]
+            else:
+                self.layers = thinfer.to_device_layers([synth.layer_weights(s, seed=0)], device=dev)
             self.ctx = thinfer.Context(s, self.layers, None, max_batch=B, max_seq=max_seq, device=dev)
-            x_all = torch.from_numpy(synth.hidden_states(s, 0, (B, wl.prompt + wl.gen)))
+            x_all = torch.from_numpy(synth.hidden_states(s, 0, (B, wl.prompt + wl.gen))).to(dt)
             self.h_prompt = x_all[:, :wl.prompt].contiguous().pin_memory()
             self.prompt = self.h_prompt.to(dev)
             self.h_prompt_out = torch.empty_like(self.h_prompt).pin_memory()
             self.h_dec = [x_all[:, wl.prompt + i].contiguous().pin_memory() for i in range(wl.gen)]
             self.x_dec = [t.to(dev) for t in self.h_dec]
-            self.out_dec = torch.empty(B, s.hidden, dtype=torch.float16, device=dev)
-            self.h_dec_out = torch.empty(B, s.hidden, dtype=torch.float16).pin_memory()
+            self.out_dec = torch.empty(B, s.hidden, dtype=dt, device=dev)
+            self.h_dec_out = torch.empty(B, s.hidden, dtype=dt).pin_memory()
             self.h2d, self.d2h = B * s.hidden * 2, B * s.hidden * 2
 
     def prefill(self):
@@ -375,7 +379,7 @@ def run_ours(args, wl):
     B = args.batch or wl.batch
     S, s = wl.prompt, wl.shape
     peaks, peak_kind = measured_peaks()
-    R = Runner(wl, B, dev, torch, thinfer)
+    R = Runner(wl, B, dev, torch, thinfer, args.storage)
     ctx = R.ctx
     n_dec = wl.decode_steps
 
@@ -452,8 +456,8 @@ def run_ours(args, wl):
     line = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": tot_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-        "config": {"workload": wl.name(B), "key": wl.key, "batch": B, "prompt": S, "generate": wl.gen,
+        "vs_baseline": None, "dtype": args.storage, "data": "synthetic",
+        "config": {"workload": wl.name(B).replace("FP16", "BF16") if args.storage == "bf16" else wl.name(B), "key": wl.key, "batch": B, "prompt": S, "generate": wl.gen,
                    "decode_steps_per_pass": n_dec,
                    "value_is": "batch x decode steps / decode-phase time; ms_per_step covers prefill + decode",
                    "l2": f"no flush: the {weights_gb:.1f} GB of weights streamed by every decode step and the prefill "
@@ -623,6 +627,8 @@ def main():
     ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS),
                     help="c2: 7B layer; c3: 7B stack; c4: 13B stack; c5: 70B stack (default)")
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (c2: 1, 4, 16)")
+    ap.add_argument("--storage", default="f16", choices=["f16", "bf16"],
+                    help="16-bit storage type of weights, activations and KV cache (the BF16 build of the library)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", choices=["prefill", "decode", "stack"], default=None,

@@ -136,7 +136,24 @@ __global__ void __launch_bounds__(1024) argmax_rows_kernel(const float* __restri
   const float* row = logits + static_cast<size_t>(blockIdx.x) * n;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+  // eight independent loads in flight per thread: the row comes out of L2 and a dependent chain of single
+  // loads would be all latency.
+  constexpr int kU = 8;
+  int i = threadIdx.x;
+  for (; i + (kU - 1) * static_cast<int>(blockDim.x) < n; i += kU * blockDim.x) {
+    float v[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) v[u] = __ldcs(row + i + u * blockDim.x);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int idx = i + u * blockDim.x;
+      if (v[u] > best || (v[u] == best && idx < bi)) {
+        best = v[u];
+        bi = idx;
+      }
+    }
+  }
+  for (; i < n; i += blockDim.x) {
     const float v = row[i];
     if (v > best || (v == best && i < bi)) {
       best = v;
