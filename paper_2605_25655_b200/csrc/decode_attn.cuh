@@ -10,6 +10,8 @@
 // finishes last (a ticket counter; the partials are added in segment order, so
 // the result does not depend on who that is).
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace thinfer {
@@ -17,6 +19,7 @@ namespace thinfer {
 constexpr int kAttnDecWarps = 4;
 constexpr int kAttnDecUnroll = 4;
 constexpr int kAttnMaxSplits = 32;
+constexpr int kAttnMaxCluster = 8;   // CTAs of one pair that merge through distributed shared memory
 
 struct AttnDecArgs {
   const half_t* q;        // [batch][n_q_heads][D], already rotated
@@ -32,6 +35,8 @@ struct AttnDecArgs {
   int t_max;
   int n_pairs;            // batch * n_q_heads / G
   int units_per_pair;     // ceil(longest key count / keys per CTA-wide iteration)
+  int cluster;            // > 1: the launch uses thread-block clusters of this many CTAs, one cluster per pair; the
+                          // segments of a pair are then merged in the shared memory of the cluster's first CTA
   float scale_log2;       // log2(e) / sqrt(D)
   unsigned long long* dbg;  // tracing aid (16 slots) or nullptr
 };
@@ -152,9 +157,13 @@ struct AttnMergeSmem {
 // warps; a pair with one segment is finished here, otherwise the segment's partial goes to global memory and the
 // CTA of the pair that arrives last merges all of them, in segment order.
 template <int D, int G>
-__device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMergeSmem<D, G>& sm, int b, int h0, int pair,
-                                                    int seg, int n_seg) {
+__device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMergeSmem<D, G>& sm, float* cl_buf, int b,
+                                                    int h0, int pair, int seg, int n_seg) {
+  namespace cg = cooperative_groups;
   const size_t bh0 = static_cast<size_t>(b) * a.n_q_heads + h0;
+  const bool clustered = a.cluster > 1;  // then n_seg == a.cluster and seg == the CTA's rank in its cluster
+  // cluster path: segment s leaves [G][D + 2] floats (output row, then max and sum) in the first CTA's buffer
+  float* lead = clustered ? cg::this_cluster().map_shared_rank(cl_buf, 0) : nullptr;
   for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
     const int g = idx / D, i = idx - g * D;
     float mx = sm.m[0][g];
@@ -170,6 +179,13 @@ __device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMe
     }
     if (n_seg == 1) {
       a.out[(bh0 + g) * D + i] = f_to_h(O / L);
+    } else if (clustered) {
+      float* dst = lead + (seg * G + g) * (D + 2);
+      dst[i] = O;
+      if (i == 0) {
+        dst[D] = mx;
+        dst[D + 1] = L;
+      }
     } else {
       const size_t p = (bh0 + g) * kAttnMaxSplits + seg;
       a.part_o[p * D + i] = O;
@@ -179,7 +195,36 @@ __device__ __forceinline__ void attn_finish_segment(const AttnDecArgs& a, AttnMe
       }
     }
   }
-  if (n_seg > 1) {
+  if (n_seg > 1 && clustered) {
+    // every CTA of the pair has stored its segment in the first CTA's shared memory: one cluster barrier, then
+    // that CTA merges them in segment order (no round trip through L2, no ticket)
+    cg::this_cluster().sync();
+    if (seg == 0) {
+      if (threadIdx.x < G) {
+        const int g = threadIdx.x;
+        float mx = -INFINITY;
+        for (int sg = 0; sg < n_seg; ++sg) mx = fmaxf(mx, cl_buf[(sg * G + g) * (D + 2) + D]);
+        float L = 0.f;
+        for (int sg = 0; sg < n_seg; ++sg) {
+          float* ml = cl_buf + (sg * G + g) * (D + 2) + D;
+          const float al = exp2f(ml[0] - mx);  // an empty segment has max -inf: weight 0
+          L += ml[1] * al;
+          ml[0] = al;
+        }
+        cl_buf[g * (D + 2) + D + 1] = 1.f / L;
+      }
+      __syncthreads();
+      for (int idx = threadIdx.x; idx < G * D; idx += kAttnDecWarps * 32) {
+        const int g = idx / D, i = idx - g * D;
+        float acc = 0.f;
+        for (int sg = 0; sg < n_seg; ++sg) {
+          const float* row = cl_buf + (sg * G + g) * (D + 2);
+          acc = fmaf(row[i], row[D], acc);
+        }
+        a.out[(bh0 + g) * D + i] = f_to_h(acc * cl_buf[g * (D + 2) + D + 1]);
+      }
+    }
+  } else if (n_seg > 1) {
     // the CTA that arrives last merges the segments of its G heads,
     // out = sum_s o_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), s in segment order
     __threadfence();
@@ -261,6 +306,7 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
   constexpr int UN = kAttnDecUnroll;
   constexpr int UNIT = kAttnDecWarps * UN * KPL;  // keys of one CTA-wide iteration
   __shared__ AttnMergeSmem<D, G> sm;
+  __shared__ float cl_buf[kAttnMaxCluster * G * (D + 2)];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane / LPK, dl = lane % LPK;
@@ -322,7 +368,7 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_kernel(const A
       }
     }
     __syncthreads();
-    attn_finish_segment<D, G>(a, sm, b, h0, pair, seg, n_seg);
+    attn_finish_segment<D, G>(a, sm, cl_buf, b, h0, pair, seg, n_seg);
     __syncthreads();  // the shared arrays are reused by the next segment
   }
   if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));

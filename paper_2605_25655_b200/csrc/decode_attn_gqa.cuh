@@ -28,10 +28,16 @@ namespace thinfer {
 constexpr int kGqaChunk = 16;                              // keys per MMA block of a warp
 constexpr int kGqaUnit = kAttnDecWarps * kGqaChunk;        // keys of one CTA-wide iteration
 constexpr int kGqaStages = 2;
+constexpr int kGqaMaxCluster = 4;   // CTAs of one pair that merge through distributed shared memory
 
 template <int D>
 __host__ __device__ constexpr int gqa_ring_bytes() {
   return kAttnDecWarps * kGqaStages * 2 * kGqaChunk * D * 2;  // warps x stages x (K, V) x 16 rows x D halves
+}
+// dynamic shared memory: the K/V ring, then the buffer the segments of a cluster are merged in
+template <int D, int G>
+__host__ __device__ constexpr int gqa_smem_bytes() {
+  return gqa_ring_bytes<D>() + kGqaMaxCluster * G * (D + 2) * 4;
 }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr) {
@@ -72,6 +78,7 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_gqa_kernel(con
   auto cta_of = [&](long long x) { return static_cast<int>(((x + 1) * grid - 1) / n_units); };
 
   uint8_t* ring = gqa_ring + warp * (kGqaStages * 2 * TILE_BYTES);  // [stage][K | V][16 rows][ROW_BYTES]
+  float* cl_buf = reinterpret_cast<float*>(gqa_ring + gqa_ring_bytes<D>());
   const uint32_t ring_u32 = smem_u32(ring);
 
   for (long long u = u_beg; u < u_end;) {
@@ -208,7 +215,7 @@ __global__ void __launch_bounds__(kAttnDecWarps * 32) attn_decode_gqa_kernel(con
         *reinterpret_cast<float2*>(&sm.o[warp][g][8 * j + 2 * t]) = make_float2(o[j][0], o[j][1]);
     }
     __syncthreads();
-    attn_finish_segment<D, G>(a, sm, b, h0, pair, seg, n_seg);
+    attn_finish_segment<D, G>(a, sm, cl_buf, b, h0, pair, seg, n_seg);
     __syncthreads();  // the shared arrays are reused by the next segment
   }
   if (a.dbg != nullptr && threadIdx.x == 0) atomicMax(a.dbg + 15, static_cast<unsigned long long>(global_ns()));

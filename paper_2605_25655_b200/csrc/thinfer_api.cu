@@ -136,6 +136,7 @@ struct thinfer_ctx {
   uint8_t *stage_in = nullptr, *stage_out = nullptr;
   int max_splits = 1;
   int attn_waves = 1, attn_min_units = 2;  // split-KV schedule of decode attention (tuning aids)
+  int attn_cluster = 1;                    // merge the segments of a pair inside a thread-block cluster when they fit
   int sk_max_tiles = 0;                    // tuning aid: cap on the tiles of a skinny share (0: the built-in limits)
   int trace_cta_kid = -1;                  // kernel id whose CTAs log their own times while tracing is on
   // status word (pinned, mapped)
@@ -287,6 +288,7 @@ struct Launcher {
   int rc = THINFER_OK;
   bool cooperative = false;  // next launch only: all CTAs must be co-resident (grid-wide barriers inside)
   bool prefill_stage = false;  // stream-K scratch of the prefill stage instead of the decode stage's
+  int cluster = 0;             // next launch only: thread-block clusters of this many CTAs along x
 
   template <typename... KArgs, typename... Args>
   void go(int kid, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
@@ -310,7 +312,7 @@ struct Launcher {
     lc.blockDim = block;
     lc.dynamicSmemBytes = smem;
     lc.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     lc.attrs = attr;
     lc.numAttrs = 0;
     if (cooperative) {
@@ -323,6 +325,14 @@ struct Launcher {
       attr[0].val.programmaticStreamSerializationAllowed = 1;
       lc.numAttrs = 1;
     }
+    if (cluster > 1) {
+      attr[lc.numAttrs].id = cudaLaunchAttributeClusterDimension;
+      attr[lc.numAttrs].val.clusterDim.x = static_cast<unsigned>(cluster);
+      attr[lc.numAttrs].val.clusterDim.y = 1;
+      attr[lc.numAttrs].val.clusterDim.z = 1;
+      ++lc.numAttrs;
+    }
+    cluster = 0;
     cudaError_t e = cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
     if (prof) cudaEventRecord(ev.end, st);
     if (e != cudaSuccess) {
@@ -608,8 +618,8 @@ int skinny(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_
 // kernel; `smem`: its dynamic shared memory.  The number of CTAs that fit on the device at once is asked of the
 // runtime once per kernel and device.
 template <void (*kernel)(const AttnDecArgs)>
-void launch_attn_decode(Launcher& L, thinfer_ctx* c, int unit, int smem, int pairs_per_request, AttnDecArgs a,
-                        int batch, int t_len) {
+void launch_attn_decode(Launcher& L, thinfer_ctx* c, int unit, int smem, int max_cluster, int pairs_per_request,
+                        AttnDecArgs a, int batch, int t_len) {
   static SmemOptIn opt;
   static int per_sm[SmemOptIn::kMaxDevices] = {};
   if (smem > 0 && !opt.ensure(kernel, smem)) {
@@ -636,8 +646,19 @@ void launch_attn_decode(Launcher& L, thinfer_ctx* c, int unit, int smem, int pai
   grid = std::min(grid, static_cast<long long>(kAttnMaxSplits - 2) * a.n_pairs);
   // Every segment costs a query load, a merge and a ticket.  When a whole number of equal segments per pair
   // fills at least 80 % of the slots, that grid (every CTA exactly one segment) beats the exactly balanced one.
-  const long long per_pair = grid / a.n_pairs;
-  if (per_pair >= 1 && per_pair * a.n_pairs * 10 >= slots * 8) grid = per_pair * a.n_pairs;
+  long long per_pair = grid / a.n_pairs;
+  bool aligned = per_pair >= 1 && per_pair * a.n_pairs * 10 >= slots * 8;
+  // A pair whose segments fit one thread-block cluster merges them in shared memory of the cluster instead of
+  // through L2 and a ticket.  Small problems (a few units per CTA: all latency) take that route even when it
+  // leaves slots empty.
+  if (c->attn_cluster && per_pair >= 2 &&
+      ((aligned && per_pair <= max_cluster) || a.units_per_pair <= 4LL * max_cluster)) {
+    per_pair = std::min<long long>(per_pair, max_cluster);
+    aligned = true;
+    a.cluster = static_cast<int>(per_pair);
+    L.cluster = a.cluster;
+  }
+  if (aligned) grid = per_pair * a.n_pairs;
   L.go(THINFER_K_ATTN, kernel, dim3(static_cast<unsigned>(grid)), dim3(kAttnDecWarps * 32), smem, a);
 }
 
@@ -645,10 +666,11 @@ template <int D, int G>
 void attn_decode_dg(Launcher& L, thinfer_ctx* c, const AttnDecArgs& a, int batch, int t_len) {
   if constexpr (G >= 4) {
     // grouped-query models: the G heads of a pair are the rows of a tensor-core tile
-    launch_attn_decode<attn_decode_gqa_kernel<D, G>>(L, c, kGqaUnit, gqa_ring_bytes<D>(), a.n_q_heads / G, a, batch, t_len);
+    launch_attn_decode<attn_decode_gqa_kernel<D, G>>(L, c, kGqaUnit, gqa_smem_bytes<D, G>(), kGqaMaxCluster, a.n_q_heads / G, a,
+                                                     batch, t_len);
   } else {
     constexpr int kUnit = kAttnDecWarps * kAttnDecUnroll * (32 / (D / 8));
-    launch_attn_decode<attn_decode_kernel<D, G>>(L, c, kUnit, 0, a.n_q_heads / G, a, batch, t_len);
+    launch_attn_decode<attn_decode_kernel<D, G>>(L, c, kUnit, 0, kAttnMaxCluster, a.n_q_heads / G, a, batch, t_len);
   }
 }
 
@@ -1319,6 +1341,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     };
     c->attn_waves = env_int("THINFER_ATTN_WAVES", 1, 8, c->attn_waves);
     c->attn_min_units = env_int("THINFER_ATTN_MIN_UNITS", 1, 64, c->attn_min_units);
+    c->attn_cluster = env_int("THINFER_ATTN_CLUSTER", 0, 1, c->attn_cluster);
     c->sk_max_tiles = env_int("THINFER_SK_MAX_TILES", 1, 7, 0);
     c->trace_cta_kid = env_int("THINFER_TRACE_CTA_KID", 0, THINFER_K_COUNT - 1, -1);
   }
