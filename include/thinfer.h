@@ -307,6 +307,16 @@ int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, vo
                                  int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t seq,
                                  int32_t kv_stride, int32_t head_dim, void* cuda_stream);
 
+/* Decode attention alone (Eq. 6 for one query row per request and head, Section 3.4.1: per request, over its own
+ * cache), for parity tests of the split-KV schedules: q device FP16 [batch, n_q_heads, head_dim] (already rotated)
+ * attends the first t_len positions of every request in the K/V cache of (`slot`, `layer`) of `ctx` - written
+ * beforehand by a prefill, or directly through thinfer_kv_pointer - and out device FP16 [batch, n_q_heads*head_dim]
+ * receives the result.  seq_lens (host int32 [batch], may be NULL): request b attends seq_lens[b] keys instead
+ * (the slot's per-request length array on the device is overwritten: use a slot that holds no ragged sequence).
+ * Uses the context's split-KV scratch: order it with the context's other work. */
+int thinfer_op_attention_decode(thinfer_ctx* ctx, int32_t slot, int32_t layer, const void* q, void* out, int32_t batch,
+                                int32_t t_len, const int32_t* seq_lens, void* cuda_stream);
+
 /* Greedy pick of the stack's last step (the paper is silent on sampling): ids[r] = the lowest index at
  * which logits[r, :] is largest.  logits device FP32 [rows, n]; ids device int32 [rows]. */
 int thinfer_op_argmax(const void* logits, void* ids, int32_t rows, int32_t n, void* cuda_stream);

@@ -1778,6 +1778,36 @@ int thinfer_op_attention_prefill(const void* q, const void* k, const void* v, vo
   return L.rc;
 }
 
+int thinfer_op_attention_decode(thinfer_ctx* c, int32_t slot, int32_t layer, const void* q, void* out, int32_t batch,
+                                int32_t t_len, const int32_t* seq_lens, void* cuda_stream) {
+  if (c == nullptr) return THINFER_EINVAL;
+  const thinfer_config& cf = c->cfg;
+  if (q == nullptr || out == nullptr || slot < 0 || slot >= cf.buf_slots || layer < 0 || layer >= cf.n_layers)
+    return fail(c, THINFER_EINVAL, "NULL pointer, or slot / layer out of range");
+  if (batch < 1 || batch > cf.max_batch) return fail(c, THINFER_ECAPACITY, "batch %d outside [1, %d]", batch, cf.max_batch);
+  int longest = t_len;
+  if (seq_lens != nullptr) {
+    longest = 0;
+    for (int b = 0; b < batch; ++b) {
+      if (seq_lens[b] < 1 || seq_lens[b] > cf.max_seq) return fail(c, THINFER_ECAPACITY, "seq_lens[%d] = %d", b, seq_lens[b]);
+      longest = std::max(longest, seq_lens[b]);
+    }
+  }
+  if (longest < 1 || longest > cf.max_seq) return fail(c, THINFER_ECAPACITY, "%d keys outside [1, %d]", longest, cf.max_seq);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int* lens_dev = nullptr;
+  if (seq_lens != nullptr) {
+    int* dst = c->slot_lens + static_cast<size_t>(slot) * cf.max_batch;
+    if (cudaMemcpyAsync(dst, seq_lens, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return fail(c, THINFER_ECUDA, "copying the key counts failed");
+    lens_dev = dst;
+  }
+  Launcher L{c, st};
+  attn_decode(L, c, static_cast<const half_t*>(q), kv_ptr(c, slot, layer, 0), kv_ptr(c, slot, layer, 1),
+              static_cast<half_t*>(out), batch, longest, lens_dev, 0);
+  return L.rc;
+}
+
 int thinfer_op_argmax(const void* logits, void* ids, int32_t rows, int32_t n, void* cuda_stream) {
   if (logits == nullptr || ids == nullptr || rows <= 0 || n <= 0) return THINFER_EINVAL;
   Launcher L{nullptr, static_cast<cudaStream_t>(cuda_stream)};

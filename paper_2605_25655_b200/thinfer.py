@@ -27,7 +27,7 @@ EXPORTS = (
     "thinfer_kv_pointer", "thinfer_status", "thinfer_clear_status", "thinfer_capture_hidden", "thinfer_set_launch_mode", "thinfer_profile_select",
     "thinfer_profile_read", "thinfer_trace_unified", "thinfer_launch_count", "thinfer_last_error", "thinfer_destroy",
     "thinfer_op_linear", "thinfer_op_linear_noalloc", "thinfer_op_attention_prefill", "thinfer_op_rmsnorm",
-    "thinfer_op_argmax", "thinfer_selftest_bounded_wait",
+    "thinfer_op_argmax", "thinfer_op_attention_decode", "thinfer_selftest_bounded_wait",
 )
 
 
@@ -108,6 +108,7 @@ def lib(storage="f16"):
     L.thinfer_op_attention_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
     L.thinfer_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, C.c_float, vp]
     L.thinfer_op_argmax.argtypes = [vp, vp, i32, i32, vp]
+    L.thinfer_op_attention_decode.argtypes = [vp, i32, i32, vp, vp, i32, i32, C.POINTER(i32), vp]
     L.thinfer_selftest_bounded_wait.argtypes = [vp, i64, vp]
     _libs[storage] = L
     return L
@@ -265,6 +266,15 @@ class Context:
 
     def clear_status(self):
         _check(self.L.thinfer_clear_status(self.h), self.h, self.storage)
+
+    def attention_decode(self, q, t_len, slot=0, layer=0, seq_lens=None, stream=None):
+        """Decode attention alone over the cache of (slot, layer): q [batch, n_q_heads, head_dim] -> [batch, n_q_heads*d]."""
+        batch = int(q.shape[0])
+        out = self.torch.empty(batch, self.shape.n_q_heads * self.shape.head_dim, dtype=q.dtype, device=q.device)
+        lens = (C.c_int32 * batch)(*[int(v) for v in seq_lens]) if seq_lens is not None else None
+        _check(self.L.thinfer_op_attention_decode(self.h, slot, layer, q.data_ptr(), out.data_ptr(), batch, int(t_len),
+                                                  lens, _stream_ptr(stream)), self.h, self.storage)
+        return out
 
     def selftest_bounded_wait(self, limit_ns=1_000_000, stream=None):
         _check(self.L.thinfer_selftest_bounded_wait(self.h, int(limit_ns), _stream_ptr(stream)), self.h, self.storage)

@@ -151,3 +151,37 @@ def test_argmax_exact_ties_go_to_the_lowest_index(T):
     # odd row length, fewer columns than threads
     small = np.array([[0.0, 2.0, 2.0, -1.0, 2.0]], dtype=np.float32)
     assert int(thinfer.op_argmax(torch.from_numpy(small).cuda()).cpu()[0]) == 1
+
+
+# heads, KV heads, head_dim: FMA kernel with 1 and 2 query heads per KV head, tensor-core kernel with 4 and 8
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 128), (8, 4, 64), (8, 2, 128), (8, 1, 64), (16, 2, 128), (32, 32, 128)])
+def test_decode_attention_schedules(T, hq, hkv, d):
+    # the split-KV schedules of decode attention on their own, over many (batch, key count) combinations: one
+    # segment per pair, equal segments merged in a thread-block cluster (2 .. 8 CTAs), equal segments merged through
+    # a ticket, exactly balanced runs that cross pair boundaries, ragged key counts, single keys
+    from paper_2605_25655_b200 import synth
+    torch, thinfer = T
+    shape = synth.Shape(hidden=hq * d, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, ffn=64)
+    max_b, max_t = 16, 2100
+    w = {n: torch.zeros(synth.layer_tensor_shape(shape, n), dtype=torch.float16, device="cuda") for n in synth.LAYER_TENSORS}
+    ctx = thinfer.Context(shape, [w], None, max_batch=max_b, max_seq=max_t)
+    rng = np.random.default_rng(hq * 1000 + hkv * 10 + d)
+    k_np = rng.standard_normal((max_b, hkv, max_t, d)).astype(np.float16)
+    v_np = rng.standard_normal((max_b, hkv, max_t, d)).astype(np.float16)
+    ctx.kv_view(0, 0, 0).copy_(torch.from_numpy(k_np))
+    ctx.kv_view(0, 0, 1).copy_(torch.from_numpy(v_np))
+    cases = [(1, 1), (1, 33), (2, 64), (3, 65), (16, 31), (5, 129), (1, 2100), (16, 640), (7, 1023), (16, 1279), (4, 528),
+             (9, 257), (2, 2047), (12, 96)]
+    cases += [(int(rng.integers(1, 17)), int(rng.integers(1, max_t + 1))) for _ in range(10)]
+    for batch, t_len in cases:
+        q_np = (rng.standard_normal((batch, hq, d)) * 1.5).astype(np.float16)
+        ragged = (batch * 7 + t_len) % 3 == 0
+        lens = [int(rng.integers(1, t_len + 1)) for _ in range(batch)] if ragged else None
+        out = ctx.attention_decode(torch.from_numpy(q_np).cuda(), t_len, seq_lens=lens).cpu().numpy()
+        for b in range(batch):
+            n = lens[b] if ragged else t_len
+            ref = O.decode_attention(q_np[b], k_np[b, :, :n], v_np[b, :, :n])
+            assert_rows_close(out[b].reshape(hq, d), ref.reshape(hq, d),
+                              f"decode attention {hq}q/{hkv}kv d={d} batch {batch} keys {n} (request {b})", max_err=6e-3)
+    assert ctx.status() == 0
+    ctx.close()
