@@ -137,6 +137,7 @@ struct thinfer_ctx {
   int max_splits = 1;
   int attn_waves = 1, attn_min_units = 2;  // split-KV schedule of decode attention (tuning aids)
   int attn_cluster = 1;                    // merge the segments of a pair inside a thread-block cluster when they fit
+  int sk_whole_tiles = 1;                  // tuning aid: shrink the grid to shares of whole tiles when shares are ragged
   int sk_max_tiles = 0;                    // tuning aid: cap on the tiles of a skinny share (0: the built-in limits)
   int trace_cta_kid = -1;                  // kernel id whose CTAs log their own times while tracing is on
   // status word (pinned, mapped)
@@ -600,6 +601,18 @@ int skinny(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_
   while (a.tiles_max > max_tiles && grid < 64 * sms) {
     grid += sms;
     a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
+  }
+  // A share that walks tiles_max tiles but holds far fewer real rows (13B-shaped O and down projections: 17.3 rows
+  // in shares of 2 tiles) leaves half of every ring stage empty.  With a single matrix the grid may shrink instead,
+  // to shares of whole tiles: fewer CTAs, every stage full.
+  if (mats == 1 && !swiglu && a.tiles_max >= 2 && L.c != nullptr && L.c->sk_whole_tiles &&
+      static_cast<long long>(units) * 4 < 3LL * 8 * a.tiles_max * grid) {
+    const int tiles = (units + 7) / 8;
+    const int g2 = (tiles + a.tiles_max - 1) / a.tiles_max;
+    if (g2 >= sms) {  // at least one CTA per SM
+      grid = g2;
+      a.tiles_max = skinny_partition(n, swiglu, grid, a.cta0);
+    }
   }
   if (a.tiles_max > max_tiles) {
     L.rc = fail(L.c, THINFER_EUNSUPPORTED, "skinny projection: %d tiles per share", a.tiles_max);
@@ -1343,6 +1356,7 @@ int thinfer_create(const thinfer_config* cfg, const thinfer_weights* weights, vo
     c->attn_min_units = env_int("THINFER_ATTN_MIN_UNITS", 1, 64, c->attn_min_units);
     c->attn_cluster = env_int("THINFER_ATTN_CLUSTER", 0, 1, c->attn_cluster);
     c->sk_max_tiles = env_int("THINFER_SK_MAX_TILES", 1, 7, 0);
+    c->sk_whole_tiles = env_int("THINFER_SK_WHOLE_TILES", 0, 1, c->sk_whole_tiles);
     c->trace_cta_kid = env_int("THINFER_TRACE_CTA_KID", 0, THINFER_K_COUNT - 1, -1);
   }
 
