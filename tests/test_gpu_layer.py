@@ -229,8 +229,8 @@ def test_llama13b_layer_reduced_budget(T):
 
 def test_llama70b_layer_reduced_budget(T):
     # configuration 5's layer shape (hidden 8192, 64 query / 8 KV heads, FFN 28672) on a reduced token budget
+    # (batch 2 x 64 tokens of every one of the 80 layers is covered by tests/test_gpu_full_depth.py)
     shape = dataclasses.replace(synth.LLAMA_70B, n_layers=1, vocab=0)
-    _layer_case(T, shape, batch=2, seq=64, n_decode=2, seed=70)
     _layer_case(T, shape, batch=1, seq=3, n_decode=2, seed=71)        # batch 1: the FMA streaming path with 8:1 GQA
 
 
@@ -253,34 +253,6 @@ def test_llama7b_two_layer_stack_with_32000_vocab(T):
             ref_logits, _, caches, _ = O.stack_decode(cfg, sw, ids[:, t], caches, t)
             assert_rows_close(logits.cpu().numpy(), ref_logits, f"decode logits t={t}")
             _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), ref_logits)
-        assert ctx.status() == 0
-        ctx.close()
-
-
-def test_llama7b_eight_layer_stack_end_to_end_cosine(T):
-    # configuration 3's shapes at a quarter of its depth, end to end (the oracle runs on its own states, nothing
-    # is chained): final hidden-state cosine >= 0.999 per token, logits within the row-RMS tolerance, both for
-    # the per-unit decode path and for the unified decode kernel
-    torch, thinfer = T
-    shape = dataclasses.replace(synth.LLAMA_7B, n_layers=8)
-    cfg = oracle_config(shape)
-    sw = synth.stack_weights(shape, 11)
-    ids = synth.token_ids(shape, 11, (2, 66))
-    ref_logits0, _, caches, _ = O.stack_prefill(cfg, sw, ids[:, :64])
-    refs = []
-    for t in (64, 65):
-        lg, _, caches, hid = O.stack_decode(cfg, sw, ids[:, t], caches, t)
-        refs.append((lg, hid[-1]))
-    idd = torch.from_numpy(ids).cuda()
-    for mode in (1, 2):
-        ctx = _ctx(T, shape, sw["layers"], 2, 72, stack=sw)
-        ctx.set_launch_mode(mode)
-        _, logits = ctx.prefill(idd[:, :64].contiguous(), want_logits=True)
-        assert_rows_close(logits.cpu().numpy(), ref_logits0, f"mode {mode}: prefill logits after 8 layers")
-        for i, t in enumerate((64, 65)):
-            nxt, logits = ctx.decode_step(idd[:, t].contiguous(), want_logits=True)
-            assert_rows_close(logits.cpu().numpy(), refs[i][0], f"mode {mode}: decode logits t={t}")
-            _check_greedy(nxt.cpu().numpy(), logits.cpu().numpy(), refs[i][0])
         assert ctx.status() == 0
         ctx.close()
 

@@ -177,7 +177,10 @@ def test_decode_attention_schedules(T, hq, hkv, d):
         q_np = (rng.standard_normal((batch, hq, d)) * 1.5).astype(np.float16)
         ragged = (batch * 7 + t_len) % 3 == 0
         lens = [int(rng.integers(1, t_len + 1)) for _ in range(batch)] if ragged else None
-        out = ctx.attention_decode(torch.from_numpy(q_np).cuda(), t_len, seq_lens=lens).cpu().numpy()
+        qd = torch.from_numpy(q_np).cuda()
+        out = ctx.attention_decode(qd, t_len, seq_lens=lens).cpu().numpy()
+        again = ctx.attention_decode(qd, t_len, seq_lens=lens).cpu().numpy()
+        np.testing.assert_array_equal(out, again)       # segments are merged in a fixed order: no run-to-run noise
         for b in range(batch):
             n = lens[b] if ragged else t_len
             ref = O.decode_attention(q_np[b], k_np[b, :, :n], v_np[b, :, :n])
