@@ -367,6 +367,19 @@ struct SmemOptIn {
   }
 };
 
+// SM count of the current device for the context-free operator entry points (asked once per device)
+int current_sm_count() {
+  static int cached[SmemOptIn::kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= SmemOptIn::kMaxDevices) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 // ----------------------------------------------------------------------------
 // tcgen05 GEMM dispatch
 // ----------------------------------------------------------------------------
@@ -382,7 +395,7 @@ void launch_tc(Launcher& L, int kid, const CUtensorMap& w0, const CUtensorMap& w
   const int n_ft = a.tiles[0] + a.tiles[1] + a.tiles[2];
   const int n_tt = (a.rows + BN - 1) / BN;
   const int n_tiles = n_ft * n_tt;
-  int sms = L.c ? L.c->sm_count : 148;
+  int sms = L.c ? L.c->sm_count : current_sm_count();
   if (sms > kTcMaxCtas) sms = kTcMaxCtas;
   TcGemmArgs b = a;
   int grid = n_tiles < sms ? n_tiles : sms;
@@ -479,7 +492,7 @@ void gemv(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_t
   a.eps = eps;
   a.e = e;
   const int n_pairs = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
-  a.kslices = pick_kslices(n_pairs, k, L.c ? L.c->sm_count : 148);
+  a.kslices = pick_kslices(n_pairs, k, L.c ? L.c->sm_count : current_sm_count());
   const int pairs_per_cta = kGemvWarps / a.kslices;
   const int gx = (n_pairs + pairs_per_cta - 1) / pairs_per_cta;
   const dim3 block(kGemvWarps * 32);
@@ -584,7 +597,7 @@ int skinny(Launcher& L, int kid, const half_t* w0, const half_t* w1, const half_
   }
   const int units = (EPI == EPI_SWIGLU) ? n[0] : (n[0] + n[1] + n[2]) / 2;
   const bool swiglu = EPI == EPI_SWIGLU;
-  const int sms = L.c ? L.c->sm_count : 148;
+  const int sms = L.c ? L.c->sm_count : current_sm_count();
   // Two CTAs per SM with a 4-stage ring per warp (a one-CTA variant with an 8-stage ring, tried for the two
   // projections with few features per SM, was slower); more CTAs when a share would exceed kSkMaxTiles tiles.
   const int mats = swiglu ? 1 : (n[0] > 0) + (n[1] > 0) + (n[2] > 0);
