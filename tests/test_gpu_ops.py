@@ -188,3 +188,31 @@ def test_decode_attention_schedules(T, hq, hkv, d):
                               f"decode attention {hq}q/{hkv}kv d={d} batch {batch} keys {n} (request {b})", max_err=6e-3)
     assert ctx.status() == 0
     ctx.close()
+
+
+def test_decode_attention_schedules_up_to_64_requests(T):
+    # the same sweep with the largest slots the library accepts (17 .. 64 requests: more pairs than CTA slots, so
+    # the exactly balanced runs cross pair boundaries), MHA and 4 query heads per KV head
+    from paper_2605_25655_b200 import synth
+    torch, thinfer = T
+    for hq, hkv, d in ((8, 8, 128), (8, 2, 64)):
+        shape = synth.Shape(hidden=hq * d, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, ffn=64)
+        max_b, max_t = 64, 700
+        w = {n: torch.zeros(synth.layer_tensor_shape(shape, n), dtype=torch.float16, device="cuda") for n in synth.LAYER_TENSORS}
+        ctx = thinfer.Context(shape, [w], None, max_batch=max_b, max_seq=max_t)
+        rng = np.random.default_rng(hq + d)
+        k_np = rng.standard_normal((max_b, hkv, max_t, d)).astype(np.float16)
+        v_np = rng.standard_normal((max_b, hkv, max_t, d)).astype(np.float16)
+        ctx.kv_view(0, 0, 0).copy_(torch.from_numpy(k_np))
+        ctx.kv_view(0, 0, 1).copy_(torch.from_numpy(v_np))
+        for batch, t_len, ragged in ((17, 300, False), (64, 700, False), (33, 129, True), (64, 65, True), (48, 1, False)):
+            q_np = (rng.standard_normal((batch, hq, d)) * 1.5).astype(np.float16)
+            lens = [int(rng.integers(1, t_len + 1)) for _ in range(batch)] if ragged else None
+            out = ctx.attention_decode(torch.from_numpy(q_np).cuda(), t_len, seq_lens=lens).cpu().numpy()
+            for b in (0, batch // 2, batch - 1):
+                n = lens[b] if ragged else t_len
+                ref = O.decode_attention(q_np[b], k_np[b, :, :n], v_np[b, :, :n])
+                assert_rows_close(out[b].reshape(hq, d), ref.reshape(hq, d),
+                                  f"decode attention {hq}q/{hkv}kv batch {batch} keys {n} (request {b})", max_err=6e-3)
+        assert ctx.status() == 0
+        ctx.close()
