@@ -77,13 +77,17 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "c5"    # the largest configuration that fits one GPU (138 GB of weights)
 
 
-def captured_traffic(key):
-    """DRAM bytes per launch from the committed ncu captures (profiles/ncu_traffic.json); None when the
-    kernel of this workload has no capture."""
+def captured(key, field="traffic_bytes"):
+    """A figure of the committed ncu captures (profiles/ncu_traffic.json): DRAM bytes per launch, tensor-pipe
+    activity, DRAM throughput; None when the kernel of this workload has no capture."""
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if not os.path.exists(path):
         return None
-    return json.load(open(path)).get(key, {}).get("traffic_bytes")
+    return json.load(open(path)).get(key, {}).get(field)
+
+
+def captured_traffic(key):
+    return captured(key, "traffic_bytes")
 
 
 def measured_peaks():
@@ -476,12 +480,14 @@ def run_ours(args, wl):
         "roofline": {"kernel": dec_kernel + " (decode gate/up projection)", "bound": "hbm",
                      "achieved": gu_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gu_gbs / hbm_peak,
                      "traffic": captured_traffic(f"decode_gateup_{wl.key}_b{B}"),
+                     "dram_throughput_pct_captured": captured(f"decode_gateup_{wl.key}_b{B}", "dram_throughput_pct"),
                      "traffic_kind": "captured (committed profile of the same launch, profiles/ncu_traffic.json)",
                      "peak_kind": peak_kind, "avg_us": ms_dec_gu * 1e3, "launches_timed": n_dgu,
                      "algorithmic_bytes": gateup_gemv_bytes(s, B), "frac_of_nominal_peak": gu_gbs / NOMINAL_GBS},
         "roofline_prefill": {"kernel": tc_pre_rows + " (prefill gate/up projection)", "bound": "tensor",
                              "achieved": gu_tflops, "peak": tc_burst, "unit": "TFLOP/s", "frac": gu_tflops / tc_burst,
                              "traffic": captured_traffic(f"prefill_gateup_{wl.key}_b{B}"),
+                             "tensor_pipe_active_pct_captured": captured(f"prefill_gateup_{wl.key}_b{B}", "tensor_pipe_active_pct"),
                              "traffic_kind": "captured (committed profile of the same launch, profiles/ncu_traffic.json)",
                              "peak_kind": peak_kind + " bf16 burst (the kernel is timed alone)",
                              "avg_us": ms_pre_gu * 1e3, "launches_timed": n_pgu,
