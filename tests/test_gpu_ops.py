@@ -153,8 +153,10 @@ def test_argmax_exact_ties_go_to_the_lowest_index(T):
     assert int(thinfer.op_argmax(torch.from_numpy(small).cuda()).cpu()[0]) == 1
 
 
-# heads, KV heads, head_dim: FMA kernel with 1 and 2 query heads per KV head, tensor-core kernel with 4 and 8
-@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 128), (8, 4, 64), (8, 2, 128), (8, 1, 64), (16, 2, 128), (32, 32, 128)])
+# heads, KV heads, head_dim: FMA kernel with 1 and 2 query heads per KV head, tensor-core kernel with 4 and 8;
+# 16 query heads per KV head (two groups of 8 read the same keys), 6 (groups of 2), 3 (odd: one head per pass)
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 128), (8, 4, 64), (8, 2, 128), (8, 1, 64), (16, 2, 128), (32, 32, 128),
+                                      (16, 1, 64), (12, 2, 64), (3, 1, 128)])
 def test_decode_attention_schedules(T, hq, hkv, d):
     # the split-KV schedules of decode attention on their own, over many (batch, key count) combinations: one
     # segment per pair, equal segments merged in a thread-block cluster (2 .. 8 CTAs), equal segments merged through
