@@ -10,6 +10,7 @@ rate (batch x generated / total latency, Section 3.4.1) and the roofline fractio
   python bench.py --config {c2,c3,c4,c5} ...               # 7B layer / 7B stack / 13B stack / 70B stack
   python bench.py --impl reference ...                      # the CPU oracle, timed on the host cores
   python bench.py --tables                                  # operator latencies at the paper's Table 8 / 9 shapes
+  python bench.py --pipeline --config c4                    # prefill of the next batch overlapped with decode (2 KV slots)
   python bench.py --profile {prefill,decode} --config cX    # one layer of that configuration: the case ncu captures
   python bench.py --profile stack --config cX               # two layers + head: the case of the ncu launch list
 
@@ -513,6 +514,66 @@ def run_ours(args, wl):
     return 0
 
 
+def run_pipeline(args, wl):
+    """The Prefill -> Buffer -> Decode schedule of Section 3.4.2 on one device, measured: two KV slots, the prefill
+    of the next batch on one stream while the current batch decodes on another (the library's hand-off events order
+    the stages of each slot), against the same work issued on a single stream.  Reports generated tokens / s of
+    both schedules; a side measurement, not the headline."""
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    if not wl.stack:
+        raise SystemExit("--pipeline needs a stack configuration (c3, c4, c5)")
+    B, s, n_dec = args.batch or wl.batch, wl.shape, wl.decode_steps
+    dev = torch.device("cuda", 0)
+    sw = synth.device_stack_weights(s, seed=0, device=dev)
+    ctx = thinfer.Context(s, sw["layers"], {n: sw[n] for n in ("embed", "final_norm", "lm_head")}, max_batch=B,
+                          max_seq=wl.prompt + n_dec, buf_slots=2, device=dev)
+    prompts = [torch.from_numpy(synth.token_ids(s, 0, (B, wl.prompt), stream=i)).to(dev) for i in range(2)]
+    bufs = [[torch.zeros(B, dtype=torch.int32, device=dev) for _ in range(2)] for _ in range(2)]
+    first = [torch.zeros(B, dtype=torch.int32, device=dev) for _ in range(2)]
+
+    def batches(n_batches, sp, sd):
+        # batch r lives in slot r % 2: its prefill is issued while batch r - 1 decodes
+        def prefill(r):  # every buffer is allocated up front: nothing is freed while another stream may still read it
+            return ctx.prefill(prompts[r % 2], slot=r % 2, stream=sp, out=first[r % 2])
+        outs = [None, None]
+        outs[0] = prefill(0)
+        for r in range(n_batches):
+            if r + 1 < n_batches:
+                outs[(r + 1) % 2] = prefill(r + 1)
+            cur = outs[r % 2]
+            for i in range(n_dec):
+                cur = ctx.decode_step(cur, slot=r % 2, stream=sd, out=bufs[r % 2][i & 1])
+            ctx.release_slot(r % 2, stream=sd)
+
+    n_batches = max(2, args.steps)
+    res = {}
+    for name in ("serial", "pipelined"):
+        if name == "serial":
+            sp = sd = torch.cuda.current_stream()
+        else:
+            sp, sd = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        batches(2, sp, sd)                       # warm-up
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        batches(n_batches, sp, sd)
+        torch.cuda.synchronize()
+        res[name] = time.perf_counter() - t0
+        if ctx.status() != 0:
+            raise SystemExit(f"device status {ctx.status()}")
+    tokens = n_batches * B * wl.gen
+    print(json.dumps({"pipeline": {"workload": wl.name(B), "batches": n_batches, "kv_slots": 2,
+                                   "tok_s": {k: tokens / v for k, v in res.items()},
+                                   "seconds": res,
+                                   "speedup_over_serial": {k: res["serial"] / v for k, v in res.items() if k != "serial"},
+                                   "is": "generated tokens / wall time over all batches, prefill included "
+                                         "(Section 3.4.1's throughput); pipelined = prefill of batch r + 1 on a second "
+                                         "stream while batch r decodes"}}))
+    ctx.close()
+    return 0
+
+
 def run_profile_stack(args, wl):
     """The launch list's case: a TWO-layer stack of the configuration with its vocabulary head, real batch and
     prompt - every kernel of the benchmark's step appears with the arguments it has in the full model (layer 0
@@ -641,11 +702,15 @@ def main():
                     help="run one small pass and exit (the cases ncu captures): one layer of the configuration, "
                          "prefill or decode phase; or a two-layer stack with the head (the launch list)")
     ap.add_argument("--profile-decode-steps", type=int, default=2)
+    ap.add_argument("--pipeline", action="store_true",
+                    help="measure the two-slot prefill / decode overlap of Section 3.4.2 against the serial schedule")
     ap.add_argument("--tables", action="store_true", help="operator micro-benchmarks at the paper's Table 8 / 9 shapes")
     args = ap.parse_args()
     wl = WORKLOADS[args.config]
     if args.tables:
         return run_tables(args)
+    if args.pipeline:
+        return run_pipeline(args, wl)
     if args.profile == "stack":
         return run_profile_stack(args, wl)
     if args.profile:

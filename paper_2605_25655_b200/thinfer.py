@@ -174,7 +174,7 @@ class Context:
         self.h = h
 
     # -- device-buffer calls ------------------------------------------------
-    def prefill(self, inp, slot=0, stream=None, want_logits=False):
+    def prefill(self, inp, slot=0, stream=None, want_logits=False, out=None):
         torch = self.torch
         batch, seq = int(inp.shape[0]), int(inp.shape[1])
         assert inp.is_cuda and inp.is_contiguous()
@@ -185,7 +185,7 @@ class Context:
                                          _stream_ptr(stream)), self.h, self.storage)
             return out
         assert inp.dtype == torch.int32
-        ids = torch.empty(batch, dtype=torch.int32, device=self.device)
+        ids = torch.empty(batch, dtype=torch.int32, device=self.device) if out is None else out
         logits = torch.empty(batch, self.shape.vocab, dtype=torch.float32, device=self.device) if want_logits else None
         _check(self.L.thinfer_prefill(self.h, slot, inp.data_ptr(), batch, seq, ids.data_ptr(),
                                      logits.data_ptr() if want_logits else None, _stream_ptr(stream)), self.h, self.storage)
