@@ -13,6 +13,7 @@ rate (batch x generated / total latency, Section 3.4.1) and the roofline fractio
   python bench.py --pipeline --config c4                    # prefill of the next batch overlapped with decode (2 KV slots)
   python bench.py --profile {prefill,decode} --config cX    # one layer of that configuration: the case ncu captures
   python bench.py --profile stack --config cX               # two layers + head: the case of the ncu launch list
+  python bench.py --profile attention --config cX --seq S   # the prefill attention operator alone, batch 4
 
 With N > 1 (under torchrun) every rank runs an independent replica of the same workload on its own GPU: the
 path has no exchange step, so there is no collective on the data path; times are the maximum over ranks.
@@ -627,6 +628,23 @@ def run_profile_case(args, wl):
     return 0
 
 
+def run_profile_attention(args, wl):
+    """The prefill attention operator alone at Table 9's shape (batch 4, the configuration's heads, `--seq` keys):
+    three launches, for an ncu capture at a sequence length no configuration reaches."""
+    import torch
+    from paper_2605_25655_b200 import thinfer
+    s, S = wl.shape, args.seq
+    g = torch.Generator(device="cuda").manual_seed(1)
+    q = torch.randn(4, s.n_q_heads, S, s.head_dim, device="cuda", dtype=torch.float16, generator=g)
+    k, v = (torch.randn(4, s.n_kv_heads, S, s.head_dim, device="cuda", dtype=torch.float16, generator=g) for _ in range(2))
+    out = thinfer.op_attention_prefill(q, k, v)
+    for _ in range(2):
+        thinfer.op_attention_prefill(q, k, v, out=out)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": "attention", "heads": [s.n_q_heads, s.n_kv_heads], "head_dim": s.head_dim, "seq": S}))
+    return 0
+
+
 # Operator latencies the paper prints for MT-3000 (one cluster for Linear; cluster count not stated for
 # attention), quoted for context beside the B200 numbers: Table 8 (FP16 Linear, input dim 4096, ms) and
 # Table 9 ("MT Attention", batch 4, head_dim 128, ms).
@@ -698,9 +716,11 @@ def main():
                     help="16-bit storage type of weights, activations and KV cache (the BF16 build of the library)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--profile", choices=["prefill", "decode", "stack"], default=None,
+    ap.add_argument("--profile", choices=["prefill", "decode", "stack", "attention"], default=None,
                     help="run one small pass and exit (the cases ncu captures): one layer of the configuration, "
-                         "prefill or decode phase; or a two-layer stack with the head (the launch list)")
+                         "prefill or decode phase; a two-layer stack with the head (the launch list); or the prefill "
+                         "attention operator alone at --seq keys")
+    ap.add_argument("--seq", type=int, default=4096, help="--profile attention: sequence length")
     ap.add_argument("--profile-decode-steps", type=int, default=2)
     ap.add_argument("--pipeline", action="store_true",
                     help="measure the two-slot prefill / decode overlap of Section 3.4.2 against the serial schedule")
@@ -713,6 +733,8 @@ def main():
         return run_pipeline(args, wl)
     if args.profile == "stack":
         return run_profile_stack(args, wl)
+    if args.profile == "attention":
+        return run_profile_attention(args, wl)
     if args.profile:
         return run_profile_case(args, wl)
     if args.impl == "reference":
