@@ -133,6 +133,22 @@ def test_attention_first_row_returns_v0_and_uniform_keys_give_running_mean(T):
     np.testing.assert_allclose(got, mean.transpose(1, 0, 2), rtol=0, atol=4e-3)
 
 
+@pytest.mark.parametrize("s,d", [(600, 128), (333, 64)])
+def test_attention_prefill_rescales_while_the_row_maximum_keeps_growing(T, s, d):
+    """Scores that rise by more than 2^8 from one 64-key tile to the next: the running maximum of every row is
+    replaced and the accumulated output rescaled in (nearly) every tile (Section 3.3.2's online form)."""
+    torch, thinfer = T
+    rng = np.random.default_rng(s + d)
+    q, k, v = _rand16(rng, (1, 2, s, d), 0.25), _rand16(rng, (1, 2, s, d), 0.25), _rand16(rng, (1, 2, s, d), 1.0)
+    # 0.2 * sqrt(d) / log2(e) per key in raw score units = 0.2 per key in the kernel's base-2 units: 12.8 per tile
+    slope = 0.2 * np.sqrt(d) / np.log2(np.e)
+    q[..., 0] = np.float16(4.0)
+    k[..., 0] = (np.arange(s) * slope / 4.0).astype(np.float16)[None, None, :]
+    out = thinfer.op_attention_prefill(torch.from_numpy(q).cuda(), torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda())
+    torch.cuda.synchronize()
+    assert_rows_close(out.cpu().numpy()[0], O.causal_attention(q[0], k[0], v[0]), f"growing maximum S={s} d={d}", max_err=6e-3)
+
+
 def test_argmax_exact_ties_go_to_the_lowest_index(T):
     torch, thinfer = T
     n = 32000
