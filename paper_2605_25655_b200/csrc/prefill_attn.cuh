@@ -41,6 +41,8 @@ constexpr int kAttnThreads = 352;  // two softmax groups of 128 + one MMA-issuin
 struct AttnPreArgs {
   half_t* out;  // [batch][seq_len][n_q_heads * D]
   int n_q_heads, n_kv_heads, seq_len;
+  int n_items;      // batch * n_q_heads: the (request, head) pairs
+  int chunk_items;  // (request, head) pairs whose K and V stay in L2 together
   float scale_log2;  // log2(e) / sqrt(D)
   int* status;
 };
@@ -87,8 +89,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qt = (a.seq_len + kAttnBQ - 1) / kAttnBQ;
   const int n_pairs = (n_qt + 1) / 2;
-  const int pair = n_pairs - 1 - blockIdx.x;  // longest rows first
-  const int h = blockIdx.y, b = blockIdx.z;
+  // CTAs are handed out in the order of their index.  Inside a chunk of (request, head) pairs whose K and V fit
+  // in L2 together, all pairs of query blocks with the most key tiles come first, then the next shorter ones: the
+  // SMs that finish early pick up short work, and every K/V tile is still fetched from memory once.
+  const int per_chunk = a.chunk_items * n_pairs;
+  const int chunk = blockIdx.x / per_chunk, in_chunk = blockIdx.x - chunk * per_chunk;
+  const int first_item = chunk * a.chunk_items, cnt = min(a.chunk_items, a.n_items - first_item);
+  const int pair = n_pairs - 1 - in_chunk / cnt;  // longest rows first
+  const int item = first_item + in_chunk % cnt;
+  const int h = item % a.n_q_heads, b = item / a.n_q_heads;
   const int hk = h / (a.n_q_heads / a.n_kv_heads);
   // causal: block t attends keys 0 .. q0_t + 127 (clipped to the sequence); a block past the sequence has no tiles
   int q0[2], n_kt[2];
