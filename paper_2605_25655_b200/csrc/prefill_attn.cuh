@@ -268,10 +268,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         tmem_st_wait();
       }
-      // this tile's P buffer was read by P(j-2) V_{j-2}
-      if (j >= 2) {
-        if (!mbar_wait(&bar_o[t * 2 + (j & 1)], ((j >> 1) - 1) & 1, a.status)) { ok = false; break; }
-      }
+      // This tile's P buffer was read by P(j-2) V_{j-2}.  That product was issued before S(j) by the same thread,
+      // and the arrival on bar_s that let this tile start follows every MMA issued before it: nothing to wait for.
       // weights, their row sum (FP32, two lanes per instruction), P as FP16 for the tensor core -> shared memory
       // (128-byte swizzle)
       uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
