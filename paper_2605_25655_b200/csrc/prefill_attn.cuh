@@ -6,9 +6,9 @@
 //   Stage 2  scale + softmax     one thread per query row reads its score row
 //                                from tensor memory (no cross-thread reduction
 //                                needed), FP32, online form across K/V tiles
-//   Stage 3  O_blk += P V_j      P is written to shared memory as FP16 in the
-//                                128-byte swizzled layout and fed back to
-//                                tcgen05.mma; O accumulates in tensor memory
+//   Stage 3  O_blk += P V_j      P is written back to tensor memory as packed
+//                                FP16 and is the A operand of tcgen05.mma from
+//                                there; O accumulates in tensor memory
 //
 // Scores and weights never leave the SM.  One CTA handles TWO blocks of 128
 // query rows of one (request, head), each owned by a group of four warps (one
@@ -48,8 +48,8 @@ struct AttnPreArgs {
 };
 
 __host__ __device__ constexpr int attn_pre_smem_bytes(int d) {
-  // 2 x Q (D/64 sub-tiles of 128 rows x 128 B) + 3 x (K + V) (D/64 sub-tiles of 64 keys x 128 B) + 2 x 2 x P + barriers
-  return (d / 64) * (2 * 16384 + 6 * 8192) + 4 * 16384 + 256;
+  // 2 x Q (D/64 sub-tiles of 128 rows x 128 B) + 3 x (K + V) (D/64 sub-tiles of 64 keys x 128 B) + barriers
+  return (d / 64) * (2 * 16384 + 6 * 8192) + 256;
 }
 
 template <int D>
@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   constexpr int Q_BYTES = SUB * 16384;
   constexpr int KV_SUB = kAttnBK * 128;       // one 64-column block of a K or V tile
   constexpr int KV_BYTES = SUB * KV_SUB;
-  constexpr int P_BYTES = kAttnBQ * kAttnBK * 2;
+  constexpr uint32_t TM_P = 384;              // P buffers: 32 columns (64 packed weights) per block and buffer
   constexpr int NBUF = 3;
   constexpr int TMEM_COLS = 512;
   constexpr uint32_t IDESC_S = idesc_f16(128, kAttnBK, 0, 0);  // Q (K-major) x K^T (K-major)
@@ -72,13 +72,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   uint8_t* sm_q = smem;                        // [2] query blocks
   uint8_t* sm_k = sm_q + 2 * Q_BYTES;          // [NBUF]
   uint8_t* sm_v = sm_k + NBUF * KV_BYTES;      // [NBUF]
-  uint8_t* sm_p = sm_v + NBUF * KV_BYTES;      // [2 blocks][2 buffers] x 128 rows x 64 keys
-  uint64_t* bar_q = reinterpret_cast<uint64_t*>(sm_p + 4 * P_BYTES);
+  uint64_t* bar_q = reinterpret_cast<uint64_t*>(sm_v + NBUF * KV_BYTES);
   uint64_t* bar_kv = bar_q + 1;          // [NBUF]     tile loaded (transaction bytes)
   uint64_t* bar_free = bar_kv + NBUF;    // [2][NBUF]  block t has finished with the tile in this ring slot
   uint64_t* bar_s = bar_free + 2 * NBUF; // [2]        scores of block t complete in tensor memory
   uint64_t* bar_sf = bar_s + 2;          // [2]        group t holds its score row in registers
-  uint64_t* bar_p = bar_sf + 2;          // [2][2]     weights written to P buffer
+  uint64_t* bar_p = bar_sf + 2;          // [2][2]     weights written to P buffer (tensor memory)
   uint64_t* bar_o = bar_p + 4;           // [2][2]     the P V product that read P buffer is complete
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_o + 4);
   if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled tiles need 1024-byte alignment
@@ -150,7 +149,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   tc_fence_after();
   pdl_wait();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
-  // tensor-memory columns: S0 0..63, S1 64..127, O0 128..255, O1 256..383
+  // tensor-memory columns: S0 0..63, S1 64..127, O0 128..255, O1 256..383, P[block][buffer] 384 + 64 block + 32 buffer
 
   if (warp == 10) {
     if (lane == 0) {
@@ -169,7 +168,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       // Descriptors differ only in the start-address field (bits 0..13, bytes >> 4): one base each, offsets added.
       const uint64_t dq0 = smem_desc_sw128(smem_u32(sm_q + t * Q_BYTES), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm_k), 16, 1024);
-      const uint64_t dp0 = smem_desc_sw128(smem_u32(sm_p + t * 2 * P_BYTES), 16, 1024);
+      const uint32_t tm_p = tmem_base + TM_P + t * 64;
       const uint64_t dv0 = smem_desc_sw128(smem_u32(sm_v), KV_SUB, 1024);
       const uint32_t tm_s = tmem_base + t * 64, tm_o = tmem_base + 128 + t * 128;
       const int n_t = t ? n_kt[1] : n_kt[0];
@@ -184,13 +183,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         tc_commit(&bar_s[t]);
       };
       auto issue_pv = [&](int j) {  // Stage 3: O_t += P_t V_j
-        // P: 32 bytes per K=16 step inside the 128-byte row.  V: rows are keys (128 B each = 64 head
-        // elements), 16 keys per step; the next 64 head elements are one sub-tile further (leading offset)
-        const uint64_t dp = dp0 + static_cast<uint64_t>((j & 1) * (P_BYTES >> 4));
+        // P: 8 tensor-memory columns per K=16 step.  V: rows are keys (128 B each = 64 head elements), 16 keys
+        // per step; the next 64 head elements are one sub-tile further (leading offset)
+        const uint32_t ap = tm_p + (j & 1) * 32;
         const uint64_t dv = dv0 + static_cast<uint64_t>((j % NBUF) * (KV_BYTES >> 4));
 #pragma unroll
         for (int ks = 0; ks < kAttnBK / 16; ++ks)
-          tc_mma_f16(tm_o, dp + ks * (32 >> 4), dv + ks * (2048 >> 4), IDESC_O, (j | ks) != 0);
+          tc_mma_f16_ts(tm_o, ap + ks * 8, dv + ks * (2048 >> 4), IDESC_O, (j | ks) != 0);
         tc_commit(&bar_o[t * 2 + (j & 1)]);
         tc_commit(&bar_free[t * NBUF + j % NBUF]);
       };
@@ -270,14 +269,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       }
       // This tile's P buffer was read by P(j-2) V_{j-2}.  That product was issued before S(j) by the same thread,
       // and the arrival on bar_s that let this tile start follows every MMA issued before it: nothing to wait for.
-      // weights, their row sum (FP32, two lanes per instruction), P as FP16 for the tensor core -> shared memory
-      // (128-byte swizzle)
+      // weights, their row sum (FP32, two lanes per instruction), P as packed FP16 for the tensor core -> tensor
+      // memory (lane = row, two weights per column)
       uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
-      uint8_t* prow = sm_p + (t * 2 + (j & 1)) * P_BYTES + row * 128;
+      uint32_t pk[32];
       const uint64_t scale2 = f32x2(a.scale_log2, a.scale_log2), neg_m2 = f32x2(-m, -m);
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        uint32_t pk[16];
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           const uint32_t s0 = half == 0 ? r0[c] : r1[c];
@@ -291,17 +289,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
           sum2[(c >> 1) & 3] = add_f32x2(sum2[(c >> 1) & 3], f32x2(p0, p1));
           const half2_t hp = f2_to_h2(p0, p1);
-          pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&hp);
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int phys = (half * 4 + i) ^ (row & 7);
-          *reinterpret_cast<uint4*>(prow + phys * 16) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+          pk[half * 16 + (c >> 1)] = *reinterpret_cast<const uint32_t*>(&hp);
         }
       }
+      tmem_st32(lane_addr + TM_P + t * 64 + (j & 1) * 32, pk);
+      tmem_st_wait();
       const float2 sum = f32x2_unpack(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])));
       l = l * alpha + (sum.x + sum.y);
-      fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(&bar_p[t * 2 + (j & 1)]);
     }
