@@ -100,7 +100,9 @@ def test_rmsnorm(T, rows, n):
 # batch, q heads, kv heads, seq, cache stride, head_dim
 ATTN_SHAPES = [(1, 4, 4, 32, 40, 64), (2, 4, 2, 128, 128, 128), (1, 2, 2, 129, 200, 128), (2, 8, 2, 300, 384, 64),
                (1, 32, 32, 512, 640, 128), (1, 1, 1, 1, 8, 128), (1, 2, 1, 77, 77, 64),
-               (1, 2, 2, 1024, 1024, 128), (1, 2, 1, 4096, 4096, 128), (1, 1, 1, 2049, 2100, 64)]
+               (1, 2, 2, 1024, 1024, 128), (1, 2, 1, 4096, 4096, 128), (1, 1, 1, 2049, 2100, 64),
+               # eight query heads per KV head; 40 (request, head) pairs walked longest first in two chunks (32 + 8)
+               (1, 16, 2, 700, 704, 128), (1, 40, 40, 2048, 2048, 128)]
 
 
 @pytest.mark.parametrize("b,hq,hkv,s,t,d", ATTN_SHAPES)
